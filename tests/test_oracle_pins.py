@@ -1,0 +1,410 @@
+"""Pins for the CPU oracle: each test checks it against something other than itself
+(finite differences, closed forms, library routines, brute force, invariants)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import mslt_oracle as O
+from paper_2011_13635_b200 import inputs as I
+
+TINY = I.StageConfig("pin", hidden=8, heads=2, ffn=16, vocab=11, max_pos=6, layers=2, trainable=1,
+                     batch=2, seq=5, pred=3, dtype="fp32", varlen=(3, 5), seed_index=77)
+
+
+def tiny_model(cfg=TINY, std=0.3, top_k=None, seed=5):
+    w = I.make_weights(cfg, seed=seed, variant="parity", std=std)
+    m = O.MsltOracle(w, cfg.heads, ln_eps=1e-12)
+    m.set_trainable(cfg.trainable if top_k is None else top_k)
+    return m
+
+
+def tiny_batch(cfg=TINY, seed=9):
+    return I.make_batch(cfg, seed=seed)
+
+
+# -- backward formulas: central finite differences on every trainable element ---------------
+
+@pytest.mark.parametrize("top_k", [0, 1, 2])
+def test_gradients_match_finite_differences(top_k):
+    m = tiny_model(top_k=top_k)
+    tok, lens, pos, lab = tiny_batch()
+    assert lens.min() < TINY.seq, "the case must contain padding"
+    loss, g = m.loss_and_grads(tok, lens, pos, lab)
+    assert set(g.keys()) == set(m.trainable_names())
+    h = 1e-5
+    for name in m.trainable_names():
+        w = m.p[name]
+        fd = np.zeros_like(w)
+        it = np.nditer(w, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = w[idx]
+            w[idx] = keep + h
+            lp = m.loss(tok, lens, pos, lab)
+            w[idx] = keep - h
+            lm = m.loss(tok, lens, pos, lab)
+            w[idx] = keep
+            fd[idx] = (lp - lm) / (2 * h)
+        scale = max(np.abs(fd).max(), 1e-8)
+        err = np.abs(fd - g[name]).max() / scale
+        assert err < 1e-6, (name, err)
+        if name != "emb.pos":      # rows past S are legitimately zero
+            assert np.abs(g[name]).max() > 0, name
+
+
+def test_frozen_tensor_has_gradient_but_is_not_updated():
+    m = tiny_model(top_k=1)
+    tok, lens, pos, lab = tiny_batch()
+    name = "layer.0.ffn1.weight"
+    w = m.p[name]
+    keep = w[0, 0]
+    w[0, 0] = keep + 1e-5
+    lp = m.loss(tok, lens, pos, lab)
+    w[0, 0] = keep - 1e-5
+    lm = m.loss(tok, lens, pos, lab)
+    w[0, 0] = keep
+    assert abs(lp - lm) > 1e-12          # the loss does depend on it
+    before = {k: v.copy() for k, v in m.p.items()}
+    for _ in range(3):
+        m.step(tok, lens, pos, lab)
+    for k in before:
+        frozen = k.startswith("emb.") or k.startswith("layer.0.")
+        same = np.array_equal(before[k], m.p[k])
+        assert same == frozen, k
+
+
+# -- forward conventions against library routines ----------------------------------------------
+
+def test_encoder_layer_matches_torch_transformer_encoder_layer():
+    cfg = TINY
+    m = tiny_model()
+    rng = np.random.default_rng(0)
+    x = rng.standard_normal((cfg.batch, cfg.seq, cfg.hidden))
+    lens = np.array([3, 5])
+    ref = torch.nn.TransformerEncoderLayer(cfg.hidden, cfg.heads, cfg.ffn, dropout=0.0,
+                                           activation="gelu", layer_norm_eps=1e-12,
+                                           batch_first=True, norm_first=False).double()
+    P = lambda t: torch.from_numpy(m.p["layer.1." + t])
+    with torch.no_grad():
+        ref.self_attn.in_proj_weight.copy_(P("qkv.weight"))
+        ref.self_attn.in_proj_bias.copy_(P("qkv.bias"))
+        ref.self_attn.out_proj.weight.copy_(P("out.weight"))
+        ref.self_attn.out_proj.bias.copy_(P("out.bias"))
+        ref.norm1.weight.copy_(P("ln1.gamma")); ref.norm1.bias.copy_(P("ln1.beta"))
+        ref.linear1.weight.copy_(P("ffn1.weight")); ref.linear1.bias.copy_(P("ffn1.bias"))
+        ref.linear2.weight.copy_(P("ffn2.weight")); ref.linear2.bias.copy_(P("ffn2.bias"))
+        ref.norm2.weight.copy_(P("ln2.gamma")); ref.norm2.bias.copy_(P("ln2.beta"))
+    ref.train()   # keeps torch on its plain (non-fused, non-nested) path; dropout is 0
+    pad = torch.from_numpy(np.arange(cfg.seq)[None, :] >= lens[:, None])
+    want = ref(torch.from_numpy(x), src_key_padding_mask=pad).detach().numpy()
+    got, _ = m._layer_forward(1, x, lens)
+    for b in range(cfg.batch):           # rows at padded positions are unspecified
+        np.testing.assert_allclose(got[b, :lens[b]], want[b, :lens[b]], rtol=0, atol=1e-12)
+
+
+def test_head_and_loss_match_torch_functional():
+    m = tiny_model()
+    tok, lens, pos, lab = tiny_batch()
+    x, _, _ = m.encode(tok, lens)
+    F = torch.nn.functional
+    xt = torch.from_numpy(x)
+    rows, labels = [], []
+    for b in range(tok.shape[0]):
+        for j in range(pos.shape[1]):
+            if pos[b, j] >= 0:
+                rows.append(xt[b, pos[b, j]]); labels.append(int(lab[b, j]))
+    hm = torch.stack(rows)
+    T = lambda n: torch.from_numpy(m.p[n])
+    t = F.gelu(F.linear(hm, T("head.transform.weight"), T("head.transform.bias")))
+    t = F.layer_norm(t, (TINY.hidden,), T("head.ln.gamma"), T("head.ln.beta"), eps=1e-12)
+    logits = F.linear(t, T("emb.word"), T("head.decoder.bias"))
+    want = F.cross_entropy(logits, torch.tensor(labels)).item()
+    assert abs(m.loss(tok, lens, pos, lab) - want) < 1e-12
+
+
+def test_embedding_matches_torch():
+    m = tiny_model()
+    tok, _, _, _ = tiny_batch()
+    F = torch.nn.functional
+    e = F.embedding(torch.from_numpy(tok.astype(np.int64)), torch.from_numpy(m.p["emb.word"]))
+    e = e + torch.from_numpy(m.p["emb.pos"][: tok.shape[1]])
+    want = F.layer_norm(e, (TINY.hidden,), torch.from_numpy(m.p["emb.ln.gamma"]),
+                        torch.from_numpy(m.p["emb.ln.beta"]), eps=1e-12).numpy()
+    got, _ = m._embed(tok)
+    np.testing.assert_allclose(got, want, atol=1e-12, rtol=0)
+
+
+def test_gelu_values_and_derivative():
+    # Phi(1) = 0.841344746068543 (standard normal table), so gelu(1) = Phi(1)
+    assert abs(O.gelu(np.array([1.0]))[0] - 0.841344746068543) < 1e-14
+    assert O.gelu(np.array([0.0]))[0] == 0.0
+    u = np.linspace(-4, 4, 41)
+    fd = (O.gelu(u + 1e-6) - O.gelu(u - 1e-6)) / 2e-6
+    np.testing.assert_allclose(O.gelu_grad(u), fd, atol=1e-9)
+    # the tanh approximation is visibly different: the exact form is what is used
+    tanh_form = 0.5 * u * (1 + np.tanh(math.sqrt(2 / math.pi) * (u + 0.044715 * u ** 3)))
+    assert np.abs(tanh_form - O.gelu(u)).max() > 1e-4
+
+
+# -- softmax and LayerNorm invariants -------------------------------------------------------------
+
+def test_softmax_rows_sum_to_one_and_mask_is_exact_zero():
+    rng = np.random.default_rng(1)
+    sc = rng.standard_normal((3, 2, 7, 7)) * 5
+    lens = np.array([7, 4, 1])
+    p = O.masked_softmax(sc, lens)
+    np.testing.assert_allclose(p.sum(-1), 1.0, atol=1e-14)
+    for b, n in enumerate(lens):
+        assert np.all(p[b, :, :, n:] == 0.0)
+        assert np.all(p[b, :, :, :n] > 0.0)
+    assert np.all(p[2, :, :, 0] == 1.0)        # a single valid key takes all the mass
+
+
+def test_single_token_sequence_context_equals_value():
+    cfg = I.scaled(TINY, seq=1, batch=1, varlen=None, pred=1)
+    m = tiny_model(cfg)
+    x = np.random.default_rng(2).standard_normal((1, 1, cfg.hidden))
+    _, st = m._layer_forward(0, x, np.array([1]))
+    v = st["v"].transpose(0, 2, 1, 3).reshape(1, 1, cfg.hidden)
+    np.testing.assert_allclose(st["c"], v, atol=1e-15)
+
+
+def test_layer_norm_moments():
+    rng = np.random.default_rng(3)
+    z = rng.standard_normal((5, 64)) * 3 + 2
+    y, xhat, _ = O.layer_norm(z, np.ones(64), np.zeros(64), 1e-12)
+    np.testing.assert_allclose(xhat.mean(-1), 0, atol=1e-13)
+    np.testing.assert_allclose((xhat ** 2).mean(-1), 1, atol=1e-10)
+    assert np.array_equal(y, xhat)
+    g = rng.standard_normal(64); b = rng.standard_normal(64)
+    y2, _, _ = O.layer_norm(z, g, b, 1e-12)
+    np.testing.assert_allclose(y2, xhat * g + b, atol=1e-15)
+
+
+# -- loss closed forms ----------------------------------------------------------------------------
+
+def test_zero_decoder_gives_log_vocab():
+    for V in (11, 1024, 30522):
+        cfg = I.scaled(TINY, vocab=V)
+        w = I.make_weights(cfg, seed=4, std=0.3)
+        w["emb.word"][:] = 0
+        w["head.decoder.bias"][:] = 0
+        m = O.MsltOracle(w, cfg.heads)
+        tok, lens, pos, lab = I.make_batch(cfg, seed=4)
+        assert abs(m.loss(tok, lens, pos, lab) - math.log(V)) < 1e-12
+    assert abs(math.log(30522) - 10.326203) < 1e-6 and abs(math.log(1024) - 6.931472) < 1e-6
+
+
+def test_initial_loss_is_close_to_log_vocab():
+    cfg = I.scaled(I.CONFIGS["tiny"], batch=2)
+    m = O.MsltOracle(I.make_weights(cfg), cfg.heads)
+    tok, lens, pos, lab = I.make_batch(cfg)
+    assert abs(m.loss(tok, lens, pos, lab) - math.log(cfg.vocab)) < 0.15
+
+
+def test_cross_entropy_gradient_properties():
+    rng = np.random.default_rng(5)
+    logits = rng.standard_normal((6, 9)) * 3
+    labels = np.array([1, -1, 8, 0, -1, 3])
+    loss, dl = O.cross_entropy(logits, labels, 4)
+    np.testing.assert_allclose(dl.sum(-1), 0, atol=1e-15)      # each row sums to zero
+    assert np.all(dl[1] == 0) and np.all(dl[4] == 0)
+    # brute force, one slot at a time
+    want = 0.0
+    for r, y in enumerate(labels):
+        if y >= 0:
+            want += math.log(sum(math.exp(v) for v in logits[r])) - logits[r, y]
+    assert abs(loss - want / 4) < 1e-13
+    assert O.cross_entropy(logits, np.full(6, -1), 0)[0] == 0.0
+
+
+def test_head_only_training_is_softmax_regression_by_hand():
+    """top_k = 0: features are fixed, so d loss / d decoder-bias = mean(softmax - onehot)
+    and d loss / d transform-weight follows by the chain rule, written out per slot."""
+    m = tiny_model(top_k=0)
+    tok, lens, pos, lab = tiny_batch()
+    _, g = m.loss_and_grads(tok, lens, pos, lab)
+    assert set(g) == set(O.HEAD_TENSORS)
+    x, _, _ = m.encode(tok, lens)
+    E, bv = m.p["emb.word"], m.p["head.decoder.bias"]
+    slots = [(b, j) for b in range(tok.shape[0]) for j in range(pos.shape[1]) if pos[b, j] >= 0]
+    dbv = np.zeros_like(bv)
+    for b, j in slots:
+        h = x[b, pos[b, j]]
+        u = m.p["head.transform.weight"] @ h + m.p["head.transform.bias"]
+        a = np.array([0.5 * t * (1 + math.erf(t / math.sqrt(2))) for t in u])
+        mu = a.mean(); var = ((a - mu) ** 2).mean()
+        t = m.p["head.ln.gamma"] * (a - mu) / math.sqrt(var + 1e-12) + m.p["head.ln.beta"]
+        z = E @ t + bv
+        s = np.exp(z - z.max()); s /= s.sum()
+        s[lab[b, j]] -= 1
+        dbv += s / len(slots)
+    np.testing.assert_allclose(g["head.decoder.bias"], dbv, atol=1e-14)
+
+
+# -- Adam closed forms ---------------------------------------------------------------------------------
+
+def test_adam_closed_forms():
+    rng = np.random.default_rng(6)
+    w = rng.standard_normal(50); g = rng.standard_normal(50)
+    z = np.zeros(50)
+    lr, eps = 1e-2, 1e-6
+    # step 1 with bias correction and no decay: dw = -lr * g / (|g| + eps)
+    w1, m1, v1 = O.adam_update(w, g, z, z, 1, lr, 0.9, 0.999, eps, 0.0, True)
+    np.testing.assert_allclose(w1 - w, -lr * g / (np.abs(g) + eps), atol=1e-15)
+    np.testing.assert_allclose(m1, 0.1 * g); np.testing.assert_allclose(v1, 0.001 * g * g)
+    # zero gradient: only the decay term moves the weight
+    w2, _, _ = O.adam_update(w, z, z, z, 1, lr, 0.9, 0.999, eps, 0.1, True)
+    np.testing.assert_allclose(w2, w * (1 - lr * 0.1), atol=1e-15)
+    # beta1 = beta2 = 0 without bias correction: sign-like step at any t
+    w3, _, _ = O.adam_update(w, g, rng.standard_normal(50), np.abs(rng.standard_normal(50)), 7,
+                             lr, 0.0, 0.0, eps, 0.0, False)
+    np.testing.assert_allclose(w3 - w, -lr * g / (np.abs(g) + eps), atol=1e-15)
+    # two steps with a constant gradient: m_hat = g, v_hat = g^2 again
+    wa, ma, va = O.adam_update(w, g, z, z, 1, lr, 0.9, 0.999, eps, 0.0, True)
+    wb, _, _ = O.adam_update(wa, g, ma, va, 2, lr, 0.9, 0.999, eps, 0.0, True)
+    np.testing.assert_allclose(wb - wa, -lr * g / (np.abs(g) + eps), atol=1e-14)
+
+
+def test_step_applies_decay_to_matrices_only():
+    m = tiny_model(top_k=0)
+    m.set_optimizer(lr=0.0)
+    tok, lens, pos, lab = tiny_batch()
+    before = {k: v.copy() for k, v in m.p.items()}
+    m.step(tok, lens, pos, lab)
+    for k in before:
+        assert np.array_equal(before[k], m.p[k])       # lr = 0 moves nothing
+    m2 = tiny_model(top_k=0)
+    m2.set_optimizer(lr=1e-3, weight_decay=0.5, beta1=0.0, beta2=0.0, bias_correction=0, eps=1e-6)
+    _, g = m2.loss_and_grads(tok, lens, pos, lab)
+    w0 = {k: v.copy() for k, v in m2.p.items()}
+    m2.step(tok, lens, pos, lab)
+    for n in O.HEAD_TENSORS:
+        wd = 0.5 if w0[n].ndim == 2 else 0.0
+        want = w0[n] - 1e-3 * (g[n] / (np.abs(g[n]) + 1e-6) + wd * w0[n])
+        np.testing.assert_allclose(m2.p[n], want, atol=1e-14)
+
+
+# -- staging ------------------------------------------------------------------------------------------------
+
+def test_truncated_gradients_equal_full_gradients_on_the_trainable_slice():
+    tok, lens, pos, lab = tiny_batch()
+    full = tiny_model(top_k=2)
+    _, gf = full.loss_and_grads(tok, lens, pos, lab)
+    for k in (0, 1):
+        part = tiny_model(top_k=k)
+        _, gp = part.loss_and_grads(tok, lens, pos, lab)
+        for n in gp:
+            np.testing.assert_allclose(gp[n], gf[n], atol=1e-15, rtol=0)
+        assert "emb.word" not in gp and "layer.0.qkv.weight" not in gp
+
+
+def test_add_layers_copies_top_layers_in_order():
+    cfg = I.scaled(TINY, layers=2)
+    w = I.make_weights(cfg, seed=5, std=0.3)
+    m = O.MsltOracle(w, cfg.heads, max_layers=4)
+    tok, lens, pos, lab = tiny_batch()
+    h_before, _ = m.forward(tok, lens)
+    m.add_layers(2)
+    assert m.L == 4
+    for t in O.LAYER_TENSORS:
+        assert np.array_equal(m.p[f"layer.2.{t}"], m.p[f"layer.0.{t}"])
+        assert np.array_equal(m.p[f"layer.3.{t}"], m.p[f"layer.1.{t}"])
+    assert not np.array_equal(m.p["layer.2.qkv.weight"], m.p["layer.3.qkv.weight"])
+    # the old prefix still computes the same thing
+    m2 = O.MsltOracle(w, cfg.heads)
+    h2, _ = m2.forward(tok, lens)
+    assert np.array_equal(h_before, h2)
+    with pytest.raises(ValueError):
+        m.add_layers(1)                      # arena full
+    m3 = O.MsltOracle(w, cfg.heads, max_layers=8)
+    with pytest.raises(ValueError):
+        m3.add_layers(3)                     # k > L
+    # staged training after stacking: new layers move, old ones do not
+    m.set_trainable(2)
+    before = {k: v.copy() for k, v in m.p.items()}
+    m.step(tok, lens, pos, lab)
+    for k in before:
+        frozen = k.startswith("emb.") or k.startswith("layer.0.") or k.startswith("layer.1.")
+        assert np.array_equal(before[k], m.p[k]) == frozen, k
+
+
+def test_forward_equals_forward_inside_step():
+    m = tiny_model(top_k=1)
+    tok, lens, pos, lab = tiny_batch()
+    h, logits = m.forward(tok, lens, pos)
+    x, _, _ = m.encode(tok, lens, keep_from=1)
+    assert np.array_equal(h, x)
+    l2, _ = m._head_forward(x, pos, lab)
+    ok = (pos >= 0).reshape(-1)
+    assert np.array_equal(logits[ok], l2[ok])
+
+
+# -- masking and batch structure ---------------------------------------------------------------------------------
+
+def test_padding_content_does_not_matter():
+    m = tiny_model(top_k=2)
+    tok, lens, pos, lab = tiny_batch()
+    l1, g1 = m.loss_and_grads(tok, lens, pos, lab)
+    tok2 = tok.copy()
+    for b in range(tok.shape[0]):
+        tok2[b, lens[b]:] = (tok2[b, lens[b]:] + 3) % TINY.vocab
+    assert not np.array_equal(tok, tok2)
+    l2, g2 = m.loss_and_grads(tok2, lens, pos, lab)
+    assert abs(l1 - l2) < 1e-15
+    for n in g1:
+        if n == "emb.word":
+            continue       # rows of the padded token ids receive (zero) scatter entries
+        np.testing.assert_allclose(g1[n], g2[n], atol=1e-15, rtol=0)
+    np.testing.assert_allclose(g1["emb.word"], g2["emb.word"], atol=1e-15, rtol=0)
+
+
+def test_batch_loss_and_gradients_are_slot_weighted_sums():
+    m = tiny_model(top_k=2)
+    tok, lens, pos, lab = tiny_batch()
+    L, G = m.loss_and_grads(tok, lens, pos, lab)
+    n_all = int((pos >= 0).sum())
+    acc_l, acc_g = 0.0, None
+    for b in range(tok.shape[0]):
+        sl = slice(b, b + 1)
+        nb = int((pos[sl] >= 0).sum())
+        lb, gb = m.loss_and_grads(tok[sl], lens[sl], pos[sl], lab[sl])
+        acc_l += lb * nb / n_all
+        gb = {k: v * nb / n_all for k, v in gb.items()}
+        acc_g = gb if acc_g is None else {k: acc_g[k] + gb[k] for k in gb}
+    assert abs(L - acc_l) < 1e-14
+    for n in G:
+        np.testing.assert_allclose(G[n], acc_g[n], atol=1e-14, rtol=0)
+
+
+def test_training_reduces_the_loss():
+    m = tiny_model(top_k=1)
+    m.set_optimizer(lr=1e-2)
+    tok, lens, pos, lab = tiny_batch()
+    losses = [m.step(tok, lens, pos, lab) for _ in range(20)]
+    assert losses[-1] < losses[0] - 0.1
+
+
+# -- the input generators ------------------------------------------------------------------------------------------
+
+def test_batches_follow_the_recipe():
+    cfg = I.scaled(I.CONFIGS["large_long"], batch=8)
+    tok, lens, pos, lab = I.make_batch(cfg)
+    assert tok.dtype == np.int32 and tok.shape == (8, 512)
+    assert lens.min() >= 256 and lens.max() <= 512
+    for b in range(8):
+        n = int((pos[b] >= 0).sum())
+        assert n == min(cfg.pred, max(1, round(0.15 * lens[b])))
+        assert np.all(pos[b, :n] < lens[b]) and len(set(pos[b, :n])) == n
+        assert np.all((lab[b, :n] >= 0) & (lab[b, :n] < cfg.vocab))
+        assert np.all(pos[b, n:] == -1) and np.all(lab[b, n:] == -1)
+        assert np.all(tok[b, lens[b]:] == 0)
+    t2, _, _, _ = I.make_batch(cfg)
+    assert np.array_equal(tok, t2)
+    big = I.zipf_tokens(I._rng(1, 1), 30522, (200000,))
+    assert 0.05 < (big == 0).mean() < 0.2 and big.max() > 10000   # Zipf head and tail
+    a = I.make_batch(I.scaled(I.CONFIGS["base_stage"], batch=2))
+    b = I.make_batch(I.scaled(I.CONFIGS["base_full"], batch=2))
+    assert all(np.array_equal(x, y) for x, y in zip(a, b))         # same seed, same data
