@@ -1,0 +1,207 @@
+/*
+ * mslt.h - C ABI of the per-stage training step of multi-stage layerwise
+ * training (MSLT) for BERT on one NVIDIA B200 (sm_100a).
+ *
+ * The procedure (paper, Section 3.1 last paragraph, Section 3.2 and Fig. 1):
+ * the encoder stack grows by a group of layers per stage; in each stage the
+ * bottom layers, trained earlier, only run forward to feed the top layers,
+ * while the newly added top layers and the output layer run forward and
+ * backward and are the only parameters updated.  The word-embedding matrix
+ * is shared by the input and the output layer and moves only while every
+ * layer is trainable (first stage, joint retraining).
+ *
+ * General rules
+ *  - Every function returns 0 on success or a negative mslt_status; nothing
+ *    throws or aborts across this boundary.  mslt_last_error() gives a
+ *    message for the last failure on the calling thread.
+ *  - The library allocates no device memory.  The caller owns the parameter
+ *    block and the workspace (sizes from mslt_query_bytes) and the CUDA
+ *    stream; they must outlive the context.  All work is enqueued on that
+ *    stream.  Pointers marked "device" must be device addresses on the
+ *    context's GPU; pointers marked "host" are ordinary host memory.
+ *  - Index tensors are int32, row-major.  Weight matrices are [out, in]
+ *    row-major, so the tied decoder is the [vocab, hidden] embedding table.
+ *  - There is no CPU fallback: without a CUDA device every compute call fails
+ *    with MSLT_ERR_CUDA.
+ */
+#ifndef MSLT_H_
+#define MSLT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct mslt_ctx mslt_ctx; /* opaque; host state owned by the library */
+
+typedef enum {
+  MSLT_OK = 0,
+  MSLT_ERR_ARG = -1,    /* invalid argument (null pointer, bad shape, unknown name)   */
+  MSLT_ERR_SIZE = -2,   /* shape exceeds what the context was created for             */
+  MSLT_ERR_STATE = -3,  /* call not valid in this state (k > L, arena full, ...)      */
+  MSLT_ERR_CUDA = -4,   /* a CUDA call failed, or no usable device                    */
+  MSLT_ERR_DEVICE = -5  /* a kernel reported an error: a bounded wait ran out, or an  */
+                        /* index (token id, MLM position or label) was out of range   */
+} mslt_status;
+
+/* Architecture and capacity.  BERT encoder: post-LayerNorm, erf GELU, head dim = hidden/heads. */
+typedef struct {
+  int32_t hidden;      /* H; multiple of 64, <= 1024                                  */
+  int32_t heads;       /* A; H % A == 0; dtype 1 needs H / A == 64                     */
+  int32_t ffn;         /* F; multiple of 64                                            */
+  int32_t vocab;       /* V                                                            */
+  int32_t max_pos;     /* rows of the position table, >= max_seq                       */
+  int32_t init_layers; /* encoder layers present after mslt_create (stage 1 depth)     */
+  int32_t max_layers;  /* capacity of the layer arena (final depth N)                  */
+  int32_t max_batch;   /* largest B of any later call                                  */
+  int32_t max_seq;     /* largest S; multiple of 8, <= 512                             */
+  int32_t max_pred;    /* largest P (MLM slots per sequence)                           */
+  int32_t dtype;       /* 0: fp32 everywhere; 1: bf16 weights/activations, fp32 master */
+                       /*    weights, gradients and Adam state                         */
+  float ln_eps;        /* LayerNorm epsilon (BERT: 1e-12)                              */
+} mslt_arch;
+
+/* Adam with decoupled weight decay (decay on matrices and tables only). */
+typedef struct {
+  float lr, beta1, beta2, eps, weight_decay;
+  int32_t bias_correction; /* 1: divide m, v by (1 - beta^t)                           */
+} mslt_opt;
+
+/* Bytes of device memory the caller must provide for this architecture. */
+int mslt_query_bytes(const mslt_arch* arch, size_t* param_bytes, size_t* workspace_bytes);
+
+/*
+ * Creates a context with init_layers encoder layers, all trainable (in the first
+ * stage every parameter is trained, Section 3.2).  dev_params / dev_workspace:
+ * device, at least the queried sizes, 256-byte aligned; the library zeroes
+ * both.  Parameters are left at zero: set them with mslt_set_param.
+ * cuda_stream: a cudaStream_t (NULL = the default stream).  *out: host.
+ */
+int mslt_create(const mslt_arch* arch, void* dev_params, size_t param_bytes, void* dev_workspace,
+                size_t workspace_bytes, void* cuda_stream, mslt_ctx** out);
+
+/* Frees host state only; device memory stays with the caller. */
+int mslt_destroy(mslt_ctx* ctx);
+
+/*
+ * Stacks k new layers on top (Section 3.2: new layers start as copies of the
+ * top k layers of the previous stage's model): layer L+i <- layer L-k+i, for
+ * master weights and compute copies alike.  Needs 1 <= k <= L and
+ * L + k <= max_layers (else MSLT_ERR_STATE).  The number of trainable top
+ * layers is kept; the optimizer state (m, v, step count) is zeroed.
+ */
+int mslt_add_layers(mslt_ctx* ctx, int32_t k);
+
+/*
+ * Moves the frozen/trainable boundary (Section 3.2): layers [L-top_k, L) and
+ * the output layer (MLM transform, its LayerNorm, decoder bias) are trained;
+ * top_k == L also trains the embeddings (word table shared with the decoder,
+ * position table, embedding LayerNorm).  0 <= top_k <= L.  Zeroes the
+ * optimizer state.
+ */
+int mslt_set_trainable(mslt_ctx* ctx, int32_t top_k);
+
+/* Hyper-parameters used from the next step on (learning-rate schedules are the caller's). */
+int mslt_set_optimizer(mslt_ctx* ctx, const mslt_opt* opt);
+
+/*
+ * One training step (Section 3.1/3.2, Fig. 1): forward-only pass through the
+ * frozen layers keeping nothing but the boundary activation; forward with
+ * saved activations and backward through the trainable layers and the MLM
+ * head; mean cross-entropy over the valid slots; Adam on the trainable
+ * parameters only.  Frozen parameters are never written.
+ *   d_tokens        device [B,S]   token ids in [0, vocab)
+ *   d_seq_lens      device [B] or NULL (= all S); key j of sequence b is valid iff j < len, len >= 1
+ *   d_mlm_positions device [B,P]   position in [0, len) or -1 for an empty slot
+ *   d_mlm_labels    device [B,P]   label in [0, vocab) or -1 to ignore the slot
+ *   loss_out        host float or NULL.  Non-NULL: the stream is synchronised and the loss
+ *                   and the device status word are read back (an out-of-range index or a
+ *                   kernel wait that ran out gives MSLT_ERR_DEVICE).  NULL: nothing is
+ *                   synchronised; use mslt_read_loss later.
+ */
+int mslt_step(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens,
+              const int32_t* d_mlm_positions, const int32_t* d_mlm_labels, int32_t B, int32_t S,
+              int32_t P, float* loss_out);
+
+/* Synchronises the stream and returns the loss of the last mslt_step (host pointer). */
+int mslt_read_loss(mslt_ctx* ctx, float* loss_out);
+
+/*
+ * Forward only, nothing saved at any layer, no update.
+ *   d_hidden_out  device [B,S,H] in the compute dtype (float or bf16), or NULL
+ *   d_mlm_positions device [B,P] or NULL; d_logits_out device [B*P, vocab] fp32 or NULL
+ *   (rows of empty slots are computed from a zero feature row).
+ * Synchronises the stream before returning.
+ */
+int mslt_forward(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens, int32_t B,
+                 int32_t S, void* d_hidden_out, const int32_t* d_mlm_positions, int32_t P,
+                 float* d_logits_out);
+
+/* Inspection.  Tensor names: "emb.word", "emb.pos", "emb.ln.gamma", "layer.3.ffn1.weight",
+ * "head.transform.bias", "head.decoder.bias", ...  All buffers below are host memory. */
+int mslt_num_layers(const mslt_ctx* ctx);
+int mslt_num_trainable(const mslt_ctx* ctx);
+int mslt_num_tensors(const mslt_ctx* ctx); /* tensors of the layers present now */
+int mslt_tensor_info(const mslt_ctx* ctx, int32_t index, const char** name, int32_t* rank,
+                     int64_t shape[2], int32_t* trainable);
+/* fp32 master values; n must equal the tensor's element count. */
+int mslt_get_param(mslt_ctx* ctx, const char* name, float* host_dst, size_t n);
+/* Writes the master value and, for dtype 1, its bf16 rounding (nearest even). */
+int mslt_set_param(mslt_ctx* ctx, const char* name, const float* host_src, size_t n);
+/* Raw bits of the copy the kernels read (bf16 for matrices at dtype 1, else fp32), for bit-exact checks. */
+int mslt_get_param_raw(mslt_ctx* ctx, const char* name, void* host_dst, size_t bytes);
+/* fp32 gradient of a trainable tensor as left by the last mslt_step. */
+int mslt_get_grad(mslt_ctx* ctx, const char* name, float* host_dst, size_t n);
+/* Adam moments of a trainable tensor (which = 0: m, 1: v). */
+int mslt_get_opt_state(mslt_ctx* ctx, const char* name, int32_t which, float* host_dst, size_t n);
+/* Number of kernels the library has launched on this context since creation. */
+int64_t mslt_launch_count(const mslt_ctx* ctx);
+/* Milliseconds of the phases of the last mslt_step when timing is on (mslt_set_timing(ctx,1)):
+ * [0] frozen forward, [1] trainable forward, [2] head forward+backward, [3] encoder backward,
+ * [4] Adam.  Turning timing on adds event records and one synchronisation per step. */
+int mslt_set_timing(mslt_ctx* ctx, int32_t on);
+int mslt_get_timings(mslt_ctx* ctx, float* host_ms, int32_t n);
+/* Message for the last error on this thread (ctx may be NULL). */
+const char* mslt_last_error(const mslt_ctx* ctx);
+
+/*
+ * One dense contraction with the step's fused epilogue, exposed for per-kernel tests and
+ * profiling:  D[z][m][n] = epilogue( alpha * sum_k A[z](m,k) * B[z](n,k) ).
+ * It is the kernel behind every linear layer and attention product of the step (forward:
+ * both operands k-contiguous; input-gradient and weight-gradient products: operands with
+ * the m / n index contiguous).  dtype 0 runs the fp32 CUDA-core kernel, dtype 1 the bf16
+ * tcgen05 tensor-core kernel with fp32 accumulation in tensor memory.
+ * All pointers are device pointers; strides are in elements.
+ */
+typedef struct {
+  int32_t dtype;            /* 0: A, B fp32; 1: A, B bf16                                   */
+  int32_t M, N, K, batch;   /* batch >= 1; z in [0, batch)                                  */
+  int32_t hdiv;             /* z splits as (z / hdiv, z % hdiv) for the two batch strides   */
+  const void* A;            /* element (z,m,k) at A + (z/hdiv)*a_bo + (z%hdiv)*a_bi + m*a_rs + k*a_ks */
+  int64_t a_rs, a_ks, a_bo, a_bi; /* one of a_rs, a_ks must be 1                            */
+  const void* B;            /* element (z,n,k) likewise                                     */
+  int64_t b_rs, b_ks, b_bo, b_bi;
+  void* D;                  /* element (z,m,n) at D + (z/hdiv)*d_bo + (z%hdiv)*d_bi + m*ldd + n */
+  int64_t ldd, d_bo, d_bi;
+  int32_t d_fp32;           /* 1: D is fp32 (else the A/B dtype)                            */
+  int32_t accumulate;       /* 1 (needs d_fp32): D += result (atomic adds; order not fixed) */
+  float alpha;
+  const float* bias;        /* [N] fp32 added after alpha, or NULL                          */
+  int32_t act;              /* 0 none; 1 GELU(erf); 2 multiply by GELU'(aux)                */
+  void* aux;                /* D's layout and A/B dtype. act 1: receives the pre-activation */
+                            /* (may be NULL); act 2: holds the pre-activation               */
+  const void* residual;     /* D's layout, A/B dtype, added last; or NULL                   */
+  int32_t split_k;          /* 0 = automatic; > 1 needs d_fp32 and accumulate               */
+} mslt_gemm_desc;
+
+/* Runs one contraction on `cuda_stream` and synchronises it.  d_status: device int32 word,
+ * zeroed by the caller, that receives a non-zero code if a kernel wait ran out (then the
+ * call returns MSLT_ERR_DEVICE). */
+int mslt_op_gemm(const mslt_gemm_desc* desc, void* cuda_stream, int32_t* d_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MSLT_H_ */

@@ -1,0 +1,262 @@
+"""ctypes binding of libmslt.so: argument marshalling only.
+
+Every step of the training path runs in the library's CUDA kernels; torch is
+used here for device memory, streams and nothing else.  Importing this module
+loads the shared library and fails loudly if it has not been built
+(`python -m paper_2011_13635_b200.build`).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmslt.so")
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2011_13635_b200.build`; "
+                      "there is no fallback path")
+lib = C.CDLL(LIB_PATH)
+
+
+class Arch(C.Structure):
+    _fields_ = [("hidden", C.c_int32), ("heads", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32),
+                ("max_pos", C.c_int32), ("init_layers", C.c_int32), ("max_layers", C.c_int32),
+                ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("max_pred", C.c_int32),
+                ("dtype", C.c_int32), ("ln_eps", C.c_float)]
+
+
+class Opt(C.Structure):
+    _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
+                ("weight_decay", C.c_float), ("bias_correction", C.c_int32)]
+
+
+class GemmDesc(C.Structure):
+    _fields_ = [("dtype", C.c_int32), ("M", C.c_int32), ("N", C.c_int32), ("K", C.c_int32),
+                ("batch", C.c_int32), ("hdiv", C.c_int32),
+                ("A", C.c_void_p), ("a_rs", C.c_int64), ("a_ks", C.c_int64), ("a_bo", C.c_int64),
+                ("a_bi", C.c_int64),
+                ("B", C.c_void_p), ("b_rs", C.c_int64), ("b_ks", C.c_int64), ("b_bo", C.c_int64),
+                ("b_bi", C.c_int64),
+                ("D", C.c_void_p), ("ldd", C.c_int64), ("d_bo", C.c_int64), ("d_bi", C.c_int64),
+                ("d_fp32", C.c_int32), ("accumulate", C.c_int32), ("alpha", C.c_float),
+                ("bias", C.c_void_p), ("act", C.c_int32), ("aux", C.c_void_p),
+                ("residual", C.c_void_p), ("split_k", C.c_int32)]
+
+
+EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers", "mslt_set_trainable",
+           "mslt_set_optimizer", "mslt_step", "mslt_read_loss", "mslt_forward", "mslt_num_layers",
+           "mslt_num_trainable", "mslt_num_tensors", "mslt_tensor_info", "mslt_get_param",
+           "mslt_set_param", "mslt_get_param_raw", "mslt_get_grad", "mslt_get_opt_state",
+           "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_last_error",
+           "mslt_op_gemm"]
+
+lib.mslt_last_error.restype = C.c_char_p
+lib.mslt_last_error.argtypes = [C.c_void_p]
+lib.mslt_launch_count.restype = C.c_int64
+lib.mslt_launch_count.argtypes = [C.c_void_p]
+lib.mslt_query_bytes.argtypes = [C.POINTER(Arch), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+lib.mslt_create.argtypes = [C.POINTER(Arch), C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t,
+                            C.c_void_p, C.POINTER(C.c_void_p)]
+lib.mslt_destroy.argtypes = [C.c_void_p]
+lib.mslt_add_layers.argtypes = [C.c_void_p, C.c_int32]
+lib.mslt_set_trainable.argtypes = [C.c_void_p, C.c_int32]
+lib.mslt_set_optimizer.argtypes = [C.c_void_p, C.POINTER(Opt)]
+lib.mslt_step.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                          C.c_int32, C.c_int32, C.POINTER(C.c_float)]
+lib.mslt_read_loss.argtypes = [C.c_void_p, C.POINTER(C.c_float)]
+lib.mslt_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
+                             C.c_void_p, C.c_int32, C.c_void_p]
+lib.mslt_num_layers.argtypes = [C.c_void_p]
+lib.mslt_num_trainable.argtypes = [C.c_void_p]
+lib.mslt_num_tensors.argtypes = [C.c_void_p]
+lib.mslt_tensor_info.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_char_p), C.POINTER(C.c_int32),
+                                 C.POINTER(C.c_int64), C.POINTER(C.c_int32)]
+lib.mslt_get_param.argtypes = [C.c_void_p, C.c_char_p, C.c_void_p, C.c_size_t]
+lib.mslt_set_param.argtypes = [C.c_void_p, C.c_char_p, C.c_void_p, C.c_size_t]
+lib.mslt_get_param_raw.argtypes = [C.c_void_p, C.c_char_p, C.c_void_p, C.c_size_t]
+lib.mslt_get_grad.argtypes = [C.c_void_p, C.c_char_p, C.c_void_p, C.c_size_t]
+lib.mslt_get_opt_state.argtypes = [C.c_void_p, C.c_char_p, C.c_int32, C.c_void_p, C.c_size_t]
+lib.mslt_set_timing.argtypes = [C.c_void_p, C.c_int32]
+lib.mslt_get_timings.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+lib.mslt_op_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
+
+
+class MsltError(RuntimeError):
+    def __init__(self, code: int, msg: str):
+        super().__init__(f"mslt error {code}: {msg}")
+        self.code = code
+
+
+def _check(rc: int):
+    if rc != 0:
+        raise MsltError(rc, (lib.mslt_last_error(None) or b"").decode())
+
+
+def _ptr(t) -> Optional[int]:
+    return None if t is None else t.data_ptr()
+
+
+def mslt_query_bytes(arch: Arch):
+    pb, wb = C.c_size_t(), C.c_size_t()
+    _check(lib.mslt_query_bytes(C.byref(arch), C.byref(pb), C.byref(wb)))
+    return pb.value, wb.value
+
+
+def mslt_op_gemm(desc: GemmDesc, stream: int, status) -> None:
+    _check(lib.mslt_op_gemm(C.byref(desc), C.c_void_p(stream), C.c_void_p(_ptr(status))))
+
+
+class Mslt:
+    """A stage-training context.  Device buffers are torch tensors owned by this object."""
+
+    def __init__(self, *, hidden, heads, ffn, vocab, max_pos, init_layers, max_layers, max_batch,
+                 max_seq, max_pred, dtype: str, ln_eps: float = 1e-12, device="cuda:0", stream=None):
+        import torch
+        self.torch = torch
+        if not torch.cuda.is_available():
+            raise MsltError(-4, "no CUDA device: this library has no CPU path")
+        self.device = torch.device(device)
+        self.arch = Arch(hidden, heads, ffn, vocab, max_pos, init_layers, max_layers, max_batch,
+                         max_seq, max_pred, {"fp32": 0, "bf16": 1}[dtype], ln_eps)
+        self.dtype = dtype
+        pb, wb = mslt_query_bytes(self.arch)
+        with torch.cuda.device(self.device):
+            self._params = torch.empty(pb, dtype=torch.uint8, device=self.device)
+            self._ws = torch.empty(wb, dtype=torch.uint8, device=self.device)
+            self.stream = stream if stream is not None else torch.cuda.current_stream(self.device)
+            h = C.c_void_p()
+            _check(lib.mslt_create(C.byref(self.arch), self._params.data_ptr(), pb, self._ws.data_ptr(),
+                                   wb, C.c_void_p(self.stream.cuda_stream), C.byref(h)))
+        self.h = h
+        self.param_bytes, self.workspace_bytes = pb, wb
+
+    @classmethod
+    def from_config(cls, cfg, *, init_layers=None, max_layers=None, **kw):
+        return cls(hidden=cfg.hidden, heads=cfg.heads, ffn=cfg.ffn, vocab=cfg.vocab,
+                   max_pos=cfg.max_pos, init_layers=cfg.layers if init_layers is None else init_layers,
+                   max_layers=cfg.layers if max_layers is None else max_layers,
+                   max_batch=cfg.batch, max_seq=cfg.seq, max_pred=cfg.pred, dtype=cfg.dtype, **kw)
+
+    def close(self):
+        if getattr(self, "h", None):
+            lib.mslt_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
+
+    # -- staging ------------------------------------------------------------------------------
+    def mslt_add_layers(self, k: int):
+        _check(lib.mslt_add_layers(self.h, k))
+
+    def mslt_set_trainable(self, top_k: int):
+        _check(lib.mslt_set_trainable(self.h, top_k))
+
+    def mslt_set_optimizer(self, lr, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01,
+                           bias_correction=1):
+        o = Opt(lr, beta1, beta2, eps, weight_decay, int(bias_correction))
+        _check(lib.mslt_set_optimizer(self.h, C.byref(o)))
+
+    # -- the hot path -------------------------------------------------------------------------
+    def mslt_step(self, tokens, seq_lens, mlm_positions, mlm_labels, sync: bool = True):
+        """tokens [B,S], seq_lens [B] or None, positions/labels [B,P]: int32 CUDA tensors.
+        Returns the loss (float) when sync, else None."""
+        B, S = tokens.shape
+        P = mlm_positions.shape[1]
+        loss = C.c_float()
+        _check(lib.mslt_step(self.h, tokens.data_ptr(), _ptr(seq_lens), mlm_positions.data_ptr(),
+                             mlm_labels.data_ptr(), B, S, P, C.byref(loss) if sync else None))
+        return loss.value if sync else None
+
+    def mslt_read_loss(self) -> float:
+        loss = C.c_float()
+        _check(lib.mslt_read_loss(self.h, C.byref(loss)))
+        return loss.value
+
+    def mslt_forward(self, tokens, seq_lens=None, mlm_positions=None, want_hidden=True):
+        """Returns (hidden [B,S,H] in the compute dtype or None, logits [B*P,V] fp32 or None)."""
+        torch = self.torch
+        B, S = tokens.shape
+        hidden = logits = None
+        if want_hidden:
+            hidden = torch.empty((B, S, self.arch.hidden), device=self.device,
+                                 dtype=torch.bfloat16 if self.dtype == "bf16" else torch.float32)
+        P = 0
+        if mlm_positions is not None:
+            P = mlm_positions.shape[1]
+            logits = torch.empty((B * P, self.arch.vocab), device=self.device, dtype=torch.float32)
+        _check(lib.mslt_forward(self.h, tokens.data_ptr(), _ptr(seq_lens), B, S, _ptr(hidden),
+                                _ptr(mlm_positions), P, _ptr(logits)))
+        return hidden, logits
+
+    # -- inspection -----------------------------------------------------------------------------
+    @property
+    def num_layers(self) -> int:
+        return lib.mslt_num_layers(self.h)
+
+    @property
+    def num_trainable(self) -> int:
+        return lib.mslt_num_trainable(self.h)
+
+    @property
+    def launch_count(self) -> int:
+        return lib.mslt_launch_count(self.h)
+
+    def tensors(self) -> Dict[str, dict]:
+        out = {}
+        for i in range(lib.mslt_num_tensors(self.h)):
+            name, rank, tr = C.c_char_p(), C.c_int32(), C.c_int32()
+            shape = (C.c_int64 * 2)()
+            _check(lib.mslt_tensor_info(self.h, i, C.byref(name), C.byref(rank), shape, C.byref(tr)))
+            shp = (shape[0], shape[1]) if rank.value == 2 else (shape[0],)
+            out[name.value.decode()] = dict(shape=shp, trainable=bool(tr.value))
+        return out
+
+    def _shape(self, name):
+        info = self.tensors().get(name)
+        return info["shape"] if info else (0,)   # unknown names are reported by the library
+
+    def mslt_set_param(self, name: str, value: np.ndarray):
+        v = np.ascontiguousarray(value, dtype=np.float32)
+        _check(lib.mslt_set_param(self.h, name.encode(), v.ctypes.data, v.size))
+
+    def set_params(self, weights: Dict[str, np.ndarray]):
+        for k, v in weights.items():
+            self.mslt_set_param(k, v)
+
+    def mslt_get_param(self, name: str, shape=None) -> np.ndarray:
+        shape = self._shape(name) if shape is None else shape
+        out = np.empty(shape, dtype=np.float32)
+        _check(lib.mslt_get_param(self.h, name.encode(), out.ctypes.data, out.size))
+        return out
+
+    def mslt_get_param_raw(self, name: str, shape=None) -> np.ndarray:
+        shape = self._shape(name) if shape is None else shape
+        two_byte = self.dtype == "bf16" and len(shape) == 2
+        out = np.empty(shape, dtype=np.uint16 if two_byte else np.uint32)
+        _check(lib.mslt_get_param_raw(self.h, name.encode(), out.ctypes.data, out.nbytes))
+        return out
+
+    def mslt_get_grad(self, name: str, shape=None) -> np.ndarray:
+        shape = self._shape(name) if shape is None else shape
+        out = np.empty(shape, dtype=np.float32)
+        _check(lib.mslt_get_grad(self.h, name.encode(), out.ctypes.data, out.size))
+        return out
+
+    def mslt_get_opt_state(self, name: str, which: int, shape=None) -> np.ndarray:
+        shape = self._shape(name) if shape is None else shape
+        out = np.empty(shape, dtype=np.float32)
+        _check(lib.mslt_get_opt_state(self.h, name.encode(), which, out.ctypes.data, out.size))
+        return out
+
+    def mslt_set_timing(self, on: bool):
+        _check(lib.mslt_set_timing(self.h, int(on)))
+
+    def mslt_get_timings(self) -> Dict[str, float]:
+        buf = (C.c_float * 5)()
+        _check(lib.mslt_get_timings(self.h, buf, 5))
+        return dict(zip(["frozen_fwd", "train_fwd", "head", "encoder_bwd", "adam"], list(buf)))

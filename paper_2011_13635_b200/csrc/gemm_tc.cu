@@ -1,0 +1,633 @@
+// bf16 dense contraction on the 5th-generation tensor cores (sm_100a):
+//   D[z][m][n] = epilogue(alpha * sum_k A[z](m,k) * B[z](n,k)),  fp32 accumulation in TMEM.
+//
+// One persistent CTA per SM walks a list of (split, batch, m-tile, n-tile) work items.
+//   warp 0   : TMA producer.  128-byte-swizzled operand tiles go global -> shared through a ring
+//              of stages, each guarded by a full/empty mbarrier pair.
+//   warp 1   : allocates tensor memory and issues tcgen05.mma (one thread) for 128 x BN x 16
+//              steps; tcgen05.commit hands shared-memory stages back to the producer and
+//              accumulators over to the epilogue.
+//   warps 2-5: epilogue.  Each warp owns one 32-lane quarter of TMEM, reads the accumulator
+//              with tcgen05.ld and applies scale, bias, GELU / GELU', residual, then stores bf16
+//              or fp32 (plain or as vector reductions for split-k).  Two accumulators of up to 256
+//              columns let the epilogue of one tile overlap the main loop of the next.
+// Operands may be k-contiguous ("K-major") or row-contiguous ("MN-major"); the second form is
+// what input-gradient and weight-gradient products need, and is fed to the tensor cores through
+// the MN-major shared-memory descriptor, so no transposed copies exist anywhere.
+// Every wait is bounded: when one runs out the CTA raises a status bit, drains and returns.
+#include <cuda.h>
+#include <stdio.h>
+#include <string.h>
+
+#include <mutex>
+#include <string>
+#include <unordered_map>
+
+#include "common.cuh"
+#include "gemm.h"
+
+namespace mslt {
+
+namespace {
+
+constexpr int BM = 128;           // rows of an output tile = TMEM lanes
+constexpr int BK = 64;            // k extent of a stage: 64 bf16 = one 128-byte swizzle row
+constexpr int UMMA_K = 16;        // k extent of one tcgen05.mma for 16-bit operands
+constexpr int MAX_STAGES = 8;
+constexpr int A_STAGE_BYTES = BM * BK * 2;
+constexpr int NUM_THREADS = 192;
+constexpr uint32_t TMEM_COLS = 512;
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+
+struct TcParams {
+  int M, N, K, batch, hdiv;
+  int bn, stages, a_mn, b_mn;
+  int m_tiles, n_tiles, splits, kb_total, kb_per_split, total_work;
+  int a_perm[3], b_perm[3];  // slot (1..3) of the (outer, inner-batch, outer-batch) coordinates
+  char* D;
+  long long ldd, d_bo, d_bi;
+  int d_fp32, accumulate, vec_ok;
+  float alpha;
+  const float* bias;
+  int act;
+  bf16* aux;
+  const bf16* residual;
+  int* status;
+  uint32_t idesc;
+};
+
+// ---- PTX wrappers -----------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) {
+  return (uint32_t)__cvta_generic_to_shared(p);
+}
+__device__ __forceinline__ unsigned long long globaltimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait.  Returns false when the limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
+                                          int* status) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const unsigned long long t0 = globaltimer();
+  uint32_t spins = 0;
+  while (true) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((++spins & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if (globaltimer() - t0 > WAIT_LIMIT_NS) {
+        *abort_flag = 1;
+        atomicOr(status, ST_WAIT_TIMEOUT);
+        return false;
+      }
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0,
+                                            int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() {
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_fence_after() {
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar)
+               : "memory");
+}
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                       uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+  uint32_t r[32];
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+  for (int i = 0; i < 32; i++) v[i] = __uint_as_float(r[i]);
+}
+
+// Shared-memory matrix descriptor for a 128-byte-swizzled tile whose rows are 128 bytes apart and
+// whose 8-row groups are 1024 bytes apart.  lbo_bytes: distance between 64-element column blocks
+// of an MN-major operand (ignored by the hardware for K-major swizzled tiles).
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+  d |= (uint64_t)((1024u >> 4) & 0x3FFFu) << 32;  // stride between 8-row groups
+  d |= (uint64_t)1 << 46;                         // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                         // 128-byte swizzle
+  return d;
+}
+
+// ---- the kernel ---------------------------------------------------------------------------------
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // tiles need 1024-byte alignment for the 128-byte swizzle pattern
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  const int b_stage_bytes = p.bn * BK * 2;
+  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+  uint64_t* bars = (uint64_t*)(smem + (size_t)p.stages * stage_bytes);
+  uint64_t* full_bar = bars;
+  uint64_t* empty_bar = bars + MAX_STAGES;
+  uint64_t* tfull_bar = bars + 2 * MAX_STAGES;
+  uint64_t* tempty_bar = bars + 2 * MAX_STAGES + 2;
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * MAX_STAGES + 4);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; s++) {
+      mbar_init(smem_u32(&full_bar[s]), 1);
+      mbar_init(smem_u32(&empty_bar[s]), 1);
+    }
+    for (int a = 0; a < 2; a++) {
+      mbar_init(smem_u32(&tfull_bar[a]), 1);
+      mbar_init(smem_u32(&tempty_bar[a]), 4);
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  const int tiles_per_z = p.m_tiles * p.n_tiles;
+  const int per_split = tiles_per_z * p.batch;
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    uint32_t it = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < p.total_work && ok; w += gridDim.x) {
+      const int split = w / per_split;
+      int r = w - split * per_split;
+      const int z = r / tiles_per_z;
+      r -= z * tiles_per_z;
+      const int mt = r / p.n_tiles, nt = r - mt * p.n_tiles;
+      const int zo = z / p.hdiv, zi = z - zo * p.hdiv;
+      const int kb0 = split * p.kb_per_split;
+      const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+      for (int kb = kb0; kb < kb1; kb++, it++) {
+        const uint32_t s = it % p.stages, round = it / p.stages;
+        if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+        const uint32_t fb = smem_u32(&full_bar[s]);
+        mbar_expect_tx(fb, stage_bytes);
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t sb = sa + A_STAGE_BYTES;
+        int c[4];
+        if (!p.a_mn) {  // box {64 k, 128 rows}
+          c[0] = kb * BK; c[p.a_perm[0]] = mt * BM; c[p.a_perm[1]] = zi; c[p.a_perm[2]] = zo;
+          tma_load_4d(sa, &tmA, fb, c[0], c[1], c[2], c[3]);
+        } else {        // two boxes {64 rows, 64 k}
+          c[p.a_perm[0]] = kb * BK; c[p.a_perm[1]] = zi; c[p.a_perm[2]] = zo;
+#pragma unroll
+          for (int h = 0; h < BM / 64; h++) {
+            c[0] = mt * BM + h * 64;
+            tma_load_4d(sa + h * (64 * BK * 2), &tmA, fb, c[0], c[1], c[2], c[3]);
+          }
+        }
+        if (!p.b_mn) {  // box {64 k, bn rows}
+          c[0] = kb * BK; c[p.b_perm[0]] = nt * p.bn; c[p.b_perm[1]] = zi; c[p.b_perm[2]] = zo;
+          tma_load_4d(sb, &tmB, fb, c[0], c[1], c[2], c[3]);
+        } else {
+          c[p.b_perm[0]] = kb * BK; c[p.b_perm[1]] = zi; c[p.b_perm[2]] = zo;
+          for (int h = 0; h < p.bn / 64; h++) {
+            c[0] = nt * p.bn + h * 64;
+            tma_load_4d(sb + h * (64 * BK * 2), &tmB, fb, c[0], c[1], c[2], c[3]);
+          }
+        }
+      }
+    }
+    if (!ok || *abort_flag) {
+      // give up: let the copies already in flight land before the CTA leaves
+      const uint32_t n = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
+      for (uint32_t i = 0; i < n; i++) {
+        const uint32_t j = it - 1 - i;
+        const uint32_t fb = smem_u32(&full_bar[j % p.stages]);
+        const unsigned long long t0 = globaltimer();
+        while (!mbar_try_wait(fb, (j / p.stages) & 1) && globaltimer() - t0 < 100000000ull) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------- MMA issuer -------------------------------
+    uint32_t it = 0, tile = 0;
+    bool ok = true;
+    const uint32_t a_lbo = p.a_mn ? 64 * BK * 2 : 16;
+    const uint32_t b_lbo = p.b_mn ? 64 * BK * 2 : 16;
+    const uint32_t a_kstep = p.a_mn ? UMMA_K * 128 : UMMA_K * 2;  // bytes per 16-wide k step
+    const uint32_t b_kstep = p.b_mn ? UMMA_K * 128 : UMMA_K * 2;
+    for (int w = blockIdx.x; w < p.total_work && ok; w += gridDim.x, tile++) {
+      const int split = w / per_split;
+      const int kb0 = split * p.kb_per_split;
+      const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+      const uint32_t acc = tile & 1, use = tile >> 1;
+      if (!mbar_wait(smem_u32(&tempty_bar[acc]), (use & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + acc * 256;
+      for (int kb = kb0; kb < kb1; kb++, it++) {
+        const uint32_t s = it % p.stages, round = it / p.stages;
+        if (!mbar_wait(smem_u32(&full_bar[s]), round & 1, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t sb = sa + A_STAGE_BYTES;
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; k++) {
+          const uint64_t ad = make_smem_desc(sa + k * a_kstep, a_lbo);
+          const uint64_t bd = make_smem_desc(sb + k * b_kstep, b_lbo);
+          tc_mma(d_tmem, ad, bd, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+        }
+        tc_commit(smem_u32(&empty_bar[s]));  // stage is free once these MMAs have read it
+      }
+      if (ok) tc_commit(smem_u32(&tfull_bar[acc]));  // accumulator complete
+    }
+    if (!ok || *abort_flag) {
+      // make sure no MMA is still writing tensor memory before it is freed
+      tc_commit(smem_u32(&tfull_bar[0]));
+      const unsigned long long t0 = globaltimer();
+      while (globaltimer() - t0 < 1000000ull) {}
+    }
+  } else if (warp >= 2) {
+    // ------------------------------- epilogue -------------------------------
+    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    uint32_t tile = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < p.total_work && ok; w += gridDim.x, tile++) {
+      const int split = w / per_split;
+      int r = w - split * per_split;
+      const int z = r / tiles_per_z;
+      r -= z * tiles_per_z;
+      const int mt = r / p.n_tiles, nt = r - mt * p.n_tiles;
+      const int zo = z / p.hdiv, zi = z - zo * p.hdiv;
+      const uint32_t acc = tile & 1, use = tile >> 1;
+      if (!mbar_wait(smem_u32(&tfull_bar[acc]), use & 1, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const int m = mt * BM + q * 32 + lane;
+      const long long off0 = zo * p.d_bo + zi * p.d_bi + (long long)m * p.ldd;
+      const int n_base = nt * p.bn;
+      for (int cidx = 0; cidx < p.bn / 32; cidx++) {
+        const int n0 = n_base + cidx * 32;
+        if (n0 >= p.N) break;  // uniform over the warp
+        float v[32];
+        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256 + cidx * 32, v);
+        if (m < p.M) {
+          const long long off = off0 + n0;
+          const bool fullv = p.vec_ok && (n0 + 32 <= p.N);
+#pragma unroll
+          for (int j = 0; j < 32; j++) v[j] *= p.alpha;
+          if (p.bias) {
+            if (n0 + 32 <= p.N) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                const float4 b4 = *reinterpret_cast<const float4*>(p.bias + n0 + j);
+                v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j++)
+                if (n0 + j < p.N) v[j] += p.bias[n0 + j];
+            }
+          }
+          if (p.act == 1) {
+            if (p.aux) {
+              if (fullv) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 8) {
+                  float t[8];
+#pragma unroll
+                  for (int e = 0; e < 8; e++) t[e] = v[j + e];
+                  VecT<bf16>::store(p.aux + off + j, t);
+                }
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; j++)
+                  if (n0 + j < p.N) p.aux[off + j] = __float2bfloat16_rn(v[j]);
+              }
+            }
+#pragma unroll
+            for (int j = 0; j < 32; j++) v[j] = gelu_f(v[j]);
+          } else if (p.act == 2) {
+            if (fullv) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                float t[8];
+                VecT<bf16>::load(p.aux + off + j, t);
+#pragma unroll
+                for (int e = 0; e < 8; e++) v[j + e] *= gelu_grad_f(t[e]);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j++)
+                if (n0 + j < p.N) v[j] *= gelu_grad_f(__bfloat162float(p.aux[off + j]));
+            }
+          }
+          if (p.residual) {
+            if (fullv) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                float t[8];
+                VecT<bf16>::load(p.residual + off + j, t);
+#pragma unroll
+                for (int e = 0; e < 8; e++) v[j + e] += t[e];
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j++)
+                if (n0 + j < p.N) v[j] += __bfloat162float(p.residual[off + j]);
+            }
+          }
+          if (p.d_fp32) {
+            float* dp = reinterpret_cast<float*>(p.D) + off;
+            if (p.accumulate) {
+              if (fullv) {
+#pragma unroll
+                for (int j = 0; j < 32; j += 4)
+                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dp + j), "f"(v[j]),
+                               "f"(v[j + 1]), "f"(v[j + 2]), "f"(v[j + 3])
+                               : "memory");
+              } else {
+#pragma unroll
+                for (int j = 0; j < 32; j++)
+                  if (n0 + j < p.N) atomicAdd(dp + j, v[j]);
+              }
+            } else if (fullv) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(dp + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j++)
+                if (n0 + j < p.N) dp[j] = v[j];
+            }
+          } else {
+            bf16* dp = reinterpret_cast<bf16*>(p.D) + off;
+            if (fullv) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                float t[8];
+#pragma unroll
+                for (int e = 0; e < 8; e++) t[e] = v[j + e];
+                VecT<bf16>::store(dp + j, t);
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; j++)
+                if (n0 + j < p.N) dp[j] = __float2bfloat16_rn(v[j]);
+            }
+          }
+        }
+      }
+      // hand the accumulator back to the MMA warp
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
+                 : "memory");
+  }
+}
+
+// ---- host side: tensor maps and launch ------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = (EncodeTiledFn)p;
+  });
+  return fn;
+}
+
+struct MapKey {
+  const void* ptr;
+  long long rows, K, rs, ks, bo, bi;
+  int hdiv, nb, box_rows;
+  bool operator==(const MapKey& o) const { return memcmp(this, &o, sizeof(MapKey)) == 0; }
+};
+struct MapKeyHash {
+  size_t operator()(const MapKey& k) const {
+    const uint64_t* w = reinterpret_cast<const uint64_t*>(&k);
+    uint64_t h = 1469598103934665603ull;
+    for (size_t i = 0; i < sizeof(MapKey) / 8; i++) h = (h ^ w[i]) * 1099511628211ull;
+    return (size_t)h;
+  }
+};
+struct MapVal {
+  CUtensorMap map;
+  int perm[3];
+};
+
+// Builds (or fetches) the rank-4 tensor map of one operand: dim 0 is the contiguous index (k for a
+// K-major operand, the row index otherwise); the other matrix index and the two batch indices
+// follow in order of increasing stride.
+int get_map(const void* ptr, long long rows, long long K, long long rs, long long ks, long long bo,
+            long long bi, int hdiv, int nb, int box_rows, MapVal* out, char* err) {
+  static std::unordered_map<MapKey, MapVal, MapKeyHash> cache;
+  static std::mutex mu;
+  MapKey key;
+  memset(&key, 0, sizeof(key));
+  key.ptr = ptr; key.rows = rows; key.K = K; key.rs = rs; key.ks = ks; key.bo = bo; key.bi = bi;
+  key.hdiv = hdiv; key.nb = nb; key.box_rows = box_rows;
+  std::lock_guard<std::mutex> lock(mu);
+  auto itf = cache.find(key);
+  if (itf != cache.end()) { *out = itf->second; return 0; }
+  EncodeTiledFn enc = get_encode();
+  if (!enc) { snprintf(err, 256, "gemm: cuTensorMapEncodeTiled is not available"); return MSLT_ERR_CUDA; }
+  const bool mn = rs == 1 && ks != 1;
+  // logical dims after dim 0: 0 = the other matrix index, 1 = inner batch, 2 = outer batch
+  long long ext[3] = {mn ? K : rows, hdiv, nb};
+  long long str[3] = {mn ? ks : rs, bi, bo};
+  unsigned box[3] = {(unsigned)(mn ? 64 : box_rows), 1, 1};
+  const long long ext0 = mn ? rows : K;
+  const long long big = (long long)1 << 38;
+  for (int i = 0; i < 3; i++)
+    if (ext[i] == 1 && (i > 0)) str[i] = 0;
+  // dims of extent 1 get a harmless stride at the end of the order
+  int order[3] = {0, 1, 2};
+  auto eff = [&](int i) { return (ext[i] == 1 && i > 0) ? big : str[i]; };
+  for (int i = 0; i < 3; i++)
+    for (int j = i + 1; j < 3; j++)
+      if (eff(order[j]) < eff(order[i])) { int t = order[i]; order[i] = order[j]; order[j] = t; }
+  cuuint64_t gdim[4], gstr[3];
+  cuuint32_t bdim[4], estr[4] = {1, 1, 1, 1};
+  gdim[0] = (cuuint64_t)ext0;
+  bdim[0] = 64;
+  long long last = 16;
+  for (int sl = 0; sl < 3; sl++) {
+    const int li = order[sl];
+    gdim[sl + 1] = (cuuint64_t)ext[li];
+    bdim[sl + 1] = box[li];
+    long long sb = eff(li) == big ? last : str[li] * 2;
+    if (sb <= 0 || sb % 16) {
+      snprintf(err, 256, "gemm: operand stride %lld bytes is not a positive multiple of 16", sb);
+      return MSLT_ERR_ARG;
+    }
+    gstr[sl] = (cuuint64_t)sb;
+    last = sb * (long long)ext[li];
+    out->perm[li] = sl + 1;
+  }
+  if ((uintptr_t)ptr & 15) { snprintf(err, 256, "gemm: operand base is not 16-byte aligned"); return MSLT_ERR_ARG; }
+  CUresult r = enc(&out->map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(ptr), gdim, gstr, bdim,
+                   estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  if (r != CUDA_SUCCESS) {
+    snprintf(err, 256, "gemm: cuTensorMapEncodeTiled failed with code %d (dims %llu,%llu,%llu,%llu)", (int)r,
+             (unsigned long long)gdim[0], (unsigned long long)gdim[1], (unsigned long long)gdim[2],
+             (unsigned long long)gdim[3]);
+    return MSLT_ERR_CUDA;
+  }
+  if (cache.size() > 4096) cache.clear();
+  cache[key] = *out;
+  return 0;
+}
+
+}  // namespace
+
+int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* err) {
+  static int num_sms = 0;
+  static int smem_optin = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (num_sms <= 0) { snprintf(err, 256, "gemm: no CUDA device"); return MSLT_ERR_CUDA; }
+  }
+  if (!status) { snprintf(err, 256, "gemm: the tensor-core kernel needs a device status word"); return MSLT_ERR_ARG; }
+  TcParams p;
+  memset(&p, 0, sizeof(p));
+  p.M = d.M; p.N = d.N; p.K = d.K; p.batch = d.batch; p.hdiv = d.hdiv;
+  p.a_mn = (d.a_rs == 1 && d.a_ks != 1) ? 1 : 0;
+  p.b_mn = (d.b_rs == 1 && d.b_ks != 1) ? 1 : 0;
+  p.bn = d.N <= 64 ? 64 : (d.N <= 128 ? 128 : 256);
+  p.m_tiles = (d.M + BM - 1) / BM;
+  p.n_tiles = (d.N + p.bn - 1) / p.bn;
+  p.kb_total = (d.K + BK - 1) / BK;
+  const long long tiles = (long long)p.m_tiles * p.n_tiles * d.batch;
+  int splits = 1;
+  if (d.split_k > 1) {
+    splits = d.split_k;
+  } else if (d.split_k == 0 && d.d_fp32 && d.accumulate && tiles < num_sms && p.kb_total >= 8) {
+    splits = (int)(num_sms / tiles);
+    const int max_by_k = p.kb_total / 4;  // keep at least four k blocks per split
+    if (splits > max_by_k) splits = max_by_k;
+    if (splits < 1) splits = 1;
+  }
+  if (splits > 1 && !(d.d_fp32 && d.accumulate)) {
+    snprintf(err, 256, "gemm: split_k needs an fp32 accumulating output");
+    return MSLT_ERR_ARG;
+  }
+  if (splits > p.kb_total) splits = p.kb_total;
+  p.kb_per_split = (p.kb_total + splits - 1) / splits;
+  p.splits = (p.kb_total + p.kb_per_split - 1) / p.kb_per_split;
+  const long long total = tiles * p.splits;
+  if (total > 0x7fffffffll) { snprintf(err, 256, "gemm: too many tiles"); return MSLT_ERR_SIZE; }
+  p.total_work = (int)total;
+  const int stage_bytes = A_STAGE_BYTES + p.bn * BK * 2;
+  int stages = (196 * 1024) / stage_bytes;
+  if (stages > MAX_STAGES) stages = MAX_STAGES;
+  p.stages = stages;
+  const size_t smem_bytes = (size_t)stages * stage_bytes + 1024 + 256;
+  if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "gemm: not enough shared memory"); return MSLT_ERR_CUDA; }
+
+  MapVal ma, mb;
+  const int nb = d.batch / d.hdiv;
+  if (d.batch % d.hdiv) { snprintf(err, 256, "gemm: batch must be a multiple of hdiv"); return MSLT_ERR_ARG; }
+  int rc = get_map(d.A, d.M, d.K, d.a_rs, d.a_ks, d.a_bo, d.a_bi, d.hdiv, nb, BM, &ma, err);
+  if (rc) return rc;
+  rc = get_map(d.B, d.N, d.K, d.b_rs, d.b_ks, d.b_bo, d.b_bi, d.hdiv, nb, p.bn, &mb, err);
+  if (rc) return rc;
+  for (int i = 0; i < 3; i++) { p.a_perm[i] = ma.perm[i]; p.b_perm[i] = mb.perm[i]; }
+
+  p.D = (char*)d.D; p.ldd = d.ldd; p.d_bo = d.d_bo; p.d_bi = d.d_bi;
+  p.d_fp32 = d.d_fp32; p.accumulate = d.accumulate; p.alpha = d.alpha; p.bias = d.bias; p.act = d.act;
+  p.aux = (bf16*)d.aux; p.residual = (const bf16*)d.residual; p.status = status;
+  // 16-byte vector access in the epilogue needs every row segment to start on a 16-byte boundary
+  // in each of the buffers it touches (bf16 ones are the stricter case: 8 elements)
+  auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
+  p.vec_ok = (d.ldd % 8 == 0 && d.d_bo % 8 == 0 && d.d_bi % 8 == 0 && al16(d.D) && al16(d.aux) &&
+              al16(d.residual) && al16(d.bias)) ? 1 : 0;
+  // instruction descriptor: fp32 accumulate, bf16 x bf16, operand majors, N and M of the tile
+  p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
+            ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    if (e != cudaSuccess) { snprintf(err, 256, "gemm: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+    attr_set = true;
+  }
+  const int grid = p.total_work < num_sms ? p.total_work : num_sms;
+  gemm_tc_kernel<<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { snprintf(err, 256, "gemm: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+  return 0;
+}
+
+}  // namespace mslt

@@ -1,0 +1,729 @@
+// Fused memory-bound kernels of the MSLT stage step: embedding gather + LayerNorm,
+// LayerNorm forward/backward, masked softmax forward/backward, MLM row
+// gather/scatter, softmax cross-entropy with in-place gradient, column sums for
+// bias gradients, embedding gradient scatter and Adam on the trainable slice.
+// All are HBM-bound: rows are moved with 16-byte accesses, one warp (or one
+// block) per row, reductions by warp shuffles, statistics in fp32.
+#include "kernels.h"
+
+#include <algorithm>
+
+#include "common.cuh"
+
+namespace mslt {
+
+constexpr int LN_MAXE = 32;  // elements of a row held by one lane: hidden <= 1024
+
+static inline int div_up(int64_t a, int64_t b) { return (int)((a + b - 1) / b); }
+
+// ---------------------------------------------------------------------------------------
+// LayerNorm forward.  y = gamma * (z - mean) * rstd + beta, biased variance.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__device__ __forceinline__ void ln_finish_row(float (&x)[LN_MAXE], int lane, int H,
+                                              const float* __restrict__ gamma,
+                                              const float* __restrict__ beta, T* __restrict__ yrow,
+                                              float* __restrict__ stat, float eps) {
+  constexpr int VN = VecT<T>::N;
+  constexpr int NV = LN_MAXE / VN;
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    if ((lane + 32 * i) * VN < H) {
+#pragma unroll
+      for (int e = 0; e < VN; e++) s += x[i * VN + e];
+    }
+  }
+  const float mean = warp_sum(s) / (float)H;
+  float q = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    if ((lane + 32 * i) * VN < H) {
+#pragma unroll
+      for (int e = 0; e < VN; e++) {
+        float d = x[i * VN + e] - mean;
+        q += d * d;
+      }
+    }
+  }
+  const float rstd = rsqrtf(warp_sum(q) / (float)H + eps);
+  if (stat != nullptr && lane == 0) {
+    stat[0] = mean;
+    stat[1] = rstd;
+  }
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < H) {
+      float o[VN];
+#pragma unroll
+      for (int e = 0; e < VN; e++)
+        o[e] = gamma[c + e] * ((x[i * VN + e] - mean) * rstd) + beta[c + e];
+      VecT<T>::store(yrow + c, o);
+    }
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) ln_fwd_kernel(const T* __restrict__ z,
+                                                     const float* __restrict__ gamma,
+                                                     const float* __restrict__ beta,
+                                                     T* __restrict__ y, float* __restrict__ stats,
+                                                     int rows, int H, float eps) {
+  constexpr int VN = VecT<T>::N;
+  constexpr int NV = LN_MAXE / VN;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  float x[LN_MAXE];
+  const T* zr = z + (int64_t)row * H;
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    float t[VN];
+    if (c < H) {
+      VecT<T>::load(zr + c, t);
+#pragma unroll
+      for (int e = 0; e < VN; e++) x[i * VN + e] = t[e];
+    }
+  }
+  ln_finish_row<T>(x, lane, H, gamma, beta, y + (int64_t)row * H,
+                   stats ? stats + 2 * (int64_t)row : nullptr, eps);
+}
+
+// Embedding: z = word[token] + pos[s]; optional stash of z; then LayerNorm.
+template <typename T>
+__global__ void __launch_bounds__(256)
+embed_ln_kernel(const int* __restrict__ tokens, const T* __restrict__ word,
+                const T* __restrict__ pos, const float* __restrict__ gamma,
+                const float* __restrict__ beta, T* __restrict__ y, T* __restrict__ zstash,
+                float* __restrict__ stats, int rows, int S, int H, int V, float eps,
+                int* __restrict__ status) {
+  constexpr int VN = VecT<T>::N;
+  constexpr int NV = LN_MAXE / VN;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  int tok = tokens[row];
+  if (tok < 0 || tok >= V) {
+    if (lane == 0) atomicOr(status, ST_BAD_TOKEN);
+    tok = 0;
+  }
+  const T* wr = word + (int64_t)tok * H;
+  const T* pr = pos + (int64_t)(row % S) * H;
+  float x[LN_MAXE];
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < H) {
+      float a[VN], b[VN];
+      VecT<T>::load(wr + c, a);
+      VecT<T>::load(pr + c, b);
+      // round the sum to the storage type first: the backward pass normalises the stashed copy
+#pragma unroll
+      for (int e = 0; e < VN; e++) a[e] = to_f<T>(from_f<T>(a[e] + b[e]));
+      if (zstash != nullptr) VecT<T>::store(zstash + (int64_t)row * H + c, a);
+#pragma unroll
+      for (int e = 0; e < VN; e++) x[i * VN + e] = a[e];
+    }
+  }
+  ln_finish_row<T>(x, lane, H, gamma, beta, y + (int64_t)row * H,
+                   stats ? stats + 2 * (int64_t)row : nullptr, eps);
+}
+
+// ---------------------------------------------------------------------------------------
+// LayerNorm backward: dz = rstd * (dxhat - mean(dxhat) - xhat * mean(dxhat * xhat)),
+// dgamma += sum_rows dy * xhat, dbeta += sum_rows dy (fp32 atomics, one per column per block).
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z, const float* __restrict__ stats,
+              const float* __restrict__ gamma, T* __restrict__ dz, float* __restrict__ dgamma,
+              float* __restrict__ dbeta, int rows, int H) {
+  constexpr int VN = VecT<T>::N;
+  constexpr int NV = LN_MAXE / VN;
+  __shared__ float red[8][LN_MAXE * 32];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int gw = blockIdx.x * 8 + warp, nw = gridDim.x * 8;
+  float ag[LN_MAXE], ab[LN_MAXE], g[LN_MAXE];
+#pragma unroll
+  for (int i = 0; i < LN_MAXE; i++) { ag[i] = 0.f; ab[i] = 0.f; g[i] = 0.f; }
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < H) {
+#pragma unroll
+      for (int e = 0; e < VN; e++) g[i * VN + e] = gamma[c + e];
+    }
+  }
+  const float invH = 1.0f / (float)H;
+  for (int row = gw; row < rows; row += nw) {
+    const float mean = stats[2 * (int64_t)row], rstd = stats[2 * (int64_t)row + 1];
+    float dyv[LN_MAXE], xh[LN_MAXE];
+    float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (lane + 32 * i) * VN;
+      if (c < H) {
+        float a[VN], b[VN];
+        VecT<T>::load(dy + (int64_t)row * H + c, a);
+        VecT<T>::load(z + (int64_t)row * H + c, b);
+#pragma unroll
+        for (int e = 0; e < VN; e++) {
+          const float xhat = (b[e] - mean) * rstd;
+          const float dxh = a[e] * g[i * VN + e];
+          dyv[i * VN + e] = dxh;
+          xh[i * VN + e] = xhat;
+          s1 += dxh;
+          s2 += dxh * xhat;
+          ag[i * VN + e] += a[e] * xhat;
+          ab[i * VN + e] += a[e];
+        }
+      }
+    }
+    s1 = warp_sum(s1) * invH;
+    s2 = warp_sum(s2) * invH;
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (lane + 32 * i) * VN;
+      if (c < H) {
+        float o[VN];
+#pragma unroll
+        for (int e = 0; e < VN; e++)
+          o[e] = rstd * (dyv[i * VN + e] - s1 - xh[i * VN + e] * s2);
+        VecT<T>::store(dz + (int64_t)row * H + c, o);
+      }
+    }
+  }
+  // block reduction of the column sums, then one atomic per column
+#pragma unroll
+  for (int pass = 0; pass < 2; pass++) {
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (lane + 32 * i) * VN;
+#pragma unroll
+      for (int e = 0; e < VN; e++)
+        red[warp][c + e] = pass == 0 ? ag[i * VN + e] : ab[i * VN + e];
+    }
+    __syncthreads();
+    float* dst = pass == 0 ? dgamma : dbeta;
+    for (int c = threadIdx.x; c < H; c += 256) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; w++) s += red[w][c];
+      atomicAdd(dst + c, s);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Scaled masked softmax over the last axis of [rows, S]; key j valid iff j < len(sequence).
+// ---------------------------------------------------------------------------------------
+constexpr int SM_MAXE = 16;  // S <= 512
+
+template <typename T>
+__global__ void __launch_bounds__(256)
+softmax_fwd_kernel(const T* __restrict__ sc, T* __restrict__ p, const int* __restrict__ seq_lens,
+                   int rows, int S, int rows_per_seq, float scale) {
+  constexpr int VN = VecT<T>::N;
+  constexpr int NV = SM_MAXE / VN;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  int len = seq_lens ? seq_lens[row / rows_per_seq] : S;
+  len = min(max(len, 1), S);
+  float x[SM_MAXE];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < S) {
+      float t[VN];
+      VecT<T>::load(sc + (int64_t)row * S + c, t);
+#pragma unroll
+      for (int e = 0; e < VN; e++) {
+        const float v = (c + e < len) ? t[e] * scale : -INFINITY;
+        x[i * VN + e] = v;
+        mx = fmaxf(mx, v);
+      }
+    }
+  }
+  mx = warp_max(mx);
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < S) {
+#pragma unroll
+      for (int e = 0; e < VN; e++) {
+        const float v = (c + e < len) ? expf(x[i * VN + e] - mx) : 0.f;
+        x[i * VN + e] = v;
+        s += v;
+      }
+    }
+  }
+  const float inv = 1.0f / warp_sum(s);
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < S) {
+      float o[VN];
+#pragma unroll
+      for (int e = 0; e < VN; e++) o[e] = x[i * VN + e] * inv;
+      VecT<T>::store(p + (int64_t)row * S + c, o);
+    }
+  }
+}
+
+// ds = p * (dp - sum_j dp * p) * scale, written over dp
+template <typename T>
+__global__ void __launch_bounds__(256)
+softmax_bwd_kernel(T* __restrict__ dp, const T* __restrict__ p, int rows, int S, float scale) {
+  constexpr int VN = VecT<T>::N;
+  constexpr int NV = SM_MAXE / VN;
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  if (row >= rows) return;
+  float a[SM_MAXE], b[SM_MAXE];
+  float dot = 0.f;
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < S) {
+      float t[VN], u[VN];
+      VecT<T>::load(dp + (int64_t)row * S + c, t);
+      VecT<T>::load(p + (int64_t)row * S + c, u);
+#pragma unroll
+      for (int e = 0; e < VN; e++) {
+        a[i * VN + e] = t[e];
+        b[i * VN + e] = u[e];
+        dot += t[e] * u[e];
+      }
+    }
+  }
+  dot = warp_sum(dot);
+#pragma unroll
+  for (int i = 0; i < NV; i++) {
+    const int c = (lane + 32 * i) * VN;
+    if (c < S) {
+      float o[VN];
+#pragma unroll
+      for (int e = 0; e < VN; e++) o[e] = b[i * VN + e] * (a[i * VN + e] - dot) * scale;
+      VecT<T>::store(dp + (int64_t)row * S + c, o);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// MLM slots: validity, source rows, labels, count; sequence-length check.
+// ---------------------------------------------------------------------------------------
+__global__ void slots_prepare_kernel(const int* __restrict__ positions,
+                                     const int* __restrict__ labels,
+                                     const int* __restrict__ seq_lens, int B, int S, int P, int V,
+                                     int* __restrict__ rowsrc, int* __restrict__ rowlabel,
+                                     int* __restrict__ n_valid, float* __restrict__ inv_n,
+                                     int* __restrict__ status) {
+  __shared__ int cnt;
+  if (threadIdx.x == 0) cnt = 0;
+  __syncthreads();
+  int local = 0, bad = 0;
+  for (int r = threadIdx.x; r < B * P; r += blockDim.x) {
+    const int b = r / P;
+    const int pos = positions[r];
+    const int lab = labels ? labels[r] : 0;
+    bool ok = pos >= 0 && lab >= 0;
+    if (pos >= S) { bad |= ST_BAD_POSITION; ok = false; }
+    if (lab >= V) { bad |= ST_BAD_LABEL; ok = false; }
+    rowsrc[r] = ok ? b * S + pos : -1;
+    rowlabel[r] = ok ? lab : -1;
+    local += ok ? 1 : 0;
+  }
+  if (seq_lens != nullptr) {
+    for (int b = threadIdx.x; b < B; b += blockDim.x)
+      if (seq_lens[b] < 1 || seq_lens[b] > S) bad |= ST_BAD_LENGTH;
+  }
+  if (local) atomicAdd(&cnt, local);
+  if (bad) atomicOr(status, bad);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    *n_valid = cnt;
+    *inv_n = cnt > 0 ? 1.0f / (float)cnt : 0.f;
+  }
+}
+
+// hm[r,:] = x[rowsrc[r],:], or zero for an empty slot
+template <typename T>
+__global__ void gather_rows_kernel(const T* __restrict__ x, const int* __restrict__ rowsrc,
+                                   T* __restrict__ out, int R, int H) {
+  constexpr int VN = VecT<T>::N;
+  const int r = blockIdx.x;
+  const int src = rowsrc[r];
+  for (int c = threadIdx.x * VN; c < H; c += blockDim.x * VN) {
+    float t[VN];
+    if (src >= 0) {
+      VecT<T>::load(x + (int64_t)src * H + c, t);
+    } else {
+#pragma unroll
+      for (int e = 0; e < VN; e++) t[e] = 0.f;
+    }
+    VecT<T>::store(out + (int64_t)r * H + c, t);
+  }
+}
+
+// dx[rowsrc[r],:] += d[r,:]; one block per sequence walks its slots in order, so repeated
+// positions add up without atomics.  dx must be zeroed beforehand.
+template <typename T>
+__global__ void scatter_rows_kernel(const T* __restrict__ d, const int* __restrict__ rowsrc,
+                                    T* __restrict__ dx, int P, int H) {
+  constexpr int VN = VecT<T>::N;
+  const int b = blockIdx.x;
+  for (int c = threadIdx.x * VN; c < H; c += blockDim.x * VN) {
+    for (int j = 0; j < P; j++) {
+      const int r = b * P + j;
+      const int src = rowsrc[r];
+      if (src < 0) continue;
+      float a[VN], t[VN];
+      VecT<T>::load(dx + (int64_t)src * H + c, a);
+      VecT<T>::load(d + (int64_t)r * H + c, t);
+#pragma unroll
+      for (int e = 0; e < VN; e++) a[e] += t[e];
+      VecT<T>::store(dx + (int64_t)src * H + c, a);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Softmax cross-entropy over the vocabulary, one block per slot.  nll = logsumexp - logit[label];
+// dlogits = (softmax - onehot) * inv_n.  Empty slots get nll 0 and a zero gradient row.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+cross_entropy_kernel(const float* __restrict__ logits, int64_t ldl, const int* __restrict__ rowlabel,
+                     const float* __restrict__ inv_n, T* __restrict__ dlogits, int64_t ldd,
+                     float* __restrict__ nll, int V) {
+  constexpr int VN = VecT<T>::N;
+  __shared__ float sm[8], ss[8];
+  __shared__ float s_lse;
+  const int r = blockIdx.x;
+  const int label = rowlabel[r];
+  const float* lr = logits + (int64_t)r * ldl;
+  T* dr = dlogits ? dlogits + (int64_t)r * ldd : nullptr;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (label < 0) {
+    if (threadIdx.x == 0) nll[r] = 0.f;
+    if (dr != nullptr) {
+      float zero[VN];
+#pragma unroll
+      for (int e = 0; e < VN; e++) zero[e] = 0.f;
+      for (int64_t c = (int64_t)threadIdx.x * VN; c < ldd; c += 256 * VN) VecT<T>::store(dr + c, zero);
+    }
+    return;
+  }
+  // pass 1: running maximum and rescaled sum
+  float m = -INFINITY, s = 0.f;
+  for (int c = threadIdx.x * 4; c < V; c += 256 * 4) {
+    float4 v = *reinterpret_cast<const float4*>(lr + c);
+    float t[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      if (c + e < V) {
+        const float nm = fmaxf(m, t[e]);
+        s = s * expf(m - nm) + expf(t[e] - nm);
+        m = nm;
+      }
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, o);
+    const float os = __shfl_xor_sync(0xffffffffu, s, o);
+    const float nm = fmaxf(m, om);
+    s = (m == -INFINITY ? 0.f : s * expf(m - nm)) + (om == -INFINITY ? 0.f : os * expf(om - nm));
+    m = nm;
+  }
+  if (lane == 0) { sm[warp] = m; ss[warp] = s; }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float M = sm[0], Sx = ss[0];
+    for (int w = 1; w < 8; w++) {
+      const float nm = fmaxf(M, sm[w]);
+      Sx = (M == -INFINITY ? 0.f : Sx * expf(M - nm)) + (sm[w] == -INFINITY ? 0.f : ss[w] * expf(sm[w] - nm));
+      M = nm;
+    }
+    const float lse = M + logf(Sx);
+    s_lse = lse;
+    nll[r] = lse - lr[label];
+  }
+  __syncthreads();
+  if (dr == nullptr) return;
+  const float lse = s_lse;
+  const float inv = *inv_n;
+  for (int64_t c = (int64_t)threadIdx.x * VN; c < ldd; c += 256 * VN) {
+    float o[VN];
+#pragma unroll
+    for (int h = 0; h < VN / 4; h++) {
+      float4 v = *reinterpret_cast<const float4*>(lr + c + 4 * h);
+      o[4 * h] = v.x; o[4 * h + 1] = v.y; o[4 * h + 2] = v.z; o[4 * h + 3] = v.w;
+    }
+#pragma unroll
+    for (int e = 0; e < VN; e++) {
+      const int64_t j = c + e;
+      o[e] = j < V ? (expf(o[e] - lse) - (j == label ? 1.f : 0.f)) * inv : 0.f;
+    }
+    VecT<T>::store(dr + c, o);
+  }
+}
+
+__global__ void loss_reduce_kernel(const float* __restrict__ nll, int R,
+                                   const float* __restrict__ inv_n, float* __restrict__ loss) {
+  __shared__ float part[32];
+  float s = 0.f;
+  for (int r = threadIdx.x; r < R; r += blockDim.x) s += nll[r];
+  s = warp_sum(s);
+  if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    float t = 0.f;
+    for (int w = 0; w < (int)(blockDim.x >> 5); w++) t += part[w];
+    *loss = t * (*inv_n);
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Column sums (bias gradients): out[n] += sum_rows x[row, n].
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+colsum_kernel(const T* __restrict__ x, int64_t ld, int rows, int N, int rows_per_block,
+              float* __restrict__ out) {
+  constexpr int VN = VecT<T>::N;
+  __shared__ float red[8][32 * VN];
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const int c = (blockIdx.x * 32 + tx) * VN;
+  const int r0 = blockIdx.y * rows_per_block;
+  const int r1 = min(rows, r0 + rows_per_block);
+  float acc[VN];
+#pragma unroll
+  for (int e = 0; e < VN; e++) acc[e] = 0.f;
+  if (c < N) {
+    for (int r = r0 + ty; r < r1; r += 8) {
+      float t[VN];
+      VecT<T>::load(x + (int64_t)r * ld + c, t);
+#pragma unroll
+      for (int e = 0; e < VN; e++) acc[e] += t[e];
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < VN; e++) red[ty][tx * VN + e] = acc[e];
+  __syncthreads();
+  for (int i = threadIdx.x; i < 32 * VN; i += 256) {
+    const int col = blockIdx.x * 32 * VN + i;
+    if (col < N) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < 8; w++) s += red[w][i];
+      atomicAdd(out + col, s);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Embedding gradient: dword[token[t], :] += dz[t, :], dpos[t % S, :] += dz[t, :].
+// ---------------------------------------------------------------------------------------
+template <typename T>
+__global__ void embed_scatter_kernel(const T* __restrict__ dz, const int* __restrict__ tokens,
+                                     float* __restrict__ dword, float* __restrict__ dpos, int S,
+                                     int H, int V) {
+  constexpr int VN = VecT<T>::N;
+  const int t = blockIdx.x;
+  int tok = tokens[t];
+  if (tok < 0 || tok >= V) tok = 0;
+  float* wr = dword + (int64_t)tok * H;
+  float* pr = dpos + (int64_t)(t % S) * H;
+  for (int c = threadIdx.x * VN; c < H; c += blockDim.x * VN) {
+    float a[VN];
+    VecT<T>::load(dz + (int64_t)t * H + c, a);
+#pragma unroll
+    for (int e = 0; e < VN; e++) {
+      atomicAdd(wr + c + e, a[e]);
+      atomicAdd(pr + c + e, a[e]);
+    }
+  }
+}
+
+// ---------------------------------------------------------------------------------------
+// Adam with decoupled weight decay over a table of chunks of the trainable slice.
+// ---------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+adam_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ w,
+            const float* __restrict__ g, float* __restrict__ m, float* __restrict__ v,
+            bf16* __restrict__ wb, AdamHyper h) {
+  const AdamChunk ch = chunks[blockIdx.x];
+  const float decay = h.weight_decay * ch.decay;
+  for (int i = threadIdx.x * 4; i < ch.count; i += 256 * 4) {
+    const int64_t o = ch.offset + i;
+    float4 wv = *reinterpret_cast<float4*>(w + o);
+    const float4 gv = *reinterpret_cast<const float4*>(g + o);
+    float4 mv = *reinterpret_cast<float4*>(m + o);
+    float4 vv = *reinterpret_cast<float4*>(v + o);
+    float* wp = &wv.x; const float* gp = &gv.x; float* mp = &mv.x; float* vp = &vv.x;
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const float mm = h.beta1 * mp[e] + h.omb1 * gp[e];
+      const float vn = h.beta2 * vp[e] + h.omb2 * gp[e] * gp[e];
+      const float mh = mm * h.bc1, vh = vn * h.bc2;
+      wp[e] = wp[e] - h.lr * (mh / (sqrtf(vh) + h.eps) + decay * wp[e]);
+      mp[e] = mm;
+      vp[e] = vn;
+    }
+    *reinterpret_cast<float4*>(w + o) = wv;
+    *reinterpret_cast<float4*>(m + o) = mv;
+    *reinterpret_cast<float4*>(v + o) = vv;
+    if (wb != nullptr) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(wv.x, wv.y), hi = __floats2bfloat162_rn(wv.z, wv.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(wb + o) = pk;
+    }
+  }
+}
+
+// d[i] *= gelu'(u[i]) (MLM transform backward)
+template <typename T>
+__global__ void dgelu_kernel(T* __restrict__ d, const T* __restrict__ u, int64_t n) {
+  constexpr int VN = VecT<T>::N;
+  for (int64_t i = (blockIdx.x * (int64_t)blockDim.x + threadIdx.x) * VN; i < n;
+       i += (int64_t)gridDim.x * blockDim.x * VN) {
+    float a[VN], b[VN];
+    VecT<T>::load(d + i, a);
+    VecT<T>::load(u + i, b);
+#pragma unroll
+    for (int e = 0; e < VN; e++) a[e] *= gelu_grad_f(b[e]);
+    VecT<T>::store(d + i, a);
+  }
+}
+
+__global__ void f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restrict__ dst, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n;
+       i += (int64_t)gridDim.x * blockDim.x)
+    dst[i] = __float2bfloat16_rn(src[i]);
+}
+
+// ---------------------------------------------------------------------------------------
+// host launchers
+// ---------------------------------------------------------------------------------------
+#define DISPATCH_T(bf, ...)                 \
+  do {                                      \
+    if (bf) { using T = bf16; __VA_ARGS__; } \
+    else { using T = float; __VA_ARGS__; }   \
+  } while (0)
+
+void launch_ln_fwd(bool bf, const void* z, const float* gamma, const float* beta, void* y,
+                   float* stats, int rows, int H, float eps, cudaStream_t st) {
+  if (rows <= 0) return;
+  DISPATCH_T(bf, (ln_fwd_kernel<T><<<div_up(rows, 8), 256, 0, st>>>(
+                     (const T*)z, gamma, beta, (T*)y, stats, rows, H, eps)));
+}
+
+void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* pos,
+                     const float* gamma, const float* beta, void* y, void* zstash, float* stats,
+                     int rows, int S, int H, int V, float eps, int* status, cudaStream_t st) {
+  if (rows <= 0) return;
+  DISPATCH_T(bf, (embed_ln_kernel<T><<<div_up(rows, 8), 256, 0, st>>>(
+                     tokens, (const T*)word, (const T*)pos, gamma, beta, (T*)y, (T*)zstash, stats,
+                     rows, S, H, V, eps, status)));
+}
+
+void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, const float* gamma,
+                   void* dz, float* dgamma, float* dbeta, int rows, int H, cudaStream_t st) {
+  if (rows <= 0) return;
+  int blocks = std::min(div_up(rows, 8), 148 * 4);
+  DISPATCH_T(bf, (ln_bwd_kernel<T><<<blocks, 256, 0, st>>>((const T*)dy, (const T*)z, stats, gamma,
+                                                           (T*)dz, dgamma, dbeta, rows, H)));
+}
+
+void launch_softmax_fwd(bool bf, const void* sc, void* p, const int* seq_lens, int rows, int S,
+                        int rows_per_seq, float scale, cudaStream_t st) {
+  if (rows <= 0) return;
+  DISPATCH_T(bf, (softmax_fwd_kernel<T><<<div_up(rows, 8), 256, 0, st>>>(
+                     (const T*)sc, (T*)p, seq_lens, rows, S, rows_per_seq, scale)));
+}
+
+void launch_softmax_bwd(bool bf, void* dp, const void* p, int rows, int S, float scale,
+                        cudaStream_t st) {
+  if (rows <= 0) return;
+  DISPATCH_T(bf, (softmax_bwd_kernel<T><<<div_up(rows, 8), 256, 0, st>>>((T*)dp, (const T*)p, rows,
+                                                                        S, scale)));
+}
+
+void launch_slots_prepare(const int* positions, const int* labels, const int* seq_lens, int B,
+                          int S, int P, int V, int* rowsrc, int* rowlabel, int* n_valid,
+                          float* inv_n, int* status, cudaStream_t st) {
+  slots_prepare_kernel<<<1, 256, 0, st>>>(positions, labels, seq_lens, B, S, P, V, rowsrc, rowlabel,
+                                          n_valid, inv_n, status);
+}
+
+void launch_gather_rows(bool bf, const void* x, const int* rowsrc, void* out, int R, int H,
+                        cudaStream_t st) {
+  if (R <= 0) return;
+  DISPATCH_T(bf, (gather_rows_kernel<T><<<R, 128, 0, st>>>((const T*)x, rowsrc, (T*)out, R, H)));
+}
+
+void launch_scatter_rows(bool bf, const void* d, const int* rowsrc, void* dx, int B, int P, int H,
+                         cudaStream_t st) {
+  if (B <= 0 || P <= 0) return;
+  DISPATCH_T(bf, (scatter_rows_kernel<T><<<B, 128, 0, st>>>((const T*)d, rowsrc, (T*)dx, P, H)));
+}
+
+void launch_cross_entropy(bool bf, const float* logits, int64_t ldl, const int* rowlabel,
+                          const float* inv_n, void* dlogits, int64_t ldd, float* nll, int R, int V,
+                          cudaStream_t st) {
+  if (R <= 0) return;
+  DISPATCH_T(bf, (cross_entropy_kernel<T><<<R, 256, 0, st>>>(logits, ldl, rowlabel, inv_n,
+                                                            (T*)dlogits, ldd, nll, V)));
+}
+
+void launch_loss_reduce(const float* nll, int R, const float* inv_n, float* loss, cudaStream_t st) {
+  loss_reduce_kernel<<<1, 1024, 0, st>>>(nll, R, inv_n, loss);
+}
+
+void launch_colsum(bool bf, const void* x, int64_t ld, int rows, int N, float* out,
+                   cudaStream_t st) {
+  if (rows <= 0 || N <= 0) return;
+  const int vn = bf ? 8 : 4;
+  const int gx = div_up(N, 32 * vn);
+  int gy = std::max(1, std::min(div_up(rows, 64), (148 * 4 + gx - 1) / gx));
+  const int rpb = div_up(rows, gy);
+  gy = div_up(rows, rpb);
+  DISPATCH_T(bf, (colsum_kernel<T><<<dim3(gx, gy), 256, 0, st>>>((const T*)x, ld, rows, N, rpb, out)));
+}
+
+void launch_embed_scatter(bool bf, const void* dz, const int* tokens, float* dword, float* dpos,
+                          int rows, int S, int H, int V, cudaStream_t st) {
+  if (rows <= 0) return;
+  DISPATCH_T(bf, (embed_scatter_kernel<T><<<rows, 128, 0, st>>>((const T*)dz, tokens, dword, dpos, S,
+                                                               H, V)));
+}
+
+void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,
+                 void* wb, const AdamHyper& h, cudaStream_t st) {
+  if (n_chunks <= 0) return;
+  adam_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, g, m, v, (bf16*)wb, h);
+}
+
+void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st) {
+  if (n <= 0) return;
+  const int vn = bf ? 8 : 4;
+  int blocks = (int)std::min<int64_t>((n / vn + 255) / 256, 148 * 8);
+  DISPATCH_T(bf, (dgelu_kernel<T><<<blocks, 256, 0, st>>>((T*)d, (const T*)u, n)));
+}
+
+void launch_f32_to_bf16(const float* src, void* dst, int64_t n, cudaStream_t st) {
+  if (n <= 0) return;
+  int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
+  f32_to_bf16_kernel<<<blocks, 256, 0, st>>>(src, (bf16*)dst, n);
+}
+
+}  // namespace mslt

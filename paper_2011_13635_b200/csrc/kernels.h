@@ -1,0 +1,55 @@
+// Host-side launchers of the fused memory-bound kernels (kernels.cu).
+// `bf` selects the activation type: true = bf16, false = float.  All pointers are device
+// pointers; every launcher only enqueues work on `st`.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace mslt {
+
+struct AdamChunk {
+  int64_t offset;  // element offset into the parameter arena (multiple of 4)
+  int32_t count;   // elements in this chunk (multiple of 4)
+  float decay;     // 1 for matrices and tables, 0 for vectors
+};
+struct AdamHyper {
+  float lr, beta1, beta2, eps, weight_decay;
+  float omb1, omb2;  // 1 - beta, formed in double on the host
+  float bc1, bc2;    // bias corrections 1 / (1 - beta^t), or 1
+};
+
+void launch_ln_fwd(bool bf, const void* z, const float* gamma, const float* beta, void* y,
+                   float* stats, int rows, int H, float eps, cudaStream_t st);
+void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* pos,
+                     const float* gamma, const float* beta, void* y, void* zstash, float* stats,
+                     int rows, int S, int H, int V, float eps, int* status, cudaStream_t st);
+void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, const float* gamma,
+                   void* dz, float* dgamma, float* dbeta, int rows, int H, cudaStream_t st);
+void launch_softmax_fwd(bool bf, const void* sc, void* p, const int* seq_lens, int rows, int S,
+                        int rows_per_seq, float scale, cudaStream_t st);
+void launch_softmax_bwd(bool bf, void* dp, const void* p, int rows, int S, float scale,
+                        cudaStream_t st);
+void launch_slots_prepare(const int* positions, const int* labels, const int* seq_lens, int B,
+                          int S, int P, int V, int* rowsrc, int* rowlabel, int* n_valid,
+                          float* inv_n, int* status, cudaStream_t st);
+void launch_gather_rows(bool bf, const void* x, const int* rowsrc, void* out, int R, int H,
+                        cudaStream_t st);
+void launch_scatter_rows(bool bf, const void* d, const int* rowsrc, void* dx, int B, int P, int H,
+                         cudaStream_t st);
+// logits fp32 [R, ldl]; dlogits (activation type) [R, ldd] or null; ldl >= ldd, both multiples of 8
+void launch_cross_entropy(bool bf, const float* logits, int64_t ldl, const int* rowlabel,
+                          const float* inv_n, void* dlogits, int64_t ldd, float* nll, int R, int V,
+                          cudaStream_t st);
+void launch_loss_reduce(const float* nll, int R, const float* inv_n, float* loss, cudaStream_t st);
+// out[n] += sum over rows; N a multiple of the 16-byte vector width, out has room for N floats
+void launch_colsum(bool bf, const void* x, int64_t ld, int rows, int N, float* out,
+                   cudaStream_t st);
+void launch_embed_scatter(bool bf, const void* dz, const int* tokens, float* dword, float* dpos,
+                          int rows, int S, int H, int V, cudaStream_t st);
+void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,
+                 void* wb, const AdamHyper& h, cudaStream_t st);
+// d[i] *= gelu'(u[i]); n a multiple of the vector width
+void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st);
+void launch_f32_to_bf16(const float* src, void* dst, int64_t n, cudaStream_t st);
+
+}  // namespace mslt

@@ -1,0 +1,117 @@
+"""Shared helpers of the GPU parity tests: drive the CUDA library and the CPU oracle on the
+same seeded inputs and compare them element by element."""
+from __future__ import annotations
+
+import numpy as np
+
+from oracle import mslt_oracle as O
+from paper_2011_13635_b200 import inputs as I
+
+# Tolerances (loss: relative; tensors: max-abs error over max-abs reference value).
+#   fp32 path: every contraction accumulates in fp32 in k order, statistics in fp32.
+#   bf16 path: activations, saved activations and activation gradients are rounded to bf16
+#   (relative 2^-9 per rounding); weight gradients accumulate in fp32.
+TOL = {"fp32": dict(loss=2e-3, grad=1e-4, weight=1e-4, hidden=1e-4, update_l1=2e-3),
+       "bf16": dict(loss=2e-3, grad=3e-2, weight=3e-2, hidden=3e-2, update_l1=0.15)}
+
+
+def max_rel(a: np.ndarray, r: np.ndarray) -> float:
+    """max_i |a_i - r_i| / max_i |r_i|."""
+    a = np.asarray(a, dtype=np.float64)
+    r = np.asarray(r, dtype=np.float64)
+    den = np.abs(r).max()
+    num = np.abs(a - r).max()
+    if den == 0.0:
+        return 0.0 if num == 0.0 else float("inf")
+    return float(num / den)
+
+
+def to_cuda(torch, *arrays):
+    return [None if a is None else torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in arrays]
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Round-to-nearest-even fp32 -> bf16 bit patterns (uint16), by integer arithmetic."""
+    u = np.ascontiguousarray(x, dtype=np.float32).view(np.uint32).astype(np.uint64)
+    bias = ((u >> 16) & 1) + 0x7FFF
+    return ((u + bias) >> 16).astype(np.uint16)
+
+
+def build_pair(cfg: I.StageConfig, lr: float, max_layers=None, init_layers=None, seed=None, **opt):
+    """(library context, oracle) with identical weights, boundary and hyper-parameters."""
+    from paper_2011_13635_b200.binding import Mslt
+    L0 = cfg.layers if init_layers is None else init_layers
+    w = I.make_weights(cfg, seed=seed, variant="parity", n_layers=L0)
+    oracle = O.MsltOracle(w, cfg.heads, ln_eps=1e-12, max_layers=max_layers or cfg.layers)
+    hyper = dict(I.ADAM_DEFAULTS)
+    hyper.update(opt)
+    hyper["lr"] = lr
+    # both sides get the same numbers: the C ABI carries hyper-parameters as float32
+    hyper = {k: (float(np.float32(v)) if k != "bias_correction" else v) for k, v in hyper.items()}
+    oracle.set_optimizer(**hyper)
+    m = Mslt.from_config(cfg, init_layers=L0, max_layers=max_layers or cfg.layers)
+    m.set_params(w)
+    m.mslt_set_optimizer(**hyper)
+    if init_layers is None:
+        oracle.set_trainable(cfg.trainable)
+        m.mslt_set_trainable(cfg.trainable)
+    return m, oracle
+
+
+def compare_step(m, oracle, cfg, batch, tol, report=None):
+    """One step on both sides; asserts loss, gradients, weights and the frozen slice."""
+    import torch
+    tok, lens, pos, lab = batch
+    names = oracle.trainable_names()
+    all_names = list(oracle.p.keys())
+    frozen = [n for n in all_names if n not in names]
+    w_before = {n: m.mslt_get_param(n) for n in names}
+    m_before = {n: m.mslt_get_opt_state(n, 0) for n in names}
+    v_before = {n: m.mslt_get_opt_state(n, 1) for n in names}
+    raw_frozen = {n: (m.mslt_get_param(n), m.mslt_get_param_raw(n)) for n in frozen}
+    ow_before = {n: oracle.p[n].copy() for n in names}
+
+    d_tok, d_lens, d_pos, d_lab = to_cuda(torch, tok, lens if cfg.varlen else None, pos, lab)
+    loss_g = m.mslt_step(d_tok, d_lens, d_pos, d_lab)
+    loss_o = oracle.step(tok, lens, pos, lab)
+    rel_loss = abs(loss_g - loss_o) / abs(loss_o)
+    assert rel_loss < tol["loss"], (loss_g, loss_o)
+
+    worst = dict(grad=("", 0.0), weight=("", 0.0), update=("", 0.0))
+    o = oracle.opt
+    t = oracle.t
+    for n in names:
+        g = m.mslt_get_grad(n)
+        e = max_rel(g, oracle.grads[n])
+        if e > worst["grad"][1]:
+            worst["grad"] = (n, e)
+        assert e < tol["grad"], ("grad", n, e)
+        w_after = m.mslt_get_param(n)
+        e = max_rel(w_after, oracle.p[n])
+        if e > worst["weight"][1]:
+            worst["weight"] = (n, e)
+        assert e < tol["weight"], ("weight", n, e)
+        # the update itself: mean |dw - dw_ref| / mean |dw_ref| (Adam's first steps are
+        # sign-like, so single elements with a near-zero gradient may flip under rounding)
+        dw, dwo = w_after - w_before[n], oracle.p[n] - ow_before[n]
+        e = float(np.abs(dw - dwo).mean() / max(np.abs(dwo).mean(), 1e-30))
+        if e > worst["update"][1]:
+            worst["update"] = (n, e)
+        assert e < tol["update_l1"], ("update", n, e)
+        # the Adam kernel alone: the oracle's update formula applied to the library's own inputs
+        wd = o["weight_decay"] if w_before[n].ndim == 2 else 0.0
+        w_ref, m_ref, v_ref = O.adam_update(w_before[n].astype(np.float64), g.astype(np.float64),
+                                            m_before[n].astype(np.float64), v_before[n].astype(np.float64),
+                                            t, o["lr"], o["beta1"], o["beta2"], o["eps"], wd,
+                                            bool(o["bias_correction"]))
+        assert max_rel(w_after, w_ref) < 2e-6, ("adam w", n)
+        assert max_rel(m.mslt_get_opt_state(n, 0), m_ref) < 2e-6, ("adam m", n)
+        assert max_rel(m.mslt_get_opt_state(n, 1), v_ref) < 2e-6, ("adam v", n)
+        if cfg.dtype == "bf16" and w_after.ndim == 2:
+            assert np.array_equal(m.mslt_get_param_raw(n), bf16_round(w_after)), ("bf16 copy", n)
+    for n in frozen:
+        assert np.array_equal(m.mslt_get_param(n), raw_frozen[n][0]), ("frozen master moved", n)
+        assert np.array_equal(m.mslt_get_param_raw(n), raw_frozen[n][1]), ("frozen copy moved", n)
+    if report is not None:
+        report.append(dict(loss_gpu=loss_g, loss_oracle=loss_o, rel_loss=rel_loss, **worst))
+    return loss_g, loss_o, worst
