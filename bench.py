@@ -1,0 +1,323 @@
+"""Benchmark of the MSLT per-stage BERT training step on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config NAME] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path (frozen-prefix forward, trainable forward and
+backward, MLM head and loss, Adam on the trainable slice) over one synthetic batch.  The path
+does not shard: with N > 1 every rank runs an independent replica on its own batch (no
+collective on the data path) and the aggregate throughput is reported.
+
+Prints ONE JSON line (rank 0).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2011_13635_b200 import inputs as I  # noqa: E402
+
+METRIC = "sequences/sec per MSLT stage step"
+UNIT = "sequences/s"
+
+
+def measured_peaks():
+    """Measured B200 peaks of this machine; the stated earlier measurement if the file is absent."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return dict(hbm_gbs=d["hbm_gbs"], bf16_tflops=d["bf16_tflops"],
+                    bf16_tflops_sustained=d.get("bf16_tflops_sustained", d["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def step_flops(cfg: I.StageConfig) -> float:
+    """Dense floating-point operations of one step (2*M*N*K per contraction)."""
+    T, H, S, L, k = cfg.batch * cfg.seq, cfg.hidden, cfg.seq, cfg.layers, cfg.trainable
+    R, V = cfg.batch * cfg.pred, cfg.vocab
+    fwd_layer = 24.0 * T * H * H + 4.0 * T * S * H
+    total = L * fwd_layer + k * 2 * fwd_layer
+    if 0 < k < L:
+        total -= 6.0 * T * H * H          # no input gradient below the frozen boundary
+    total += 2.0 * R * H * H + 2.0 * R * H * V          # head forward
+    total += 4.0 * R * H * H + 2.0 * R * H * V          # head backward
+    if k == L:
+        total += 2.0 * R * H * V                        # decoder weight gradient
+    return total
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def __enter__(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+        return self
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def __exit__(self, *exc):
+        if self.proc is not None:
+            time.sleep(0.15)
+            self.proc.terminate()
+            self.thread.join(timeout=2)
+
+    def summary(self):
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except (ValueError, IndexError):
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+def describe(cfg: I.StageConfig) -> dict:
+    return dict(workload=f"{cfg.name}: {cfg.layers} layers ({cfg.frozen} frozen + {cfg.trainable} "
+                         f"trainable), hidden {cfg.hidden}, heads {cfg.heads}, ffn {cfg.ffn}, vocab "
+                         f"{cfg.vocab}, seq {cfg.seq}, batch {cfg.batch} per GPU, {cfg.pred} MLM slots",
+                batch_per_gpu=cfg.batch, seq_len=cfg.seq, layers=cfg.layers, frozen=cfg.frozen,
+                trainable=cfg.trainable, parallelism="replicas only (no collective)",
+                l2="working set of one step (GBs of weights and activations) exceeds the 126 MB L2")
+
+
+# ------------------------------------------------------------------------------------------------
+# reference arm: the CPU oracle, as it stands, on a bounded sample of the workload
+# ------------------------------------------------------------------------------------------------
+def oracle_sample(cfg: I.StageConfig, n_seq: int):
+    from oracle import mslt_oracle as O      # the one place bench.py may touch oracle/
+    small = I.scaled(cfg, batch=n_seq)
+    w = I.make_weights(small, variant="bench")
+    m = O.MsltOracle(w, small.heads)
+    m.set_trainable(small.trainable)
+    return m, I.make_batch(small), small
+
+
+def host_threads() -> int:
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return int(max(n)) if n else (os.cpu_count() or 1)
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def cpu_baseline(cfg: I.StageConfig, n_seq: int, steps: int = 1, warmup: int = 0):
+    m, batch, small = oracle_sample(cfg, n_seq)
+    for _ in range(warmup):
+        m.step(*batch)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        m.step(*batch)
+    dt = time.perf_counter() - t0
+    return dict(value=n_seq * steps / dt, unit=UNIT, cores=host_threads(), kind="oracle",
+                sample=f"{steps} step(s) of the float64 numpy oracle on {n_seq} of the {cfg.batch} "
+                       f"sequences of the batch, full architecture ({dt:.1f} s)"), dt
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    n_seq = 2
+    base, dt = cpu_baseline(cfg, n_seq, steps=args.steps, warmup=args.warmup)
+    line = dict(impl="reference", metric=METRIC, value=base["value"], unit=UNIT, n_gpus=args.gpus,
+                steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * dt / args.steps,
+                higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
+                config=describe(cfg), cpu_baseline=base,
+                e2e=dict(value=base["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------------------------
+# our arm
+# ------------------------------------------------------------------------------------------------
+def make_model(cfg, torch):
+    from paper_2011_13635_b200.binding import Mslt
+    m = Mslt.from_config(cfg)
+    m.set_params(I.make_weights(cfg, variant="bench"))
+    m.mslt_set_trainable(cfg.trainable)
+    m.mslt_set_optimizer(**I.ADAM_DEFAULTS)
+    return m
+
+
+def time_steps(m, dev, torch, steps, warmup, sync_fn):
+    tok, lens, pos, lab = dev
+    for _ in range(warmup):
+        m.mslt_step(tok, lens, pos, lab, sync=False)
+    sync_fn()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    before = m.launch_count
+    e0.record()
+    for _ in range(steps):
+        m.mslt_step(tok, lens, pos, lab, sync=False)
+    e1.record()
+    sync_fn()
+    return e0.elapsed_time(e1), m.launch_count - before
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    def sync():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    host = [np.ascontiguousarray(a) for a in I.make_batch(cfg, seed=I.config_seed(cfg) + 1000 * rank)]
+    if cfg.varlen is None:
+        host[1] = None
+    pinned = [None if a is None else torch.from_numpy(a).pin_memory() for a in host]
+    dev = [None if a is None else a.cuda(non_blocking=True) for a in pinned]
+    m = make_model(cfg, torch)
+    loss0 = m.mslt_step(*dev)                       # also checks the device status word
+    if not np.isfinite(loss0):
+        raise RuntimeError("non-finite loss")
+
+    with ClockSampler(local) as clk:
+        ms, launches = time_steps(m, dev, torch, args.steps, args.warmup, sync)
+    loss_end = m.mslt_read_loss()
+    t = torch.tensor([ms], device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    value = cfg.batch * world * args.steps / (ms * 1e-3)
+
+    # end to end: pinned host inputs copied in, loss read back, every step
+    sync()
+    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for _ in range(args.steps):
+        d = [None if a is None else a.cuda(non_blocking=True) for a in pinned]
+        m.mslt_step(*d)
+    t1.record()
+    sync()
+    te = torch.tensor([t0.elapsed_time(t1)], device="cuda")
+    if world > 1:
+        dist.all_reduce(te, op=dist.ReduceOp.MAX)
+    e2e = dict(value=cfg.batch * world * args.steps / (float(te.item()) * 1e-3), unit=UNIT,
+               h2d_bytes_per_step=int(sum(a.nbytes for a in host if a is not None)),
+               d2h_bytes_per_step=16)
+
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
+                warmup=args.warmup, ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype=cfg.dtype, data="synthetic", config=describe(cfg), e2e=e2e,
+                gpu_launches=int(launches), clocks=clk.summary(),
+                loss=dict(first=loss0, last=loss_end))
+
+    if rank == 0:
+        peaks = measured_peaks()
+        # per-kernel pass: the same steps again with an event pair around every contraction
+        m.mslt_set_timing(2)
+        m.mslt_get_gemm_profile()
+        n_prof = max(1, min(args.steps, 5))
+        for _ in range(n_prof):
+            m.mslt_step(*dev, sync=False)
+        torch.cuda.synchronize()
+        prof = m.mslt_get_gemm_profile()
+        phases = m.mslt_get_timings()
+        m.mslt_set_timing(0)
+        lin, att = prof["linear"], prof["attention"]
+        lin_tflops = lin["flops"] / (lin["ms"] * 1e-3) / 1e12 if lin["ms"] > 0 else 0.0
+        peak = peaks["bf16_tflops_sustained"] if cfg.dtype == "bf16" else None
+        if cfg.dtype == "bf16":
+            line["roofline"] = dict(
+                bound="tensor", kernel="gemm_tc_kernel (linear-layer products of the step)",
+                achieved=lin_tflops, peak=peak, unit="TFLOP/s", frac=lin_tflops / peak, traffic=None,
+                peak_source=f"{peaks['source']}: cuBLAS bf16 sustained (kernel timed inside a long step)",
+                launches_per_step=lin["launches"] / n_prof,
+                avg_launch_us=1e3 * lin["ms"] / max(lin["launches"], 1),
+                flops_per_step=lin["flops"] / n_prof,
+                share_of_step_time=lin["ms"] / n_prof / (ms / args.steps))
+        else:
+            line["roofline"] = dict(bound="alu", kernel="gemm_simt_kernel", achieved=lin_tflops, peak=None,
+                                    unit="TFLOP/s", frac=None, traffic=None)
+        line["attention_gemms"] = dict(
+            tflops=att["flops"] / (att["ms"] * 1e-3) / 1e12 if att["ms"] > 0 else 0.0,
+            ms_per_step=att["ms"] / n_prof, launches_per_step=att["launches"] / n_prof)
+        line["phases_ms"] = phases
+        line["step_tflops"] = step_flops(cfg) / (ms / args.steps * 1e-3) / 1e12
+        m.close()
+        del m
+        torch.cuda.empty_cache()
+        if world == 1 and args.ratio and cfg.name == "base_stage":
+            full = I.CONFIGS["base_full"]
+            mf = make_model(full, torch)
+            k = max(3, min(args.steps, 10))
+            ms_f, _ = time_steps(mf, dev, torch, k, 3, sync)
+            line["stage_vs_full"] = dict(
+                staged_ms=ms / args.steps, full_ms=ms_f / k, ratio=(ms / args.steps) / (ms_f / k),
+                note="step time of 9 frozen + 3 trainable layers over all 12 trainable, same shapes, "
+                     "data and seed, one GPU, no communication")
+            mf.close()
+        if world == 1:
+            n_seq = args.cpu_seqs
+            line["cpu_baseline"], _ = cpu_baseline(cfg, n_seq)
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="base_stage", choices=sorted(I.CONFIGS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-seqs", type=int, default=8, help="sequences in the oracle's timed sample")
+    ap.add_argument("--no-ratio", dest="ratio", action="store_false")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    cfg = I.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

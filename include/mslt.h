@@ -163,6 +163,11 @@ int64_t mslt_launch_count(const mslt_ctx* ctx);
  * [4] Adam.  Turning timing on adds event records and one synchronisation per step. */
 int mslt_set_timing(mslt_ctx* ctx, int32_t on);
 int mslt_get_timings(mslt_ctx* ctx, float* host_ms, int32_t n);
+/* Timing level 2 (mslt_set_timing(ctx, 2)) also brackets every contraction of a step with an
+ * event pair.  This call returns and clears what has been accumulated since the last call, as 6
+ * host doubles: for the linear-layer products, then for the batched attention products:
+ * launches, floating-point operations (2*M*N*K*batch), milliseconds. */
+int mslt_get_gemm_profile(mslt_ctx* ctx, double* host_out, int32_t n);
 /* Message for the last error on this thread (ctx may be NULL). */
 const char* mslt_last_error(const mslt_ctx* ctx);
 

@@ -51,7 +51,8 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_set_optimizer", "mslt_step", "mslt_read_loss", "mslt_forward", "mslt_num_layers",
            "mslt_num_trainable", "mslt_num_tensors", "mslt_tensor_info", "mslt_get_param",
            "mslt_set_param", "mslt_get_param_raw", "mslt_get_grad", "mslt_get_opt_state",
-           "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_last_error",
+           "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_gemm_profile",
+           "mslt_last_error",
            "mslt_op_gemm"]
 
 lib.mslt_last_error.restype = C.c_char_p
@@ -82,6 +83,7 @@ lib.mslt_get_grad.argtypes = [C.c_void_p, C.c_char_p, C.c_void_p, C.c_size_t]
 lib.mslt_get_opt_state.argtypes = [C.c_void_p, C.c_char_p, C.c_int32, C.c_void_p, C.c_size_t]
 lib.mslt_set_timing.argtypes = [C.c_void_p, C.c_int32]
 lib.mslt_get_timings.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+lib.mslt_get_gemm_profile.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
 lib.mslt_op_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
 
 
@@ -253,8 +255,14 @@ class Mslt:
         _check(lib.mslt_get_opt_state(self.h, name.encode(), which, out.ctypes.data, out.size))
         return out
 
-    def mslt_set_timing(self, on: bool):
-        _check(lib.mslt_set_timing(self.h, int(on)))
+    def mslt_set_timing(self, level: int):
+        _check(lib.mslt_set_timing(self.h, int(level)))
+
+    def mslt_get_gemm_profile(self) -> Dict[str, dict]:
+        buf = (C.c_double * 6)()
+        _check(lib.mslt_get_gemm_profile(self.h, buf, 6))
+        return {k: dict(launches=int(buf[3 * i]), flops=buf[3 * i + 1], ms=buf[3 * i + 2])
+                for i, k in enumerate(["linear", "attention"])}
 
     def mslt_get_timings(self) -> Dict[str, float]:
         buf = (C.c_float * 5)()

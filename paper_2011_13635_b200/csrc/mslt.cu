@@ -97,6 +97,12 @@ struct mslt_ctx {
   cudaEvent_t ev[6];
   float phase_ms[5];
   bool have_events;
+  // per-contraction profiling (timing level 2): one event pair per GEMM launch of a step
+  int profile;
+  std::vector<cudaEvent_t> pev;
+  struct PRec { int cls; double flops; };
+  std::vector<PRec> prec;
+  double prof[2][3];  // per class (0 linear, 1 batched attention): launches, flops, ms
 };
 
 namespace {
@@ -275,7 +281,13 @@ int run_gemm(mslt_ctx* c, const mslt_gemm_desc& d) {
   if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) return 0;
   char err[256] = "";
   const int64_t before = gemm_launches();
+  const bool prof = c->profile && c->prec.size() * 2 + 2 <= c->pev.size();
+  if (prof) cudaEventRecord(c->pev[2 * c->prec.size()], c->st);
   int rc = gemm_launch(d, c->ws.scalars, c->st, err);
+  if (prof) {
+    cudaEventRecord(c->pev[2 * c->prec.size() + 1], c->st);
+    c->prec.push_back({d.batch > 1 ? 1 : 0, 2.0 * d.M * d.N * (double)d.K * d.batch});
+  }
   c->launches += gemm_launches() - before;
   if (rc) return fail(rc, "%s", err);
   return 0;
@@ -547,6 +559,8 @@ int mslt_create(const mslt_arch* arch, void* dev_params, size_t param_bytes, voi
   c->launches = 0;
   c->timing = false;
   c->have_events = false;
+  c->profile = 0;
+  memset(c->prof, 0, sizeof(c->prof));
   c->Vp = (int)pad_to(arch->vocab, 8);
   build_tensor_table(*arch, c->tensors, c->n_elems);
   for (size_t i = 0; i < c->tensors.size(); i++) c->by_name[c->tensors[i].name] = (int)i;
@@ -584,6 +598,7 @@ int mslt_destroy(mslt_ctx* c) {
   if (!c) return 0;
   if (c->have_events)
     for (int i = 0; i < 6; i++) cudaEventDestroy(c->ev[i]);
+  for (cudaEvent_t e : c->pev) cudaEventDestroy(e);
   delete c;
   return 0;
 }
@@ -636,6 +651,7 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
     c->have_events = true;
   }
   CUDA_TRY(cudaMemsetAsync(w.scalars, 0, 16, c->st));
+  c->prec.clear();
   mark(c, 0);
   KL(launch_slots_prepare(d_pos, d_lab, d_seq_lens, B, S, P, V, w.rowsrc, w.rowlabel, w.scalars + 1,
                           inv_n, status, c->st));
@@ -691,6 +707,15 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   if (c->timing && c->have_events) {
     CUDA_TRY(cudaEventSynchronize(c->ev[5]));
     for (int i = 0; i < 5; i++) cudaEventElapsedTime(&c->phase_ms[i], c->ev[i], c->ev[i + 1]);
+  }
+  if (c->profile) {
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (size_t i = 0; i < c->prec.size(); i++) {
+      float ms = 0.f;
+      cudaEventElapsedTime(&ms, c->pev[2 * i], c->pev[2 * i + 1]);
+      double* a = c->prof[c->prec[i].cls];
+      a[0] += 1.0; a[1] += c->prec[i].flops; a[2] += ms;
+    }
   }
   return finish(c, loss_out);
 }
@@ -830,6 +855,19 @@ int64_t mslt_launch_count(const mslt_ctx* c) { return c ? c->launches : 0; }
 int mslt_set_timing(mslt_ctx* c, int32_t on) {
   if (!c) return fail(MSLT_ERR_ARG, "null context");
   c->timing = on != 0;
+  c->profile = on >= 2 ? 1 : 0;
+  if (c->profile && c->pev.empty()) {
+    c->pev.resize(2 * 1024);
+    for (cudaEvent_t& e : c->pev) CUDA_TRY(cudaEventCreate(&e));
+  }
+  return 0;
+}
+
+int mslt_get_gemm_profile(mslt_ctx* c, double* out, int32_t n) {
+  if (!c || !out || n < 6) return fail(MSLT_ERR_ARG, "need room for 6 doubles");
+  for (int k = 0; k < 2; k++)
+    for (int j = 0; j < 3; j++) out[3 * k + j] = c->prof[k][j];
+  memset(c->prof, 0, sizeof(c->prof));
   return 0;
 }
 
