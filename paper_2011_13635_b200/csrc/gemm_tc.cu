@@ -7,10 +7,11 @@
 //   warp 1   : allocates tensor memory and issues tcgen05.mma (one thread) for 128 x BN x 16
 //              steps; tcgen05.commit hands shared-memory stages back to the producer and
 //              accumulators over to the epilogue.
-//   warps 2-5: epilogue.  Each warp owns one 32-lane quarter of TMEM, reads the accumulator
-//              with tcgen05.ld and applies scale, bias, GELU / GELU', residual, then stores bf16
-//              or fp32 (plain or as vector reductions for split-k).  Two accumulators of up to 256
-//              columns let the epilogue of one tile overlap the main loop of the next.
+//   warps 2-9: epilogue.  Two warps per 32-lane quarter of TMEM read the accumulator with
+//              tcgen05.ld, apply scale, bias, GELU / GELU', residual, and store bf16 or fp32
+//              (plain, or as vector reductions for split-k) through a swizzled staging buffer so
+//              that global stores are whole row segments.  Two accumulators of up to 256 columns
+//              let the epilogue of one tile overlap the main loop of the next.
 // Operands may be k-contiguous ("K-major") or row-contiguous ("MN-major"); the second form is
 // what input-gradient and weight-gradient products need, and is fed to the tensor cores through
 // the MN-major shared-memory descriptor, so no transposed copies exist anywhere.
@@ -35,7 +36,9 @@ constexpr int BK = 64;            // k extent of a stage: 64 bf16 = one 128-byte
 constexpr int UMMA_K = 16;        // k extent of one tcgen05.mma for 16-bit operands
 constexpr int MAX_STAGES = 8;
 constexpr int A_STAGE_BYTES = BM * BK * 2;
-constexpr int NUM_THREADS = 192;
+constexpr int NUM_EPI_WARPS = 8;
+constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
+constexpr int STAGING_BYTES = 4096;  // per epilogue warp
 constexpr uint32_t TMEM_COLS = 512;
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
 
@@ -161,6 +164,110 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
   return d;
 }
 
+// erf by the rational-times-exponential form of Abramowitz & Stegun 7.1.26 (absolute error
+// below 1.5e-7, far inside bf16 resolution); the exponential exp(-x^2) with x = u / sqrt(2) is
+// also the Gaussian factor the derivative needs.
+__device__ __forceinline__ void erf_parts(float u, float& erf_v, float& gauss) {
+  const float x = u * 0.70710678118654752f;
+  const float ax = fabsf(x);
+  const float t = __fdividef(1.0f, fmaf(0.3275911f, ax, 1.0f));
+  gauss = __expf(-ax * ax);
+  float poly = fmaf(t, 1.061405429f, -1.453152027f);
+  poly = fmaf(t, poly, 1.421413741f);
+  poly = fmaf(t, poly, -0.284496736f);
+  poly = fmaf(t, poly, 0.254829592f);
+  erf_v = copysignf(1.0f - poly * t * gauss, x);
+}
+__device__ __forceinline__ float gelu_fast(float u) {
+  float e, g;
+  erf_parts(u, e, g);
+  return 0.5f * u * (1.0f + e);
+}
+__device__ __forceinline__ float gelu_grad_fast(float u) {
+  float e, g;
+  erf_parts(u, e, g);
+  return 0.5f * (1.0f + e) + u * g * 0.39894228040143268f;
+}
+
+// Staging buffer of one epilogue warp: 32 rows of 128 bytes.  Lane r writes its row as 16-byte
+// pieces; the slot functions permute the pieces so that both this row-per-lane write and the
+// row-segment-per-quarter-warp read that follows are free of bank conflicts.
+__device__ __forceinline__ uint32_t slot_f32(int r, int c) {  // c in 0..7: 8 pieces of 4 floats
+  return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
+}
+__device__ __forceinline__ uint32_t slot_b16(int r, int c) {  // c in 0..3: 4 pieces of 8 bf16
+  return (uint32_t)(r * 128 + (((c + ((r & 1) << 2)) ^ ((r >> 1) & 3)) << 4));
+}
+
+// Writes a 32 x 32 chunk (lane = row, v = its 32 columns) to `base` (row-major, leading dimension
+// ldd, element (m_warp + row, n0 + col)) with coalesced 16-byte stores.
+__device__ __forceinline__ void stage_store_bf16(uint8_t* stg, int lane, const float (&v)[32], bf16* base,
+                                                 long long ldd, int m_warp, int n0, int M, int N,
+                                                 int vec_ok) {
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    uint4 pk;
+    __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+    for (int e = 0; e < 4; e++) h[e] = __floats2bfloat162_rn(v[8 * c + 2 * e], v[8 * c + 2 * e + 1]);
+    *reinterpret_cast<uint4*>(stg + slot_b16(lane, c)) = pk;
+  }
+  __syncwarp();
+#pragma unroll
+  for (int it = 0; it < 4; it++) {
+    const int row = it * 8 + (lane >> 2), c = lane & 3;
+    const uint4 val = *reinterpret_cast<const uint4*>(stg + slot_b16(row, c));
+    const int mm = m_warp + row, nn = n0 + c * 8;
+    if (mm < M && nn < N) {
+      bf16* dst = base + (long long)mm * ldd + nn;
+      if (vec_ok && nn + 8 <= N) {
+        *reinterpret_cast<uint4*>(dst) = val;
+      } else {
+        const bf16* e8 = reinterpret_cast<const bf16*>(&val);
+#pragma unroll
+        for (int e = 0; e < 8; e++)
+          if (nn + e < N) dst[e] = e8[e];
+      }
+    }
+  }
+  __syncwarp();
+}
+
+__device__ __forceinline__ void stage_store_f32(uint8_t* stg, int lane, const float (&v)[32], float* base,
+                                                long long ldd, int m_warp, int n0, int M, int N, int vec_ok,
+                                                int accumulate) {
+#pragma unroll
+  for (int c = 0; c < 8; c++)
+    *reinterpret_cast<float4*>(stg + slot_f32(lane, c)) =
+        make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+  __syncwarp();
+#pragma unroll
+  for (int it = 0; it < 8; it++) {
+    const int row = it * 4 + (lane >> 3), c = lane & 7;
+    const float4 val = *reinterpret_cast<const float4*>(stg + slot_f32(row, c));
+    const int mm = m_warp + row, nn = n0 + c * 4;
+    if (mm < M && nn < N) {
+      float* dst = base + (long long)mm * ldd + nn;
+      if (vec_ok && nn + 4 <= N) {
+        if (accumulate)
+          asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(val.x), "f"(val.y),
+                       "f"(val.z), "f"(val.w)
+                       : "memory");
+        else
+          *reinterpret_cast<float4*>(dst) = val;
+      } else {
+        const float e4[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+        for (int e = 0; e < 4; e++)
+          if (nn + e < N) {
+            if (accumulate) atomicAdd(dst + e, e4[e]); else dst[e] = e4[e];
+          }
+      }
+    }
+  }
+  __syncwarp();
+}
+
 // ---- the kernel ---------------------------------------------------------------------------------
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -170,7 +277,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   const int b_stage_bytes = p.bn * BK * 2;
   const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
-  uint64_t* bars = (uint64_t*)(smem + (size_t)p.stages * stage_bytes);
+  uint8_t* staging = smem + (size_t)p.stages * stage_bytes;
+  uint64_t* bars = (uint64_t*)(staging + NUM_EPI_WARPS * STAGING_BYTES);
   uint64_t* full_bar = bars;
   uint64_t* empty_bar = bars + MAX_STAGES;
   uint64_t* tfull_bar = bars + 2 * MAX_STAGES;
@@ -187,7 +295,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; a++) {
       mbar_init(smem_u32(&tfull_bar[a]), 1);
-      mbar_init(smem_u32(&tempty_bar[a]), 4);
+      mbar_init(smem_u32(&tempty_bar[a]), NUM_EPI_WARPS);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -300,7 +408,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp >= 2) {
     // ------------------------------- epilogue -------------------------------
-    const int q = warp & 3;  // TMEM lane quarter this warp may read
+    // Two warps share each TMEM lane quarter and take alternate 32-column chunks.  A warp reads
+    // its 32 x 32 chunk (one row per lane), applies the epilogue, then turns the chunk through a
+    // swizzled staging buffer so that global stores cover whole row segments.
+    const int q = warp & 3;              // TMEM lane quarter this warp may read
+    const int hsel = (warp - 2) >> 2;    // which of the two warps of the quarter
+    uint8_t* stg = staging + (size_t)(warp - 2) * STAGING_BYTES;
     uint32_t tile = 0;
     bool ok = true;
     for (int w = blockIdx.x; w < p.total_work && ok; w += gridDim.x, tile++) {
@@ -313,120 +426,74 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t acc = tile & 1, use = tile >> 1;
       if (!mbar_wait(smem_u32(&tfull_bar[acc]), use & 1, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      const int m = mt * BM + q * 32 + lane;
-      const long long off0 = zo * p.d_bo + zi * p.d_bi + (long long)m * p.ldd;
+      const int m_warp = mt * BM + q * 32;  // first row of this warp
+      const int m = m_warp + lane;
+      const long long zoff = zo * p.d_bo + zi * p.d_bi;
+      const long long off0 = zoff + (long long)m * p.ldd;
       const int n_base = nt * p.bn;
-      for (int cidx = 0; cidx < p.bn / 32; cidx++) {
+      for (int cidx = hsel; cidx < p.bn / 32; cidx += 2) {
         const int n0 = n_base + cidx * 32;
         if (n0 >= p.N) break;  // uniform over the warp
         float v[32];
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256 + cidx * 32, v);
-        if (m < p.M) {
-          const long long off = off0 + n0;
-          const bool fullv = p.vec_ok && (n0 + 32 <= p.N);
+        const long long off = off0 + n0;
+        const bool fullv = p.vec_ok && (n0 + 32 <= p.N);
+        const bool row_ok = m < p.M;
 #pragma unroll
-          for (int j = 0; j < 32; j++) v[j] *= p.alpha;
-          if (p.bias) {
-            if (n0 + 32 <= p.N) {
+        for (int j = 0; j < 32; j++) v[j] *= p.alpha;
+        if (p.bias) {
+          if (n0 + 32 <= p.N) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 4) {
-                const float4 b4 = *reinterpret_cast<const float4*>(p.bias + n0 + j);
-                v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; j++)
-                if (n0 + j < p.N) v[j] += p.bias[n0 + j];
-            }
-          }
-          if (p.act == 1) {
-            if (p.aux) {
-              if (fullv) {
-#pragma unroll
-                for (int j = 0; j < 32; j += 8) {
-                  float t[8];
-#pragma unroll
-                  for (int e = 0; e < 8; e++) t[e] = v[j + e];
-                  VecT<bf16>::store(p.aux + off + j, t);
-                }
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; j++)
-                  if (n0 + j < p.N) p.aux[off + j] = __float2bfloat16_rn(v[j]);
-              }
-            }
-#pragma unroll
-            for (int j = 0; j < 32; j++) v[j] = gelu_f(v[j]);
-          } else if (p.act == 2) {
-            if (fullv) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                float t[8];
-                VecT<bf16>::load(p.aux + off + j, t);
-#pragma unroll
-                for (int e = 0; e < 8; e++) v[j + e] *= gelu_grad_f(t[e]);
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; j++)
-                if (n0 + j < p.N) v[j] *= gelu_grad_f(__bfloat162float(p.aux[off + j]));
-            }
-          }
-          if (p.residual) {
-            if (fullv) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                float t[8];
-                VecT<bf16>::load(p.residual + off + j, t);
-#pragma unroll
-                for (int e = 0; e < 8; e++) v[j + e] += t[e];
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; j++)
-                if (n0 + j < p.N) v[j] += __bfloat162float(p.residual[off + j]);
-            }
-          }
-          if (p.d_fp32) {
-            float* dp = reinterpret_cast<float*>(p.D) + off;
-            if (p.accumulate) {
-              if (fullv) {
-#pragma unroll
-                for (int j = 0; j < 32; j += 4)
-                  asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dp + j), "f"(v[j]),
-                               "f"(v[j + 1]), "f"(v[j + 2]), "f"(v[j + 3])
-                               : "memory");
-              } else {
-#pragma unroll
-                for (int j = 0; j < 32; j++)
-                  if (n0 + j < p.N) atomicAdd(dp + j, v[j]);
-              }
-            } else if (fullv) {
-#pragma unroll
-              for (int j = 0; j < 32; j += 4)
-                *reinterpret_cast<float4*>(dp + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; j++)
-                if (n0 + j < p.N) dp[j] = v[j];
+            for (int j = 0; j < 32; j += 4) {
+              const float4 b4 = *reinterpret_cast<const float4*>(p.bias + n0 + j);
+              v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
             }
           } else {
-            bf16* dp = reinterpret_cast<bf16*>(p.D) + off;
-            if (fullv) {
 #pragma unroll
-              for (int j = 0; j < 32; j += 8) {
-                float t[8];
-#pragma unroll
-                for (int e = 0; e < 8; e++) t[e] = v[j + e];
-                VecT<bf16>::store(dp + j, t);
-              }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 32; j++)
-                if (n0 + j < p.N) dp[j] = __float2bfloat16_rn(v[j]);
-            }
+            for (int j = 0; j < 32; j++)
+              if (n0 + j < p.N) v[j] += p.bias[n0 + j];
           }
         }
+        if (p.act == 1) {
+          if (p.aux) stage_store_bf16(stg, lane, v, p.aux + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
+#pragma unroll
+          for (int j = 0; j < 32; j++) v[j] = gelu_fast(v[j]);
+        } else if (p.act == 2 && row_ok) {
+          if (fullv) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              float t[8];
+              VecT<bf16>::load(p.aux + off + j, t);
+#pragma unroll
+              for (int e = 0; e < 8; e++) v[j + e] *= gelu_grad_fast(t[e]);
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j++)
+              if (n0 + j < p.N) v[j] *= gelu_grad_fast(__bfloat162float(p.aux[off + j]));
+          }
+        }
+        if (p.residual && row_ok) {
+          if (fullv) {
+#pragma unroll
+            for (int j = 0; j < 32; j += 8) {
+              float t[8];
+              VecT<bf16>::load(p.residual + off + j, t);
+#pragma unroll
+              for (int e = 0; e < 8; e++) v[j + e] += t[e];
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; j++)
+              if (n0 + j < p.N) v[j] += __bfloat162float(p.residual[off + j]);
+          }
+        }
+        if (p.d_fp32)
+          stage_store_f32(stg, lane, v, reinterpret_cast<float*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N,
+                          p.vec_ok, p.accumulate);
+        else
+          stage_store_bf16(stg, lane, v, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N,
+                           p.vec_ok);
       }
       // hand the accumulator back to the MMA warp
       tc_fence_before();
@@ -593,7 +660,7 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   int stages = (196 * 1024) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   p.stages = stages;
-  const size_t smem_bytes = (size_t)stages * stage_bytes + 1024 + 256;
+  const size_t smem_bytes = (size_t)stages * stage_bytes + NUM_EPI_WARPS * STAGING_BYTES + 1024 + 256;
   if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "gemm: not enough shared memory"); return MSLT_ERR_CUDA; }
 
   MapVal ma, mb;
