@@ -205,6 +205,9 @@ typedef struct {
  * zeroed by the caller, that receives a non-zero code if a kernel wait ran out (then the
  * call returns MSLT_ERR_DEVICE). */
 int mslt_op_gemm(const mslt_gemm_desc* desc, void* cuda_stream, int32_t* d_status);
+/* The same contraction, only enqueued: no synchronisation and no read of the status word, which
+ * the caller inspects after synchronising the stream itself. */
+int mslt_op_gemm_enqueue(const mslt_gemm_desc* desc, void* cuda_stream, int32_t* d_status);
 
 #ifdef __cplusplus
 }

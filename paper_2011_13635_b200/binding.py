@@ -53,7 +53,7 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_set_param", "mslt_get_param_raw", "mslt_get_grad", "mslt_get_opt_state",
            "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_gemm_profile",
            "mslt_last_error",
-           "mslt_op_gemm"]
+           "mslt_op_gemm", "mslt_op_gemm_enqueue"]
 
 lib.mslt_last_error.restype = C.c_char_p
 lib.mslt_last_error.argtypes = [C.c_void_p]
@@ -85,6 +85,7 @@ lib.mslt_set_timing.argtypes = [C.c_void_p, C.c_int32]
 lib.mslt_get_timings.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
 lib.mslt_get_gemm_profile.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
 lib.mslt_op_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
+lib.mslt_op_gemm_enqueue.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
 
 
 class MsltError(RuntimeError):
@@ -110,6 +111,10 @@ def mslt_query_bytes(arch: Arch):
 
 def mslt_op_gemm(desc: GemmDesc, stream: int, status) -> None:
     _check(lib.mslt_op_gemm(C.byref(desc), C.c_void_p(stream), C.c_void_p(_ptr(status))))
+
+
+def mslt_op_gemm_enqueue(desc: GemmDesc, stream: int, status) -> None:
+    _check(lib.mslt_op_gemm_enqueue(C.byref(desc), C.c_void_p(stream), C.c_void_p(_ptr(status))))
 
 
 class Mslt:

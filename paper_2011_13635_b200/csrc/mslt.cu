@@ -878,7 +878,7 @@ int mslt_get_timings(mslt_ctx* c, float* ms, int32_t n) {
   return 0;
 }
 
-int mslt_op_gemm(const mslt_gemm_desc* d, void* cuda_stream, int32_t* d_status) {
+static int check_gemm_desc(const mslt_gemm_desc* d) {
   if (!d || !d->A || !d->B || !d->D) return fail(MSLT_ERR_ARG, "null pointer");
   if (d->M < 1 || d->N < 1 || d->K < 1 || d->batch < 1 || d->hdiv < 1)
     return fail(MSLT_ERR_ARG, "bad GEMM shape");
@@ -889,11 +889,21 @@ int mslt_op_gemm(const mslt_gemm_desc* d, void* cuda_stream, int32_t* d_status) 
   int ndev = 0;
   if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0)
     return fail(MSLT_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  return 0;
+}
+
+int mslt_op_gemm_enqueue(const mslt_gemm_desc* d, void* cuda_stream, int32_t* d_status) {
+  TRY(check_gemm_desc(d));
   char err[256] = "";
-  cudaStream_t st = (cudaStream_t)cuda_stream;
-  int rc = gemm_launch(*d, d_status, st, err);
+  int rc = gemm_launch(*d, d_status, (cudaStream_t)cuda_stream, err);
   if (rc) return fail(rc, "%s", err);
   CUDA_TRY(cudaGetLastError());
+  return 0;
+}
+
+int mslt_op_gemm(const mslt_gemm_desc* d, void* cuda_stream, int32_t* d_status) {
+  TRY(mslt_op_gemm_enqueue(d, cuda_stream, d_status));
+  cudaStream_t st = (cudaStream_t)cuda_stream;
   CUDA_TRY(cudaStreamSynchronize(st));
   if (d_status) {
     int h = 0;
