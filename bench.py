@@ -251,16 +251,16 @@ def run_ours(args, cfg):
         peaks = measured_peaks()
         # per-kernel pass: the same steps again with an event pair around every contraction
         m.mslt_set_timing(2)
-        m.mslt_get_gemm_profile()
+        m.mslt_get_kernel_profile()
         n_prof = max(1, min(args.steps, 5))
         for _ in range(n_prof):
             m.mslt_step(*dev, sync=False)
         torch.cuda.synchronize()
-        prof = m.mslt_get_gemm_profile()
+        prof = m.mslt_get_kernel_profile()
         phases = m.mslt_get_timings()
         m.mslt_set_timing(0)
         lin, att = prof["linear"], prof["attention"]
-        lin_tflops = lin["flops"] / (lin["ms"] * 1e-3) / 1e12 if lin["ms"] > 0 else 0.0
+        lin_tflops = lin["work"] / (lin["ms"] * 1e-3) / 1e12 if lin["ms"] > 0 else 0.0
         peak = peaks["bf16_tflops_sustained"] if cfg.dtype == "bf16" else None
         if cfg.dtype == "bf16":
             line["roofline"] = dict(
@@ -269,15 +269,19 @@ def run_ours(args, cfg):
                 peak_source=f"{peaks['source']}: cuBLAS bf16 sustained (kernel timed inside a long step)",
                 launches_per_step=lin["launches"] / n_prof,
                 avg_launch_us=1e3 * lin["ms"] / max(lin["launches"], 1),
-                flops_per_step=lin["flops"] / n_prof,
+                flops_per_step=lin["work"] / n_prof,
                 share_of_step_time=lin["ms"] / n_prof / (ms / args.steps))
         else:
             line["roofline"] = dict(bound="alu", kernel="gemm_simt_kernel", achieved=lin_tflops, peak=None,
                                     unit="TFLOP/s", frac=None, traffic=None)
         line["attention_gemms"] = dict(
-            tflops=att["flops"] / (att["ms"] * 1e-3) / 1e12 if att["ms"] > 0 else 0.0,
+            tflops=att["work"] / (att["ms"] * 1e-3) / 1e12 if att["ms"] > 0 else 0.0,
             ms_per_step=att["ms"] / n_prof, launches_per_step=att["launches"] / n_prof)
         line["phases_ms"] = phases
+        line["hbm_kernels"] = {
+            k: dict(gbs=v["work"] / (v["ms"] * 1e-3) / 1e9, frac_of_measured_copy=v["work"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    ms_per_step=v["ms"] / n_prof, launches_per_step=v["launches"] / n_prof)
+            for k, v in prof.items() if k not in ("linear", "attention") and v["ms"] > 0}
         line["step_tflops"] = step_flops(cfg) / (ms / args.steps * 1e-3) / 1e12
         m.close()
         del m

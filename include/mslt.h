@@ -163,11 +163,14 @@ int64_t mslt_launch_count(const mslt_ctx* ctx);
  * [4] Adam.  Turning timing on adds event records and one synchronisation per step. */
 int mslt_set_timing(mslt_ctx* ctx, int32_t on);
 int mslt_get_timings(mslt_ctx* ctx, float* host_ms, int32_t n);
-/* Timing level 2 (mslt_set_timing(ctx, 2)) also brackets every contraction of a step with an
- * event pair.  This call returns and clears what has been accumulated since the last call, as 6
- * host doubles: for the linear-layer products, then for the batched attention products:
- * launches, floating-point operations (2*M*N*K*batch), milliseconds. */
-int mslt_get_gemm_profile(mslt_ctx* ctx, double* host_out, int32_t n);
+/* Timing level 2 (mslt_set_timing(ctx, 2)) also brackets every kernel launch of a step with an
+ * event pair.  This call returns and clears what has been accumulated since the last call, as
+ * 10 x 3 host doubles: per kernel class {launches, work, milliseconds}, where work is
+ * floating-point operations (2*M*N*K*batch) for the two contraction classes and algorithmic
+ * bytes for the others.  Classes, in order: linear-layer products, batched attention products,
+ * LayerNorm forward (incl. embedding), LayerNorm backward, softmax forward, softmax backward,
+ * column sums, cross-entropy, Adam, other. */
+int mslt_get_kernel_profile(mslt_ctx* ctx, double* host_out, int32_t n);
 /* Message for the last error on this thread (ctx may be NULL). */
 const char* mslt_last_error(const mslt_ctx* ctx);
 
@@ -194,11 +197,15 @@ typedef struct {
   int32_t accumulate;       /* 1 (needs d_fp32): D += result (atomic adds; order not fixed) */
   float alpha;
   const float* bias;        /* [N] fp32 added after alpha, or NULL                          */
-  int32_t act;              /* 0 none; 1 GELU(erf); 2 multiply by GELU'(aux)                */
+  int32_t act;              /* 0 none; 1 GELU(erf); 2 multiply by GELU'(aux); 3 masked       */
+                            /* softmax over each row (dtype 1 only, N <= 128, bf16 output;    */
+                            /* bias, aux and residual are not applied)                        */
   void* aux;                /* D's layout and A/B dtype. act 1: receives the pre-activation */
                             /* (may be NULL); act 2: holds the pre-activation               */
   const void* residual;     /* D's layout, A/B dtype, added last; or NULL                   */
   int32_t split_k;          /* 0 = automatic; > 1 needs d_fp32 and accumulate               */
+  const int32_t* seq_lens;  /* act 3: device [batch / hdiv]; key n of batch z is valid iff    */
+                            /* n < seq_lens[z / hdiv]; NULL = all N                           */
 } mslt_gemm_desc;
 
 /* Runs one contraction on `cuda_stream` and synchronises it.  d_status: device int32 word,

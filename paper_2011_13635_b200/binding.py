@@ -44,14 +44,14 @@ class GemmDesc(C.Structure):
                 ("D", C.c_void_p), ("ldd", C.c_int64), ("d_bo", C.c_int64), ("d_bi", C.c_int64),
                 ("d_fp32", C.c_int32), ("accumulate", C.c_int32), ("alpha", C.c_float),
                 ("bias", C.c_void_p), ("act", C.c_int32), ("aux", C.c_void_p),
-                ("residual", C.c_void_p), ("split_k", C.c_int32)]
+                ("residual", C.c_void_p), ("split_k", C.c_int32), ("seq_lens", C.c_void_p)]
 
 
 EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers", "mslt_set_trainable",
            "mslt_set_optimizer", "mslt_step", "mslt_read_loss", "mslt_forward", "mslt_num_layers",
            "mslt_num_trainable", "mslt_num_tensors", "mslt_tensor_info", "mslt_get_param",
            "mslt_set_param", "mslt_get_param_raw", "mslt_get_grad", "mslt_get_opt_state",
-           "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_gemm_profile",
+           "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_kernel_profile",
            "mslt_last_error",
            "mslt_op_gemm", "mslt_op_gemm_enqueue"]
 
@@ -83,7 +83,7 @@ lib.mslt_get_grad.argtypes = [C.c_void_p, C.c_char_p, C.c_void_p, C.c_size_t]
 lib.mslt_get_opt_state.argtypes = [C.c_void_p, C.c_char_p, C.c_int32, C.c_void_p, C.c_size_t]
 lib.mslt_set_timing.argtypes = [C.c_void_p, C.c_int32]
 lib.mslt_get_timings.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
-lib.mslt_get_gemm_profile.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
+lib.mslt_get_kernel_profile.argtypes = [C.c_void_p, C.c_void_p, C.c_int32]
 lib.mslt_op_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
 lib.mslt_op_gemm_enqueue.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
 
@@ -263,11 +263,15 @@ class Mslt:
     def mslt_set_timing(self, level: int):
         _check(lib.mslt_set_timing(self.h, int(level)))
 
-    def mslt_get_gemm_profile(self) -> Dict[str, dict]:
-        buf = (C.c_double * 6)()
-        _check(lib.mslt_get_gemm_profile(self.h, buf, 6))
-        return {k: dict(launches=int(buf[3 * i]), flops=buf[3 * i + 1], ms=buf[3 * i + 2])
-                for i, k in enumerate(["linear", "attention"])}
+    PROFILE_CLASSES = ["linear", "attention", "ln_fwd", "ln_bwd", "softmax_fwd", "softmax_bwd", "colsum",
+                       "cross_entropy", "adam", "other"]
+
+    def mslt_get_kernel_profile(self) -> Dict[str, dict]:
+        """Per kernel class: launches, work (flops for the two GEMM classes, bytes otherwise), ms."""
+        buf = (C.c_double * 30)()
+        _check(lib.mslt_get_kernel_profile(self.h, buf, 30))
+        return {k: dict(launches=int(buf[3 * i]), work=buf[3 * i + 1], ms=buf[3 * i + 2])
+                for i, k in enumerate(self.PROFILE_CLASSES)}
 
     def mslt_get_timings(self) -> Dict[str, float]:
         buf = (C.c_float * 5)()

@@ -87,6 +87,10 @@ __global__ void __launch_bounds__(256) gemm_simt_kernel(mslt_gemm_desc d) {
 }
 
 int gemm_simt_launch(const mslt_gemm_desc& d, cudaStream_t st, char* err) {
+  if (d.act == 3) {
+    snprintf(err, 256, "gemm: the softmax epilogue exists only in the tensor-core kernel");
+    return MSLT_ERR_ARG;
+  }
   dim3 grid((d.N + 63) / 64, (d.M + 63) / 64, d.batch);
   if (grid.y > 65535 || grid.z > 65535) {
     snprintf(err, 256, "gemm: grid too large for the CUDA-core kernel");

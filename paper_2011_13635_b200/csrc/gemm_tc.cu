@@ -40,7 +40,7 @@ constexpr int NUM_EPI_WARPS = 8;
 constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 constexpr int STAGING_BYTES = 4096;  // per epilogue warp
 constexpr uint32_t TMEM_COLS = 512;
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;  // 2 s
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // about 2 s of SM clock
 
 struct TcParams {
   int M, N, K, batch, hdiv;
@@ -55,6 +55,7 @@ struct TcParams {
   int act;
   bf16* aux;
   const bf16* residual;
+  const int* seq_lens;  // act 3: valid keys per outer batch index, or null
   int* status;
   uint32_t idesc;
 };
@@ -63,11 +64,8 @@ struct TcParams {
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ unsigned long long globaltimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
+// SM cycle counter: cheap to read, which matters because every bounded wait samples it
+__device__ __forceinline__ long long now_cycles() { return clock64(); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -92,13 +90,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
                                           int* status) {
   if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = globaltimer();
+  const long long t0 = now_cycles();
   uint32_t spins = 0;
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (globaltimer() - t0 > WAIT_LIMIT_NS) {
+      if (now_cycles() - t0 > WAIT_LIMIT_CYCLES) {
         *abort_flag = 1;
         atomicOr(status, ST_WAIT_TIMEOUT);
         return false;
@@ -270,7 +268,37 @@ __device__ __forceinline__ void stage_store_f32(uint8_t* stg, int lane, const fl
   __syncwarp();
 }
 
+// Hand-over between the two epilogue warps of a TMEM lane quarter: publish my sequence number
+// after my shared-memory writes, then wait (bounded) until the partner has published the same.
+__device__ __forceinline__ bool pair_sync(volatile int* flags, int me, int other, int seq, int lane,
+                                          volatile int* abort_flag, int* status) {
+  __syncwarp();
+  int ok = 1;
+  if (lane == 0) {
+    __threadfence_block();
+    flags[me] = seq;
+    const long long t0 = now_cycles();
+    uint32_t spins = 0;
+    while (flags[other] < seq) {
+      if ((++spins & 255u) == 0u) {
+        if (*abort_flag) { ok = 0; break; }
+        if (now_cycles() - t0 > WAIT_LIMIT_CYCLES) {
+          *abort_flag = 1;
+          atomicOr(status, ST_WAIT_TIMEOUT);
+          ok = 0;
+          break;
+        }
+      }
+    }
+    __threadfence_block();
+  }
+  ok = __shfl_sync(0xffffffffu, ok, 0);
+  return ok != 0;
+}
+
 // ---- the kernel ---------------------------------------------------------------------------------
+// 10 warps are allocated registers as 12, which caps a thread at 168 registers
+template <bool kSoftmax>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const TcParams p) {
@@ -287,6 +315,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   uint64_t* tempty_bar = bars + 2 * MAX_STAGES + 2;
   uint32_t* tmem_slot = (uint32_t*)(bars + 2 * MAX_STAGES + 4);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+  // softmax epilogue only: hand-over flags and per-row partial results of the two warps of a quarter
+  volatile int* xflag = (volatile int*)((uint8_t*)bars + 256);
+  float* xmax = (float*)((uint8_t*)bars + 256 + 64);
+  float* xsum = xmax + NUM_EPI_WARPS * 32;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
@@ -300,6 +332,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&tempty_bar[a]), NUM_EPI_WARPS);
     }
     *abort_flag = 0;
+    if (kSoftmax)
+      for (int i = 0; i < NUM_EPI_WARPS; i++) xflag[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -366,8 +400,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (uint32_t i = 0; i < n; i++) {
         const uint32_t j = it - 1 - i;
         const uint32_t fb = smem_u32(&full_bar[j % p.stages]);
-        const unsigned long long t0 = globaltimer();
-        while (!mbar_try_wait(fb, (j / p.stages) & 1) && globaltimer() - t0 < 100000000ull) {}
+        const long long t0 = now_cycles();
+        while (!mbar_try_wait(fb, (j / p.stages) & 1) && now_cycles() - t0 < 200000000ll) {}
       }
     }
   } else if (warp == 1 && lane == 0) {
@@ -405,8 +439,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (!ok || *abort_flag) {
       // make sure no MMA is still writing tensor memory before it is freed
       tc_commit(smem_u32(&tfull_bar[0]));
-      const unsigned long long t0 = globaltimer();
-      while (globaltimer() - t0 < 1000000ull) {}
+      const long long t0 = now_cycles();
+      while (now_cycles() - t0 < 2000000ll) {}
     }
   } else if (warp >= 2) {
     // ------------------------------- epilogue -------------------------------
@@ -433,6 +467,69 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const long long zoff = zo * p.d_bo + zi * p.d_bi;
       const long long off0 = zoff + (long long)m * p.ldd;
       const int n_base = nt * p.bn;
+      if constexpr (kSoftmax) {
+        // Scaled masked softmax over whole rows (one n-tile of at most 128 columns holds a row).
+        // Each warp keeps its (up to) two 32-column chunks in registers; the two warps of a
+        // quarter exchange row maxima and row sums through shared memory.
+        int len = p.seq_lens ? p.seq_lens[zo] : p.N;
+        len = min(max(len, 1), p.N);
+        const int c0 = hsel, c1 = hsel + 2;
+        const bool h0 = c0 * 32 < p.N && c0 < p.bn / 32, h1 = c1 * 32 < p.N && c1 < p.bn / 32;
+        float v0[32], v1[32];
+        float mx = -INFINITY;
+        const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
+        if (h0) {
+          tc_ld32(trow + c0 * 32, v0);
+#pragma unroll
+          for (int j = 0; j < 32; j++) {
+            v0[j] = (c0 * 32 + j < len) ? v0[j] * p.alpha : -INFINITY;
+            mx = fmaxf(mx, v0[j]);
+          }
+        }
+        if (h1) {
+          tc_ld32(trow + c1 * 32, v1);
+#pragma unroll
+          for (int j = 0; j < 32; j++) {
+            v1[j] = (c1 * 32 + j < len) ? v1[j] * p.alpha : -INFINITY;
+            mx = fmaxf(mx, v1[j]);
+          }
+        }
+        // the accumulator is in registers now: hand it back before the slow part
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+        const int seq = (int)tile * 2 + 1;
+        const int me = q * 2 + hsel, other = q * 2 + (hsel ^ 1);
+        xmax[me * 32 + lane] = mx;
+        if (!pair_sync(xflag, me, other, seq, lane, abort_flag, p.status)) { ok = false; break; }
+        mx = fmaxf(mx, xmax[other * 32 + lane]);
+        float sum = 0.f;
+        if (h0) {
+#pragma unroll
+          for (int j = 0; j < 32; j++) { v0[j] = __expf(v0[j] - mx); sum += v0[j]; }
+        }
+        if (h1) {
+#pragma unroll
+          for (int j = 0; j < 32; j++) { v1[j] = __expf(v1[j] - mx); sum += v1[j]; }
+        }
+        xsum[me * 32 + lane] = sum;
+        if (!pair_sync(xflag, me, other, seq + 1, lane, abort_flag, p.status)) { ok = false; break; }
+        sum += xsum[other * 32 + lane];
+        const float inv = 1.0f / sum;
+        if (h0) {
+#pragma unroll
+          for (int j = 0; j < 32; j++) v0[j] *= inv;
+          stage_store_bf16(stg, lane, v0, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, c0 * 32, p.M, p.N,
+                           p.vec_ok);
+        }
+        if (h1) {
+#pragma unroll
+          for (int j = 0; j < 32; j++) v1[j] *= inv;
+          stage_store_bf16(stg, lane, v1, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, c1 * 32, p.M, p.N,
+                           p.vec_ok);
+        }
+        continue;
+      } else {
       for (int cidx = hsel; cidx < p.bn / 32; cidx += 2) {
         const int n0 = n_base + cidx * 32;
         if (n0 >= p.N) break;  // uniform over the warp
@@ -501,6 +598,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+      }
     }
   }
 
@@ -658,11 +756,17 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   const long long total = tiles * p.splits;
   if (total > 0x7fffffffll) { snprintf(err, 256, "gemm: too many tiles"); return MSLT_ERR_SIZE; }
   p.total_work = (int)total;
+  if (d.act == 3 && (d.N > 128 || d.d_fp32 || splits != 1)) {
+    snprintf(err, 256, "gemm: the softmax epilogue needs bf16 output rows of at most 128 columns");
+    return MSLT_ERR_ARG;
+  }
   const int stage_bytes = A_STAGE_BYTES + p.bn * BK * 2;
-  int stages = (196 * 1024) / stage_bytes;
+  const int book_bytes = 256 + (d.act == 3 ? 64 + 2 * NUM_EPI_WARPS * 32 * 4 : 0);
+  int stages = (smem_optin - NUM_EPI_WARPS * STAGING_BYTES - 1024 - book_bytes) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
+  if (stages < 2) { snprintf(err, 256, "gemm: not enough shared memory"); return MSLT_ERR_CUDA; }
   p.stages = stages;
-  const size_t smem_bytes = (size_t)stages * stage_bytes + NUM_EPI_WARPS * STAGING_BYTES + 1024 + 256;
+  const size_t smem_bytes = (size_t)stages * stage_bytes + NUM_EPI_WARPS * STAGING_BYTES + 1024 + book_bytes;
   if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "gemm: not enough shared memory"); return MSLT_ERR_CUDA; }
 
   MapVal ma, mb;
@@ -677,6 +781,7 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   p.D = (char*)d.D; p.ldd = d.ldd; p.d_bo = d.d_bo; p.d_bi = d.d_bi;
   p.d_fp32 = d.d_fp32; p.accumulate = d.accumulate; p.alpha = d.alpha; p.bias = d.bias; p.act = d.act;
   p.aux = (bf16*)d.aux; p.residual = (const bf16*)d.residual; p.status = status;
+  p.seq_lens = d.seq_lens;
   // 16-byte vector access in the epilogue needs every row segment to start on a 16-byte boundary
   // in each of the buffers it touches (bf16 ones are the stricter case: 8 elements)
   auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
@@ -688,12 +793,17 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
 
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
     if (e != cudaSuccess) { snprintf(err, 256, "gemm: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
     attr_set = true;
   }
   const int grid = p.total_work < num_sms ? p.total_work : num_sms;
-  gemm_tc_kernel<<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
+  if (d.act == 3)
+    gemm_tc_kernel<true><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
+  else
+    gemm_tc_kernel<false><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { snprintf(err, 256, "gemm: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
   return 0;

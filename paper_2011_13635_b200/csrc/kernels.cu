@@ -55,10 +55,16 @@ __device__ __forceinline__ void ln_finish_row(float (&x)[LN_MAXE], int lane, int
   for (int i = 0; i < NV; i++) {
     const int c = (lane + 32 * i) * VN;
     if (c < H) {
-      float o[VN];
+      float o[VN], g[VN], b[VN];
 #pragma unroll
-      for (int e = 0; e < VN; e++)
-        o[e] = gamma[c + e] * ((x[i * VN + e] - mean) * rstd) + beta[c + e];
+      for (int e = 0; e < VN; e += 4) {  // 16-byte loads: scalar ones flood L1 with strided sectors
+        const float4 g4 = *reinterpret_cast<const float4*>(gamma + c + e);
+        const float4 b4 = *reinterpret_cast<const float4*>(beta + c + e);
+        g[e] = g4.x; g[e + 1] = g4.y; g[e + 2] = g4.z; g[e + 3] = g4.w;
+        b[e] = b4.x; b[e + 1] = b4.y; b[e + 2] = b4.z; b[e + 3] = b4.w;
+      }
+#pragma unroll
+      for (int e = 0; e < VN; e++) o[e] = g[e] * ((x[i * VN + e] - mean) * rstd) + b[e];
       VecT<T>::store(yrow + c, o);
     }
   }
@@ -135,45 +141,56 @@ embed_ln_kernel(const int* __restrict__ tokens, const T* __restrict__ word,
 // LayerNorm backward: dz = rstd * (dxhat - mean(dxhat) - xhat * mean(dxhat * xhat)),
 // dgamma += sum_rows dy * xhat, dbeta += sum_rows dy (fp32 atomics, one per column per block).
 // ---------------------------------------------------------------------------------------
-template <typename T>
-__global__ void __launch_bounds__(256)
+template <typename T, int MAXE>
+__global__ void __launch_bounds__(128)
 ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z, const float* __restrict__ stats,
               const float* __restrict__ gamma, T* __restrict__ dz, float* __restrict__ dgamma,
               float* __restrict__ dbeta, int rows, int H) {
   constexpr int VN = VecT<T>::N;
-  constexpr int NV = LN_MAXE / VN;
-  __shared__ float red[8][LN_MAXE * 32];
+  constexpr int NV = MAXE / VN;
+  constexpr int NW = 4;  // warps per block
+  __shared__ float red[NW][MAXE * 32];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int gw = blockIdx.x * 8 + warp, nw = gridDim.x * 8;
-  float ag[LN_MAXE], ab[LN_MAXE], g[LN_MAXE];
+  const int gw = blockIdx.x * NW + warp, nw = gridDim.x * NW;
+  float ag[MAXE], ab[MAXE], g[MAXE];
 #pragma unroll
-  for (int i = 0; i < LN_MAXE; i++) { ag[i] = 0.f; ab[i] = 0.f; g[i] = 0.f; }
+  for (int i = 0; i < MAXE; i++) { ag[i] = 0.f; ab[i] = 0.f; g[i] = 0.f; }
 #pragma unroll
   for (int i = 0; i < NV; i++) {
     const int c = (lane + 32 * i) * VN;
     if (c < H) {
 #pragma unroll
-      for (int e = 0; e < VN; e++) g[i * VN + e] = gamma[c + e];
+      for (int e = 0; e < VN; e += 4) {
+        const float4 g4 = *reinterpret_cast<const float4*>(gamma + c + e);
+        g[i * VN + e] = g4.x; g[i * VN + e + 1] = g4.y; g[i * VN + e + 2] = g4.z; g[i * VN + e + 3] = g4.w;
+      }
     }
   }
   const float invH = 1.0f / (float)H;
   for (int row = gw; row < rows; row += nw) {
     const float mean = stats[2 * (int64_t)row], rstd = stats[2 * (int64_t)row + 1];
-    float dyv[LN_MAXE], xh[LN_MAXE];
+    // the row stays packed in registers between the two passes (fewer registers, more warps)
+    typename VecT<T>::Raw ra[NV], rb[NV];
     float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int i = 0; i < NV; i++) {
       const int c = (lane + 32 * i) * VN;
       if (c < H) {
+        ra[i] = VecT<T>::load_raw(dy + (int64_t)row * H + c);
+        rb[i] = VecT<T>::load_raw(z + (int64_t)row * H + c);
+      }
+    }
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (lane + 32 * i) * VN;
+      if (c < H) {
         float a[VN], b[VN];
-        VecT<T>::load(dy + (int64_t)row * H + c, a);
-        VecT<T>::load(z + (int64_t)row * H + c, b);
+        VecT<T>::unpack(ra[i], a);
+        VecT<T>::unpack(rb[i], b);
 #pragma unroll
         for (int e = 0; e < VN; e++) {
           const float xhat = (b[e] - mean) * rstd;
           const float dxh = a[e] * g[i * VN + e];
-          dyv[i * VN + e] = dxh;
-          xh[i * VN + e] = xhat;
           s1 += dxh;
           s2 += dxh * xhat;
           ag[i * VN + e] += a[e] * xhat;
@@ -187,10 +204,14 @@ ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z, const float* __
     for (int i = 0; i < NV; i++) {
       const int c = (lane + 32 * i) * VN;
       if (c < H) {
-        float o[VN];
+        float a[VN], b[VN], o[VN];
+        VecT<T>::unpack(ra[i], a);
+        VecT<T>::unpack(rb[i], b);
 #pragma unroll
-        for (int e = 0; e < VN; e++)
-          o[e] = rstd * (dyv[i * VN + e] - s1 - xh[i * VN + e] * s2);
+        for (int e = 0; e < VN; e++) {
+          const float xhat = (b[e] - mean) * rstd;
+          o[e] = rstd * (a[e] * g[i * VN + e] - s1 - xhat * s2);
+        }
         VecT<T>::store(dz + (int64_t)row * H + c, o);
       }
     }
@@ -208,10 +229,10 @@ ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z, const float* __
     }
     __syncthreads();
     float* dst = pass == 0 ? dgamma : dbeta;
-    for (int c = threadIdx.x; c < H; c += 256) {
+    for (int c = threadIdx.x; c < H; c += 128) {
       float s = 0.f;
 #pragma unroll
-      for (int w = 0; w < 8; w++) s += red[w][c];
+      for (int w = 0; w < NW; w++) s += red[w][c];
       atomicAdd(dst + c, s);
     }
   }
@@ -639,9 +660,18 @@ void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* p
 void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, const float* gamma,
                    void* dz, float* dgamma, float* dbeta, int rows, int H, cudaStream_t st) {
   if (rows <= 0) return;
-  int blocks = std::min(div_up(rows, 8), 148 * 4);
-  DISPATCH_T(bf, (ln_bwd_kernel<T><<<blocks, 256, 0, st>>>((const T*)dy, (const T*)z, stats, gamma,
-                                                           (T*)dz, dgamma, dbeta, rows, H)));
+  // elements a lane holds: the smallest of 8 / 16 / 24 / 32 that covers the row keeps registers low
+  const int vn = bf ? 8 : 4;
+  const int need = (H + 32 * vn - 1) / (32 * vn) * vn;
+  const int blocks = std::min(div_up(rows, 4 * 2), 148 * 8);
+#define LN_BWD(E)                                                                                      \
+  DISPATCH_T(bf, (ln_bwd_kernel<T, E><<<blocks, 128, 0, st>>>((const T*)dy, (const T*)z, stats, gamma, \
+                                                              (T*)dz, dgamma, dbeta, rows, H)))
+  if (need <= 8) LN_BWD(8);
+  else if (need <= 16) LN_BWD(16);
+  else if (need <= 24) LN_BWD(24);
+  else LN_BWD(32);
+#undef LN_BWD
 }
 
 void launch_softmax_fwd(bool bf, const void* sc, void* p, const int* seq_lens, int rows, int S,

@@ -6,6 +6,7 @@
 #include <math.h>
 #include <stdarg.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <algorithm>
@@ -102,7 +103,7 @@ struct mslt_ctx {
   std::vector<cudaEvent_t> pev;
   struct PRec { int cls; double flops; };
   std::vector<PRec> prec;
-  double prof[2][3];  // per class (0 linear, 1 batched attention): launches, flops, ms
+  double prof[10][3];  // per kernel class: launches, work (flops or bytes), ms
 };
 
 namespace {
@@ -277,6 +278,12 @@ struct Lin {  // a plain 2-D contraction
   }
 };
 
+// true when bf16 products are routed to the CUDA-core kernel for debugging (see gemm.cu)
+bool getenv_cuda_cores() {
+  static const bool v = getenv("MSLT_BF16_CUDA_CORES") && atoi(getenv("MSLT_BF16_CUDA_CORES")) == 1;
+  return v;
+}
+
 int run_gemm(mslt_ctx* c, const mslt_gemm_desc& d) {
   if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) return 0;
   char err[256] = "";
@@ -334,10 +341,28 @@ int linear_wgrad(mslt_ctx* c, const void* dy, int T, int N, int64_t lddy, const 
     int rc_ = (x);    \
     if (rc_) return rc_; \
   } while (0)
-#define KL(x)       \
-  do {              \
-    x;              \
-    c->launches++;  \
+// kernel classes of the per-launch profile (timing level 2)
+enum { PC_LINEAR = 0, PC_ATTN_GEMM, PC_LN_FWD, PC_LN_BWD, PC_SOFTMAX_FWD, PC_SOFTMAX_BWD, PC_COLSUM,
+       PC_CROSS_ENTROPY, PC_ADAM, PC_OTHER, PC_COUNT };
+
+void prof_begin(mslt_ctx* c) {
+  if (c->profile && c->prec.size() * 2 + 2 <= c->pev.size())
+    cudaEventRecord(c->pev[2 * c->prec.size()], c->st);
+}
+void prof_end(mslt_ctx* c, int cls, double work) {
+  if (c->profile && c->prec.size() * 2 + 2 <= c->pev.size()) {
+    cudaEventRecord(c->pev[2 * c->prec.size() + 1], c->st);
+    c->prec.push_back({cls, work});
+  }
+}
+
+// launches one kernel; `work` is its algorithmic byte count (for the profile)
+#define KL(cls, work, x)          \
+  do {                            \
+    prof_begin(c);                \
+    x;                            \
+    c->launches++;                \
+    prof_end(c, cls, (double)(work)); \
   } while (0)
 
 // ---- one encoder layer, forward ------------------------------------------------------------------
@@ -354,9 +379,15 @@ int layer_forward(mslt_ctx* c, int l, const void* x, LayerBuf& b, void* out, boo
     g.d.A = b.qkv; g.d.a_rs = 3 * H; g.d.a_ks = 1; g.d.a_bo = (int64_t)S * 3 * H; g.d.a_bi = d;
     g.d.B = b.qkv + (int64_t)H * E; g.d.b_rs = 3 * H; g.d.b_ks = 1; g.d.b_bo = (int64_t)S * 3 * H; g.d.b_bi = d;
     g.d.D = b.p; g.d.ldd = S; g.d.d_bo = (int64_t)A * S * S; g.d.d_bi = (int64_t)S * S;
+    // rows of at most 128 keys fit one tile: the tensor-core kernel applies the masked softmax
+    // in its epilogue and writes probabilities straight away
+    const bool fused = c->bf && S <= 128 && !getenv_cuda_cores();
+    if (fused) { g.d.act = 3; g.d.seq_lens = seq_lens; }
     TRY(run_gemm(c, g.d));
+    if (!fused)
+      KL(PC_SOFTMAX_FWD, 2.0 * B * A * S * S * c->esz,
+         launch_softmax_fwd(c->bf, b.p, b.p, seq_lens, B * A * S, S, A * S, 1.0f, c->st));
   }
-  KL(launch_softmax_fwd(c->bf, b.p, b.p, seq_lens, B * A * S, S, A * S, 1.0f, c->st));
   {  // context[b,i,h,:] = sum_j p[b,h,i,j] v_j
     Lin g(c, S, d, S);
     g.d.batch = B * A; g.d.hdiv = A;
@@ -366,12 +397,12 @@ int layer_forward(mslt_ctx* c, int l, const void* x, LayerBuf& b, void* out, boo
     TRY(run_gemm(c, g.d));
   }
   TRY(linear_fwd(c, b.c, T, H, toff(c, l, "out.weight"), toff(c, l, "out.bias"), H, b.z1, 0, nullptr, x));
-  KL(launch_ln_fwd(c->bf, b.z1, Wv(c, toff(c, l, "ln1.gamma")), Wv(c, toff(c, l, "ln1.beta")), b.y,
+  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_ln_fwd(c->bf, b.z1, Wv(c, toff(c, l, "ln1.gamma")), Wv(c, toff(c, l, "ln1.beta")), b.y,
                    save ? b.st1 : nullptr, T, H, c->a.ln_eps, c->st));
   TRY(linear_fwd(c, b.y, T, H, toff(c, l, "ffn1.weight"), toff(c, l, "ffn1.bias"), F, b.g, 1,
                  save ? b.u : nullptr, nullptr));
   TRY(linear_fwd(c, b.g, T, F, toff(c, l, "ffn2.weight"), toff(c, l, "ffn2.bias"), H, b.z2, 0, nullptr, b.y));
-  KL(launch_ln_fwd(c->bf, b.z2, Wv(c, toff(c, l, "ln2.gamma")), Wv(c, toff(c, l, "ln2.beta")), out,
+  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_ln_fwd(c->bf, b.z2, Wv(c, toff(c, l, "ln2.gamma")), Wv(c, toff(c, l, "ln2.beta")), out,
                    save ? b.st2 : nullptr, T, H, c->a.ln_eps, c->st));
   return 0;
 }
@@ -384,18 +415,18 @@ int layer_backward(mslt_ctx* c, int l, const void* x_in, LayerBuf& b, const void
   const int E = c->esz;
   Workspace& w = c->ws;
   const float scale = 1.0f / sqrtf((float)d);
-  KL(launch_ln_bwd(c->bf, dx, b.z2, b.st2, Wv(c, toff(c, l, "ln2.gamma")), w.dz2,
+  KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, dx, b.z2, b.st2, Wv(c, toff(c, l, "ln2.gamma")), w.dz2,
                    G(c, toff(c, l, "ln2.gamma")), G(c, toff(c, l, "ln2.beta")), T, H, c->st));
   TRY(linear_wgrad(c, w.dz2, T, H, H, b.g, F, toff(c, l, "ffn2.weight")));
-  KL(launch_colsum(c->bf, w.dz2, H, T, H, G(c, toff(c, l, "ffn2.bias")), c->st));
+  KL(PC_COLSUM, 1.0 * T * H * c->esz, launch_colsum(c->bf, w.dz2, H, T, H, G(c, toff(c, l, "ffn2.bias")), c->st));
   TRY(linear_dgrad(c, w.dz2, T, H, H, toff(c, l, "ffn2.weight"), F, w.dg, 2, b.u, nullptr));
   TRY(linear_wgrad(c, w.dg, T, F, F, b.y, H, toff(c, l, "ffn1.weight")));
-  KL(launch_colsum(c->bf, w.dg, F, T, F, G(c, toff(c, l, "ffn1.bias")), c->st));
+  KL(PC_COLSUM, 1.0 * T * F * c->esz, launch_colsum(c->bf, w.dg, F, T, F, G(c, toff(c, l, "ffn1.bias")), c->st));
   TRY(linear_dgrad(c, w.dg, T, F, F, toff(c, l, "ffn1.weight"), H, w.dy, 0, nullptr, w.dz2));
-  KL(launch_ln_bwd(c->bf, w.dy, b.z1, b.st1, Wv(c, toff(c, l, "ln1.gamma")), w.dz1,
+  KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, w.dy, b.z1, b.st1, Wv(c, toff(c, l, "ln1.gamma")), w.dz1,
                    G(c, toff(c, l, "ln1.gamma")), G(c, toff(c, l, "ln1.beta")), T, H, c->st));
   TRY(linear_wgrad(c, w.dz1, T, H, H, b.c, H, toff(c, l, "out.weight")));
-  KL(launch_colsum(c->bf, w.dz1, H, T, H, G(c, toff(c, l, "out.bias")), c->st));
+  KL(PC_COLSUM, 1.0 * T * H * c->esz, launch_colsum(c->bf, w.dz1, H, T, H, G(c, toff(c, l, "out.bias")), c->st));
   TRY(linear_dgrad(c, w.dz1, T, H, H, toff(c, l, "out.weight"), H, w.dc, 0, nullptr, nullptr));
   const int64_t qs = (int64_t)S * 3 * H, ps = (int64_t)A * S * S, cs = (int64_t)S * H;
   {  // dV[j,:] = sum_i p[i,j] dC[i,:]
@@ -414,7 +445,7 @@ int layer_backward(mslt_ctx* c, int l, const void* x_in, LayerBuf& b, const void
     g.d.D = w.dp; g.d.ldd = S; g.d.d_bo = ps; g.d.d_bi = (int64_t)S * S;
     TRY(run_gemm(c, g.d));
   }
-  KL(launch_softmax_bwd(c->bf, w.dp, b.p, B * A * S, S, scale, c->st));
+  KL(PC_SOFTMAX_BWD, 3.0 * B * A * S * S * c->esz, launch_softmax_bwd(c->bf, w.dp, b.p, B * A * S, S, scale, c->st));
   {  // dQ[i,:] = sum_j dS[i,j] k_j
     Lin g(c, S, d, S);
     g.d.batch = B * A; g.d.hdiv = A;
@@ -432,7 +463,7 @@ int layer_backward(mslt_ctx* c, int l, const void* x_in, LayerBuf& b, const void
     TRY(run_gemm(c, g.d));
   }
   TRY(linear_wgrad(c, w.dqkv, T, 3 * H, 3 * H, x_in, H, toff(c, l, "qkv.weight")));
-  KL(launch_colsum(c->bf, w.dqkv, 3 * H, T, 3 * H, G(c, toff(c, l, "qkv.bias")), c->st));
+  KL(PC_COLSUM, 3.0 * T * H * c->esz, launch_colsum(c->bf, w.dqkv, 3 * H, T, 3 * H, G(c, toff(c, l, "qkv.bias")), c->st));
   if (need_dx)  // the frozen boundary stops here: nothing below needs a gradient
     TRY(linear_dgrad(c, w.dqkv, T, 3 * H, 3 * H, toff(c, l, "qkv.weight"), H, dx_out, 0, nullptr, w.dz1));
   return 0;
@@ -441,10 +472,10 @@ int layer_backward(mslt_ctx* c, int l, const void* x_in, LayerBuf& b, const void
 int head_forward(mslt_ctx* c, const void* x, int R, bool save) {
   const int H = c->a.hidden, V = c->a.vocab;
   Workspace& w = c->ws;
-  KL(launch_gather_rows(c->bf, x, w.rowsrc, w.hm, R, H, c->st));
+  KL(PC_OTHER, 2.0 * R * H * c->esz, launch_gather_rows(c->bf, x, w.rowsrc, w.hm, R, H, c->st));
   TRY(linear_fwd(c, w.hm, R, H, toff(c, -1, "head.transform.weight"), toff(c, -1, "head.transform.bias"),
                  H, w.gt, 1, save ? w.ut : nullptr, nullptr));
-  KL(launch_ln_fwd(c->bf, w.gt, Wv(c, toff(c, -1, "head.ln.gamma")), Wv(c, toff(c, -1, "head.ln.beta")),
+  KL(PC_LN_FWD, 2.0 * R * H * c->esz, launch_ln_fwd(c->bf, w.gt, Wv(c, toff(c, -1, "head.ln.gamma")), Wv(c, toff(c, -1, "head.ln.beta")),
                    w.tm, save ? w.hst : nullptr, R, H, c->a.ln_eps, c->st));
   // tied decoder: logits = tm * E^T + bv, fp32, rows padded to Vp columns
   TRY(linear_fwd(c, w.tm, R, H, toff(c, -1, "emb.word"), toff(c, -1, "head.decoder.bias"), V, w.logits,
@@ -455,7 +486,7 @@ int head_forward(mslt_ctx* c, const void* x, int R, bool save) {
 int head_backward(mslt_ctx* c, int B, int S, int P, bool full) {
   const int H = c->a.hidden, V = c->a.vocab, R = B * P, Vp = c->Vp;
   Workspace& w = c->ws;
-  KL(launch_colsum(c->bf, w.dlogits, Vp, R, Vp, G(c, toff(c, -1, "head.decoder.bias")), c->st));
+  KL(PC_COLSUM, 1.0 * R * Vp * c->esz, launch_colsum(c->bf, w.dlogits, Vp, R, Vp, G(c, toff(c, -1, "head.decoder.bias")), c->st));
   {  // dTm = dlogits * E
     Lin g(c, R, H, V);
     g.d.A = w.dlogits; g.d.a_rs = Vp; g.d.a_ks = 1;
@@ -470,14 +501,14 @@ int head_backward(mslt_ctx* c, int B, int S, int P, bool full) {
     g.d.D = G(c, toff(c, -1, "emb.word")); g.d.ldd = H; g.d.d_fp32 = 1; g.d.accumulate = 1;
     TRY(run_gemm(c, g.d));
   }
-  KL(launch_ln_bwd(c->bf, w.dtm, w.gt, w.hst, Wv(c, toff(c, -1, "head.ln.gamma")), w.dgt,
+  KL(PC_LN_BWD, 3.0 * R * H * c->esz, launch_ln_bwd(c->bf, w.dtm, w.gt, w.hst, Wv(c, toff(c, -1, "head.ln.gamma")), w.dgt,
                    G(c, toff(c, -1, "head.ln.gamma")), G(c, toff(c, -1, "head.ln.beta")), R, H, c->st));
-  KL(launch_dgelu(c->bf, w.dgt, w.ut, (int64_t)R * H, c->st));
+  KL(PC_OTHER, 3.0 * R * H * c->esz, launch_dgelu(c->bf, w.dgt, w.ut, (int64_t)R * H, c->st));
   TRY(linear_wgrad(c, w.dgt, R, H, H, w.hm, H, toff(c, -1, "head.transform.weight")));
-  KL(launch_colsum(c->bf, w.dgt, H, R, H, G(c, toff(c, -1, "head.transform.bias")), c->st));
+  KL(PC_COLSUM, 1.0 * R * H * c->esz, launch_colsum(c->bf, w.dgt, H, R, H, G(c, toff(c, -1, "head.transform.bias")), c->st));
   TRY(linear_dgrad(c, w.dgt, R, H, H, toff(c, -1, "head.transform.weight"), H, w.dhm, 0, nullptr, nullptr));
   CUDA_TRY(cudaMemsetAsync(w.dxa, 0, (size_t)B * S * H * c->esz, c->st));
-  KL(launch_scatter_rows(c->bf, w.dhm, w.rowsrc, w.dxa, B, P, H, c->st));
+  KL(PC_OTHER, 2.0 * B * P * H * c->esz, launch_scatter_rows(c->bf, w.dhm, w.rowsrc, w.dxa, B, P, H, c->st));
   return 0;
 }
 
@@ -653,10 +684,10 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   CUDA_TRY(cudaMemsetAsync(w.scalars, 0, 16, c->st));
   c->prec.clear();
   mark(c, 0);
-  KL(launch_slots_prepare(d_pos, d_lab, d_seq_lens, B, S, P, V, w.rowsrc, w.rowlabel, w.scalars + 1,
+  KL(PC_OTHER, 16.0 * B * P, launch_slots_prepare(d_pos, d_lab, d_seq_lens, B, S, P, V, w.rowsrc, w.rowlabel, w.scalars + 1,
                           inv_n, status, c->st));
   // embeddings, then the frozen prefix: forward only, two buffers, nothing kept but the output
-  KL(launch_embed_ln(c->bf, d_tokens, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
+  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_embed_ln(c->bf, d_tokens, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
                      Wv(c, toff(c, -1, "emb.ln.gamma")), Wv(c, toff(c, -1, "emb.ln.beta")), w.xa,
                      full ? w.z0 : nullptr, full ? w.st0 : nullptr, T, S, H, V, c->a.ln_eps, status,
                      c->st));
@@ -674,8 +705,8 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   }
   mark(c, 2);
   TRY(head_forward(c, cur, R, true));
-  KL(launch_cross_entropy(c->bf, w.logits, c->Vp, w.rowlabel, inv_n, w.dlogits, c->Vp, w.nll, R, V, c->st));
-  KL(launch_loss_reduce(w.nll, R, inv_n, loss, c->st));
+  KL(PC_CROSS_ENTROPY, (double)R * c->Vp * (4 + c->esz), launch_cross_entropy(c->bf, w.logits, c->Vp, w.rowlabel, inv_n, w.dlogits, c->Vp, w.nll, R, V, c->st));
+  KL(PC_OTHER, 4.0 * R, launch_loss_reduce(w.nll, R, inv_n, loss, c->st));
   TRY(zero_trainable_grads(c));
   TRY(head_backward(c, B, S, P, full));
   mark(c, 3);
@@ -688,9 +719,9 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
     if (need_dx) std::swap(dx, dx_other);
   }
   if (full) {
-    KL(launch_ln_bwd(c->bf, dx, w.z0, w.st0, Wv(c, toff(c, -1, "emb.ln.gamma")), w.dz2,
+    KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, dx, w.z0, w.st0, Wv(c, toff(c, -1, "emb.ln.gamma")), w.dz2,
                      G(c, toff(c, -1, "emb.ln.gamma")), G(c, toff(c, -1, "emb.ln.beta")), T, H, c->st));
-    KL(launch_embed_scatter(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
+    KL(PC_OTHER, 1.0 * T * H * c->esz, launch_embed_scatter(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
                             G(c, toff(c, -1, "emb.pos")), T, S, H, V, c->st));
   }
   mark(c, 4);
@@ -702,7 +733,7 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   h.omb2 = (float)(1.0 - (double)c->opt.beta2);
   h.bc1 = c->opt.bias_correction ? (float)(1.0 / (1.0 - pow((double)c->opt.beta1, (double)c->t_step))) : 1.f;
   h.bc2 = c->opt.bias_correction ? (float)(1.0 / (1.0 - pow((double)c->opt.beta2, (double)c->t_step))) : 1.f;
-  KL(launch_adam(w.chunks, c->n_chunks, c->master, c->grad, c->m, c->v, c->wb, h, c->st));
+  KL(PC_ADAM, 30.0 * c->n_chunks * kAdamChunk, launch_adam(w.chunks, c->n_chunks, c->master, c->grad, c->m, c->v, c->wb, h, c->st));
   mark(c, 5);
   if (c->timing && c->have_events) {
     CUDA_TRY(cudaEventSynchronize(c->ev[5]));
@@ -735,9 +766,9 @@ int mslt_forward(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens
   const int H = c->a.hidden, V = c->a.vocab, T = B * S;
   CUDA_TRY(cudaMemsetAsync(w.scalars, 0, 16, c->st));
   if (head)
-    KL(launch_slots_prepare(d_pos, nullptr, d_seq_lens, B, S, P, V, w.rowsrc, w.rowlabel,
+    KL(PC_OTHER, 8.0 * B * P, launch_slots_prepare(d_pos, nullptr, d_seq_lens, B, S, P, V, w.rowsrc, w.rowlabel,
                             w.scalars + 1, (float*)(w.scalars + 2), w.scalars, c->st));
-  KL(launch_embed_ln(c->bf, d_tokens, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
+  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_embed_ln(c->bf, d_tokens, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
                      Wv(c, toff(c, -1, "emb.ln.gamma")), Wv(c, toff(c, -1, "emb.ln.beta")), w.xa,
                      nullptr, nullptr, T, S, H, V, c->a.ln_eps, w.scalars, c->st));
   char* cur = w.xa;
@@ -811,7 +842,7 @@ int mslt_set_param(mslt_ctx* c, const char* name, const float* src, size_t n) {
   CUDA_TRY(cudaStreamSynchronize(c->st));
   CUDA_TRY(cudaMemcpy(c->master + t->offset, src, n * 4, cudaMemcpyHostToDevice));
   if (c->bf) {
-    KL(launch_f32_to_bf16(c->master + t->offset, c->wb + t->offset * 2, (int64_t)n, c->st));
+    KL(PC_OTHER, 6.0 * n, launch_f32_to_bf16(c->master + t->offset, c->wb + t->offset * 2, (int64_t)n, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
   }
   return 0;
@@ -863,9 +894,9 @@ int mslt_set_timing(mslt_ctx* c, int32_t on) {
   return 0;
 }
 
-int mslt_get_gemm_profile(mslt_ctx* c, double* out, int32_t n) {
-  if (!c || !out || n < 6) return fail(MSLT_ERR_ARG, "need room for 6 doubles");
-  for (int k = 0; k < 2; k++)
+int mslt_get_kernel_profile(mslt_ctx* c, double* out, int32_t n) {
+  if (!c || !out || n < 3 * PC_COUNT) return fail(MSLT_ERR_ARG, "need room for 30 doubles");
+  for (int k = 0; k < PC_COUNT; k++)
     for (int j = 0; j < 3; j++) out[3 * k + j] = c->prof[k][j];
   memset(c->prof, 0, sizeof(c->prof));
   return 0;

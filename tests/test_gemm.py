@@ -156,3 +156,35 @@ def test_batched_attention_addressing(dtype):
     p64 = p.double().cpu().numpy().reshape(Bn, A, S, S)
     ref = np.einsum("bhij,bjhd->bihd", p64, q64[:, :, 2]).reshape(Bn * S, H)
     assert np.abs(ctx.double().cpu().numpy() - ref).max() / np.abs(ref).max() < tol
+
+
+@pytest.mark.parametrize("S", [128, 72, 64, 8])
+def test_bf16_softmax_epilogue(S):
+    """Attention scores with the scaled masked softmax applied in the kernel's epilogue."""
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    Bn, A, dh = 3, 2, 64
+    H = A * dh
+    rng = np.random.default_rng(S)
+    qkv = torch.from_numpy(rng.standard_normal((Bn * S, 3 * H)).astype(np.float32) * 2).cuda().to(torch.bfloat16)
+    lens = np.array([S, max(1, S // 3), 1], dtype=np.int32)
+    d_lens = torch.from_numpy(lens).cuda()
+    prob = torch.full((Bn * A, S, S), 7.0, dtype=torch.bfloat16, device="cuda")
+    d = Bd.GemmDesc()
+    d.dtype, d.M, d.N, d.K, d.batch, d.hdiv, d.alpha = 1, S, S, dh, Bn * A, A, 0.125
+    d.A, d.a_rs, d.a_ks, d.a_bo, d.a_bi = qkv.data_ptr(), 3 * H, 1, S * 3 * H, dh
+    d.B, d.b_rs, d.b_ks, d.b_bo, d.b_bi = qkv.data_ptr() + H * 2, 3 * H, 1, S * 3 * H, dh
+    d.D, d.ldd, d.d_bo, d.d_bi = prob.data_ptr(), S, A * S * S, S * S
+    d.act, d.seq_lens = 3, d_lens.data_ptr()
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Bd.mslt_op_gemm(d, torch.cuda.current_stream().cuda_stream, status)
+    q64 = qkv.double().cpu().numpy().reshape(Bn, S, 3, A, dh)
+    sc = 0.125 * np.einsum("bihd,bjhd->bhij", q64[:, :, 0], q64[:, :, 1])
+    valid = (np.arange(S)[None, :] < lens[:, None])[:, None, None, :]
+    sc = np.where(valid, sc, -np.inf)
+    e = np.exp(sc - sc.max(-1, keepdims=True))
+    ref = (e / e.sum(-1, keepdims=True)).reshape(Bn * A, S, S)
+    got = prob.double().cpu().numpy()
+    assert np.abs(got - ref).max() < 6e-3
+    assert np.all(got[ref == 0] == 0)                  # masked keys are exactly zero
+    np.testing.assert_allclose(got.sum(-1), 1.0, atol=2e-2)
