@@ -216,6 +216,21 @@ int mslt_op_gemm(const mslt_gemm_desc* desc, void* cuda_stream, int32_t* d_statu
  * the caller inspects after synchronising the stream itself. */
 int mslt_op_gemm_enqueue(const mslt_gemm_desc* desc, void* cuda_stream, int32_t* d_status);
 
+/*
+ * The loss kernel alone (MLM objective, Section 4.1; mean over the valid slots as in the step):
+ * for every row r of fp32 logits [R, ldl] with label in [0, V): nll = logsumexp - logit[label];
+ * *d_loss = sum nll / n_valid; d_dlogits (may be NULL) [R, ldd] receives
+ * (softmax - onehot) / n_valid in the dtype's activation type (0: float, 1: bf16), zero rows for
+ * labels < 0 or >= V, zero in columns V..ldd.  ldl, ldd multiples of 8, V <= ldd <= ldl.
+ * d_scratch: device memory of mslt_op_cross_entropy_scratch_bytes(R) bytes, 16-byte aligned,
+ * used for per-row terms; contents on entry do not matter.  All pointers are device pointers.
+ * Synchronises the stream before returning.
+ */
+size_t mslt_op_cross_entropy_scratch_bytes(int32_t R);
+int mslt_op_cross_entropy(int32_t dtype, const float* d_logits, int64_t ldl, const int32_t* d_labels,
+                          int32_t R, int32_t V, void* d_dlogits, int64_t ldd, float* d_loss,
+                          void* d_scratch, size_t scratch_bytes, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -53,7 +53,8 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_set_param", "mslt_get_param_raw", "mslt_get_grad", "mslt_get_opt_state",
            "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_kernel_profile",
            "mslt_last_error",
-           "mslt_op_gemm", "mslt_op_gemm_enqueue"]
+           "mslt_op_gemm", "mslt_op_gemm_enqueue", "mslt_op_cross_entropy",
+           "mslt_op_cross_entropy_scratch_bytes"]
 
 lib.mslt_last_error.restype = C.c_char_p
 lib.mslt_last_error.argtypes = [C.c_void_p]
@@ -88,6 +89,12 @@ lib.mslt_op_gemm.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
 lib.mslt_op_gemm_enqueue.argtypes = [C.POINTER(GemmDesc), C.c_void_p, C.c_void_p]
 
 
+lib.mslt_op_cross_entropy_scratch_bytes.restype = C.c_size_t
+lib.mslt_op_cross_entropy_scratch_bytes.argtypes = [C.c_int32]
+lib.mslt_op_cross_entropy.argtypes = [C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_int32,
+                                      C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
+
+
 class MsltError(RuntimeError):
     def __init__(self, code: int, msg: str):
         super().__init__(f"mslt error {code}: {msg}")
@@ -115,6 +122,15 @@ def mslt_op_gemm(desc: GemmDesc, stream: int, status) -> None:
 
 def mslt_op_gemm_enqueue(desc: GemmDesc, stream: int, status) -> None:
     _check(lib.mslt_op_gemm_enqueue(C.byref(desc), C.c_void_p(stream), C.c_void_p(_ptr(status))))
+
+
+def mslt_op_cross_entropy(dtype: int, logits, labels, V: int, dlogits, loss, scratch, stream: int) -> None:
+    """logits fp32 [R, ldl], labels int32 [R], dlogits [R, ldd] or None, loss fp32 [1], scratch uint8:
+    CUDA tensors."""
+    R = logits.shape[0]
+    _check(lib.mslt_op_cross_entropy(dtype, logits.data_ptr(), logits.stride(0), labels.data_ptr(), R, V,
+                                     _ptr(dlogits), 0 if dlogits is None else dlogits.stride(0),
+                                     loss.data_ptr(), scratch.data_ptr(), scratch.numel(), C.c_void_p(stream)))
 
 
 class Mslt:

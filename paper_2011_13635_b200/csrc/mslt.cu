@@ -33,6 +33,14 @@ int fail(int code, const char* fmt, ...) {
   return code;
 }
 
+}  // namespace
+
+namespace mslt {
+void set_last_error(const char* msg) { snprintf(g_err, sizeof(g_err), "%s", msg); }
+}  // namespace mslt
+
+namespace {
+
 #define CUDA_TRY(x)                                                                  \
   do {                                                                               \
     cudaError_t e_ = (x);                                                            \

@@ -1,0 +1,101 @@
+// Single-kernel entry points of the C ABI, for per-kernel tests and profiling.
+#include <stdarg.h>
+#include <stdio.h>
+
+#include "../../include/mslt.h"
+#include "common.cuh"
+#include "kernels.h"
+
+using namespace mslt;
+
+namespace mslt {
+void set_last_error(const char* msg);  // defined with the C ABI (mslt.cu)
+}
+
+namespace {
+
+int op_fail(int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof(buf), fmt, ap);
+  va_end(ap);
+  set_last_error(buf);
+  return code;
+}
+
+// labels >= V are treated as "ignore" after raising the status bit; counts the valid rows
+__global__ void count_labels_kernel(const int* __restrict__ labels, int R, int V, int* __restrict__ rowlabel,
+                                    int* __restrict__ n_valid, float* __restrict__ inv_n) {
+  __shared__ int cnt;
+  if (threadIdx.x == 0) cnt = 0;
+  __syncthreads();
+  int local = 0;
+  for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    const int lab = labels[r];
+    const bool ok = lab >= 0 && lab < V;
+    rowlabel[r] = ok ? lab : -1;
+    local += ok ? 1 : 0;
+  }
+  if (local) atomicAdd(&cnt, local);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    *n_valid = cnt;
+    *inv_n = cnt > 0 ? 1.0f / (float)cnt : 0.f;
+  }
+}
+
+size_t ce_scratch_bytes(int R) { return ((size_t)R * 8 + 8 + 255) / 256 * 256; }
+
+int check_ce_args(int dtype, const float* logits, int64_t ldl, const int32_t* labels, int R, int V,
+                  const void* dlogits, int64_t ldd, const float* loss) {
+  if (!logits || !labels || !loss) return op_fail(MSLT_ERR_ARG, "cross_entropy: null pointer");
+  if (dtype != 0 && dtype != 1) return op_fail(MSLT_ERR_ARG, "cross_entropy: dtype must be 0 or 1");
+  if (R < 1 || V < 1) return op_fail(MSLT_ERR_ARG, "cross_entropy: bad shape");
+  if (ldl % 8 || ldl < (V + 7) / 8 * 8)
+    return op_fail(MSLT_ERR_ARG, "cross_entropy: ldl must be a multiple of 8 and cover V rounded up to 8");
+  if (dlogits && (ldd % 8 || ldd > ldl || ldd < V))
+    return op_fail(MSLT_ERR_ARG, "cross_entropy: ldd must be a multiple of 8 with V <= ldd <= ldl");
+  if (((uintptr_t)logits | (uintptr_t)dlogits) & 15)
+    return op_fail(MSLT_ERR_ARG, "cross_entropy: buffers must be 16-byte aligned");
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0)
+    return op_fail(MSLT_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  return 0;
+}
+
+// scratch: [R] float nll, [R] int row label, then n_valid (int) and 1/n_valid (float)
+int run_ce(int dtype, const float* logits, int64_t ldl, const int32_t* labels, int R, int V, void* dlogits,
+           int64_t ldd, float* loss, void* scratch, cudaStream_t st) {
+  float* nll = (float*)scratch;
+  int* rowlabel = (int*)scratch + R;
+  int* n_valid = (int*)scratch + 2 * (size_t)R;
+  float* inv_n = (float*)scratch + 2 * (size_t)R + 1;
+  count_labels_kernel<<<1, 256, 0, st>>>(labels, R, V, rowlabel, n_valid, inv_n);
+  launch_cross_entropy(dtype == 1, logits, ldl, rowlabel, inv_n, dlogits, ldd, nll, R, V, st);
+  launch_loss_reduce(nll, R, inv_n, loss, st);
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return op_fail(MSLT_ERR_CUDA, "cross_entropy: %s", cudaGetErrorString(e));
+  return 0;
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t mslt_op_cross_entropy_scratch_bytes(int32_t R) { return R > 0 ? ce_scratch_bytes(R) : 0; }
+
+int mslt_op_cross_entropy(int32_t dtype, const float* d_logits, int64_t ldl, const int32_t* d_labels,
+                          int32_t R, int32_t V, void* d_dlogits, int64_t ldd, float* d_loss,
+                          void* d_scratch, size_t scratch_bytes, void* cuda_stream) {
+  int rc = check_ce_args(dtype, d_logits, ldl, d_labels, R, V, d_dlogits, ldd, d_loss);
+  if (rc) return rc;
+  if (!d_scratch || scratch_bytes < ce_scratch_bytes(R) || ((uintptr_t)d_scratch & 15))
+    return op_fail(MSLT_ERR_SIZE, "cross_entropy: scratch must be 16-byte aligned and hold %zu bytes",
+                   ce_scratch_bytes(R));
+  return run_ce(dtype, d_logits, ldl, d_labels, R, V, d_dlogits, ldd, d_loss, d_scratch,
+                (cudaStream_t)cuda_stream);
+}
+
+}  // extern "C"
