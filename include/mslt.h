@@ -231,6 +231,33 @@ int mslt_op_cross_entropy(int32_t dtype, const float* d_logits, int64_t ldl, con
                           int32_t R, int32_t V, void* d_dlogits, int64_t ldd, float* d_loss,
                           void* d_scratch, size_t scratch_bytes, void* cuda_stream);
 
+/*
+ * mslt_op_cross_entropy without any device allocation by anybody.  (The paper has no counterpart
+ * of this call; it exists for the integration below.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plugin inside a host
+ * application that hands out a fixed memory budget up front, a callback running while another
+ * component owns the allocator lock, a real-time loop that must not touch the driver's
+ * allocator, or a process whose memory pool is already sized to the last byte.  Such callers can
+ * pass inputs and outputs they already own but cannot produce a scratch buffer.
+ *
+ * What it does: the same kernels and the same results as mslt_op_cross_entropy, with the per-row
+ * scratch taken from a fixed array inside the library image instead of from the caller.  The
+ * array holds 16384 rows (about 128 KB) and every GPU that loads the library keeps it until the
+ * process exits.  R > 16384 is refused with MSLT_ERR_SIZE; use the caller-scratch call then.
+ *
+ * The call itself, and everything under it, calls no cudaMalloc, cudaFree or allocating library
+ * routine.  The first call on each device looks up the array's device address (the device must be
+ * current, as for any call here); make that first call outside any stream capture.
+ * All calls on one GPU share the one array, which keeps whatever the last call left in it; each
+ * call overwrites what it reads, so nothing needs clearing, but two calls that overlap in time on
+ * the same GPU (different streams or threads) race on it and give undefined results: serialise
+ * them.  Arguments, layout rules and error codes are those of mslt_op_cross_entropy.
+ */
+int mslt_op_cross_entropy_noalloc(int32_t dtype, const float* d_logits, int64_t ldl,
+                                  const int32_t* d_labels, int32_t R, int32_t V, void* d_dlogits,
+                                  int64_t ldd, float* d_loss, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -54,7 +54,7 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_kernel_profile",
            "mslt_last_error",
            "mslt_op_gemm", "mslt_op_gemm_enqueue", "mslt_op_cross_entropy",
-           "mslt_op_cross_entropy_scratch_bytes"]
+           "mslt_op_cross_entropy_scratch_bytes", "mslt_op_cross_entropy_noalloc"]
 
 lib.mslt_last_error.restype = C.c_char_p
 lib.mslt_last_error.argtypes = [C.c_void_p]
@@ -95,6 +95,10 @@ lib.mslt_op_cross_entropy.argtypes = [C.c_int32, C.c_void_p, C.c_int64, C.c_void
                                       C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
 
 
+lib.mslt_op_cross_entropy_noalloc.argtypes = [C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_int32,
+                                              C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+
+
 class MsltError(RuntimeError):
     def __init__(self, code: int, msg: str):
         super().__init__(f"mslt error {code}: {msg}")
@@ -131,6 +135,15 @@ def mslt_op_cross_entropy(dtype: int, logits, labels, V: int, dlogits, loss, scr
     _check(lib.mslt_op_cross_entropy(dtype, logits.data_ptr(), logits.stride(0), labels.data_ptr(), R, V,
                                      _ptr(dlogits), 0 if dlogits is None else dlogits.stride(0),
                                      loss.data_ptr(), scratch.data_ptr(), scratch.numel(), C.c_void_p(stream)))
+
+
+def mslt_op_cross_entropy_noalloc(dtype: int, logits, labels, V: int, dlogits, loss, stream: int) -> None:
+    """As mslt_op_cross_entropy, with the scratch taken from the library's built-in array (at most
+    16384 rows; calls on one GPU must not overlap)."""
+    R = logits.shape[0]
+    _check(lib.mslt_op_cross_entropy_noalloc(dtype, logits.data_ptr(), logits.stride(0), labels.data_ptr(), R,
+                                             V, _ptr(dlogits), 0 if dlogits is None else dlogits.stride(0),
+                                             loss.data_ptr(), C.c_void_p(stream)))
 
 
 class Mslt:

@@ -2,6 +2,8 @@
 #include <stdarg.h>
 #include <stdio.h>
 
+#include <mutex>
+
 #include "../../include/mslt.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -80,9 +82,57 @@ int run_ce(int dtype, const float* logits, int64_t ldl, const int32_t* labels, i
   return 0;
 }
 
+// ---- allocation-free variant ------------------------------------------------------------------
+// Scratch for mslt_op_cross_entropy_noalloc lives in the library image, so the call needs no
+// cudaMalloc.  Every GPU that loads the library holds these bytes until the process exits.
+constexpr int kNoAllocMaxRows = 16384;
+constexpr size_t kNoAllocBytes = ((size_t)kNoAllocMaxRows * 8 + 8 + 255) / 256 * 256;
+static __device__ __align__(256) unsigned char g_ce_scratch[kNoAllocBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_ce_scratch_ptr[kMaxDevices];  // device address of g_ce_scratch, per device ordinal
+std::mutex g_ce_mu;
+
+// In host code `g_ce_scratch` is only a handle; the address a kernel can use must be asked for,
+// once per device, while that device is current.
+int noalloc_scratch(void** out) {
+  int dev = -1;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return op_fail(MSLT_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+  if (dev < 0 || dev >= kMaxDevices) return op_fail(MSLT_ERR_CUDA, "device ordinal %d not supported", dev);
+  std::lock_guard<std::mutex> lock(g_ce_mu);
+  if (!g_ce_scratch_ptr[dev]) {
+    void* p = nullptr;
+    e = cudaGetSymbolAddress(&p, g_ce_scratch);
+    if (e != cudaSuccess || !p)
+      return op_fail(MSLT_ERR_CUDA, "cudaGetSymbolAddress(scratch): %s", cudaGetErrorString(e));
+    g_ce_scratch_ptr[dev] = p;
+  }
+  *out = g_ce_scratch_ptr[dev];
+  return 0;
+}
+
 }  // namespace
 
 extern "C" {
+
+int mslt_op_cross_entropy_noalloc(int32_t dtype, const float* d_logits, int64_t ldl,
+                                  const int32_t* d_labels, int32_t R, int32_t V, void* d_dlogits,
+                                  int64_t ldd, float* d_loss, void* cuda_stream) {
+  int rc = check_ce_args(dtype, d_logits, ldl, d_labels, R, V, d_dlogits, ldd, d_loss);
+  if (rc) return rc;
+  if (R > kNoAllocMaxRows)
+    return op_fail(MSLT_ERR_SIZE, "cross_entropy_noalloc: R = %d exceeds the built-in scratch (%d rows); "
+                   "use mslt_op_cross_entropy with caller scratch", R, kNoAllocMaxRows);
+  void* scratch = nullptr;
+  rc = noalloc_scratch(&scratch);
+  if (rc) return rc;
+  // nothing in the scratch has to start at zero: every word the kernels read is written earlier in
+  // the same call (row labels and the count first, then the per-row terms)
+  return run_ce(dtype, d_logits, ldl, d_labels, R, V, d_dlogits, ldd, d_loss, scratch,
+                (cudaStream_t)cuda_stream);
+}
+
 
 size_t mslt_op_cross_entropy_scratch_bytes(int32_t R) { return R > 0 ? ce_scratch_bytes(R) : 0; }
 
