@@ -1,0 +1,83 @@
+"""Parity at the full architecture sizes of the benchmark configurations.
+
+The oracle cannot run a 128-sequence batch of a 12- or 24-layer model in seconds, so:
+  * every configuration runs at its full architecture (depth, widths, vocabulary, sequence length,
+    frozen/trainable split) on a batch of a few sequences and is compared element by element;
+  * the launch configuration bench.py times (BERT-Base stage, batch 128) is checked on sampled
+    sequences (sequences are independent in the forward pass, so the oracle computes those alone)
+    and through properties that hold at any size.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from oracle import mslt_oracle as O
+from paper_2011_13635_b200 import inputs as I
+from tests import parity as PT
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("name,batch", [("base_stage", 4), ("base_full", 3), ("large_stage", 2),
+                                        ("large_long", 1)])
+def test_full_architecture_small_batch(name, batch):
+    cfg = I.scaled(I.CONFIGS[name], batch=batch)
+    m, oracle = PT.build_pair(cfg, lr=1e-4)
+    rep = []
+    PT.compare_step(m, oracle, cfg, I.make_batch(cfg), PT.TOL[cfg.dtype], rep)
+    assert abs(rep[0]["loss_gpu"] - math.log(cfg.vocab)) < 0.5
+    m.close()
+
+
+def test_bench_launch_configuration_sampled():
+    """BERT-Base stage at batch 128, exactly what bench.py launches."""
+    import torch
+    cfg = I.CONFIGS["base_stage"]
+    m, _ = PT.build_pair(cfg, lr=1e-4)          # the oracle of this pair is not stepped
+    tok, lens, pos, lab = I.make_batch(cfg)
+    d_tok, d_pos, d_lab = PT.to_cuda(torch, tok, pos, lab)
+    hidden, logits = m.mslt_forward(d_tok, None, d_pos)
+    hidden = hidden.float().cpu().numpy()
+    logits = logits.cpu().numpy().reshape(cfg.batch, cfg.pred, cfg.vocab)
+    w = I.make_weights(cfg, variant="parity")
+    ref = O.MsltOracle(w, cfg.heads)
+    tol = PT.TOL["bf16"]["hidden"]
+    sample = [0, 77, 127]
+    h_ref, l_ref = ref.forward(tok[sample], lens[sample], pos[sample])
+    l_ref = l_ref.reshape(len(sample), cfg.pred, cfg.vocab)
+    for i, b in enumerate(sample):
+        assert PT.max_rel(hidden[b], h_ref[i]) < tol
+        ok = pos[b] >= 0
+        assert PT.max_rel(logits[b][ok], l_ref[i][ok]) < tol
+    # loss of the whole batch = mean over valid slots of the per-slot terms of these logits
+    ok = (pos >= 0) & (lab >= 0)
+    lg = logits[ok].astype(np.float64)
+    lse = np.log(np.exp(lg - lg.max(1, keepdims=True)).sum(1)) + lg.max(1)
+    nll = lse - lg[np.arange(len(lg)), lab[ok]]
+    frozen = [n for n, i in m.tensors().items() if not i["trainable"]]
+    before = {n: m.mslt_get_param_raw(n) for n in frozen}
+    loss = m.mslt_step(d_tok, None, d_pos, d_lab)
+    assert abs(loss - nll.mean()) / nll.mean() < 1e-5
+    # properties that hold at any size
+    g = m.mslt_get_grad("head.decoder.bias")
+    # every dlogits row sums to zero; its entries are rounded to bf16 (relative 2^-9 each)
+    assert abs(g.sum()) < 2.0 ** -8 * np.abs(g).sum()
+    for n in frozen:
+        assert np.array_equal(before[n], m.mslt_get_param_raw(n)), n
+    # gradient of the batch = slot-weighted sum of the gradients of its two halves
+    names = ["layer.11.ffn1.weight", "layer.9.qkv.weight", "head.transform.weight", "layer.10.ln1.gamma"]
+    full = {n: m.mslt_get_grad(n) for n in names}
+    m.close()
+    acc = {n: 0.0 for n in names}
+    n_all = int(ok.sum())
+    for half in (slice(0, 64), slice(64, 128)):
+        mh, _ = PT.build_pair(cfg, lr=1e-4)
+        d = PT.to_cuda(torch, tok[half], pos[half], lab[half])
+        mh.mslt_step(d[0], None, d[1], d[2])
+        wgt = int(ok[half].sum()) / n_all
+        for n in names:
+            acc[n] = acc[n] + wgt * mh.mslt_get_grad(n)
+        mh.close()
+    for n in names:
+        assert PT.max_rel(acc[n], full[n]) < 2e-2, n
