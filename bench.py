@@ -190,6 +190,22 @@ def time_steps(m, dev, torch, steps, warmup, sync_fn):
     return e0.elapsed_time(e1), m.launch_count - before
 
 
+def rank_seed(cfg, rank: int) -> int:
+    """Every replica draws its own batch."""
+    return I.config_seed(cfg) + 1000 * rank
+
+
+def aggregate(ms_local: float, batch_per_rank: int, steps: int, world: int, dist=None, device="cpu"):
+    """(max over ranks of the timed region in ms, whole-job sequences/s): replicas share nothing, so
+    the job is as slow as its slowest rank and processes world * batch sequences per step."""
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms = float(t.item())
+    return ms, batch_per_rank * world * steps / (ms * 1e-3)
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -206,7 +222,7 @@ def run_ours(args, cfg):
             dist.barrier()
             torch.cuda.synchronize()
 
-    host = [np.ascontiguousarray(a) for a in I.make_batch(cfg, seed=I.config_seed(cfg) + 1000 * rank)]
+    host = [np.ascontiguousarray(a) for a in I.make_batch(cfg, seed=rank_seed(cfg, rank))]
     if cfg.varlen is None:
         host[1] = None
     pinned = [None if a is None else torch.from_numpy(a).pin_memory() for a in host]
@@ -219,11 +235,7 @@ def run_ours(args, cfg):
     with ClockSampler(local) as clk:
         ms, launches = time_steps(m, dev, torch, args.steps, args.warmup, sync)
     loss_end = m.mslt_read_loss()
-    t = torch.tensor([ms], device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms = float(t.item())
-    value = cfg.batch * world * args.steps / (ms * 1e-3)
+    ms, value = aggregate(ms, cfg.batch, args.steps, world, dist, "cuda")
 
     # end to end: pinned host inputs copied in, loss read back, every step
     sync()
@@ -234,10 +246,8 @@ def run_ours(args, cfg):
         m.mslt_step(*d)
     t1.record()
     sync()
-    te = torch.tensor([t0.elapsed_time(t1)], device="cuda")
-    if world > 1:
-        dist.all_reduce(te, op=dist.ReduceOp.MAX)
-    e2e = dict(value=cfg.batch * world * args.steps / (float(te.item()) * 1e-3), unit=UNIT,
+    _, e2e_value = aggregate(t0.elapsed_time(t1), cfg.batch, args.steps, world, dist, "cuda")
+    e2e = dict(value=e2e_value, unit=UNIT,
                h2d_bytes_per_step=int(sum(a.nbytes for a in host if a is not None)),
                d2h_bytes_per_step=16)
 
