@@ -18,6 +18,7 @@
 // Every wait is bounded: when one runs out the CTA raises a status bit, drains and returns.
 #include <cuda.h>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include <mutex>
@@ -112,6 +113,49 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
       ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
+// ---- CTA-pair (cta_group::2) forms: the two CTAs of a cluster work on one 256-row tile ----
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t mapa_u32(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+// the copy lands in this CTA's shared memory; its bytes are counted on the leader CTA's barrier
+__device__ __forceinline__ void tma_load_4d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster,
+                                                 int c0, int c1, int c2, int c3) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes "
+      "[%0], [%1, {%3, %4, %5, %6}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {  // arrives on the barrier in both CTAs
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3)
+      : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -298,14 +342,23 @@ __device__ __forceinline__ bool pair_sync(volatile int* flags, int me, int other
 
 // ---- the kernel ---------------------------------------------------------------------------------
 // 10 warps are allocated registers as 12, which caps a thread at 168 registers
-template <bool kSoftmax>
+template <bool kSoftmax, bool kPair>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle pattern
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  const int b_stage_bytes = p.bn * BK * 2;
+  // CTA-pair mode: the two CTAs of a cluster share one 256 x 256 tile.  Each loads its own 128
+  // rows of A and its own 128 columns of B; the leader (rank 0) issues MMAs that read both CTAs'
+  // shared memory and write both CTAs' tensor memory.
+  const uint32_t cta_rank = kPair ? cluster_ctarank() : 0u;
+  const bool leader = cta_rank == 0;
+  const int bn_cta = kPair ? p.bn / 2 : p.bn;   // B columns held by this CTA
+  const int mt_rows = kPair ? 2 * BM : BM;      // rows of a work item's output tile
+  const int w_first = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int w_step = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int b_stage_bytes = bn_cta * BK * 2;
   const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
   uint8_t* staging = smem + (size_t)p.stages * stage_bytes;
   uint64_t* bars = (uint64_t*)(staging + NUM_EPI_WARPS * STAGING_BYTES);
@@ -329,7 +382,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
     for (int a = 0; a < 2; a++) {
       mbar_init(smem_u32(&tfull_bar[a]), 1);
-      mbar_init(smem_u32(&tempty_bar[a]), NUM_EPI_WARPS);
+      mbar_init(smem_u32(&tempty_bar[a]), kPair ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS);
     }
     *abort_flag = 0;
     if (kSoftmax)
@@ -337,13 +390,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                 "r"(TMEM_COLS)
-                 : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    if (kPair) {
+      asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    } else {
+      asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                   "r"(TMEM_COLS)
+                   : "memory");
+      asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
   }
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();  // the peer's barriers must exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -354,7 +415,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     // ------------------------------- TMA producer -------------------------------
     uint32_t it = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < p.total_work && ok; w += gridDim.x) {
+    for (int w = w_first; w < p.total_work && ok; w += w_step) {
       const int split = w / per_split;
       int r = w - split * per_split;
       const int z = r / tiles_per_z;
@@ -366,37 +427,49 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int kb = kb0; kb < kb1; kb++, it++) {
         const uint32_t s = it % p.stages, round = it / p.stages;
         if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
-        const uint32_t fb = smem_u32(&full_bar[s]);
-        mbar_expect_tx(fb, stage_bytes);
+        const uint32_t fb_own = smem_u32(&full_bar[s]);
+        // pair mode: both CTAs' copies are counted on the leader's barrier
+        const uint32_t fb = kPair ? mapa_u32(fb_own, 0) : fb_own;
+        if (leader) mbar_expect_tx(fb_own, kPair ? 2 * stage_bytes : stage_bytes);
         const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
         const uint32_t sb = sa + A_STAGE_BYTES;
+        const int row0 = mt * mt_rows + (int)cta_rank * BM;
+        const int col0 = nt * p.bn + (int)cta_rank * bn_cta;
         int c[4];
         if (!p.a_mn) {  // box {64 k, 128 rows}
-          c[0] = kb * BK; c[p.a_perm[0]] = mt * BM; c[p.a_perm[1]] = zi; c[p.a_perm[2]] = zo;
-          tma_load_4d(sa, &tmA, fb, c[0], c[1], c[2], c[3]);
+          c[0] = kb * BK; c[p.a_perm[0]] = row0; c[p.a_perm[1]] = zi; c[p.a_perm[2]] = zo;
+          if (kPair) tma_load_4d_pair(sa, &tmA, fb, c[0], c[1], c[2], c[3]);
+          else tma_load_4d(sa, &tmA, fb, c[0], c[1], c[2], c[3]);
         } else {        // two boxes {64 rows, 64 k}
           c[p.a_perm[0]] = kb * BK; c[p.a_perm[1]] = zi; c[p.a_perm[2]] = zo;
 #pragma unroll
           for (int h = 0; h < BM / 64; h++) {
-            c[0] = mt * BM + h * 64;
-            tma_load_4d(sa + h * (64 * BK * 2), &tmA, fb, c[0], c[1], c[2], c[3]);
+            c[0] = row0 + h * 64;
+            if (kPair) tma_load_4d_pair(sa + h * (64 * BK * 2), &tmA, fb, c[0], c[1], c[2], c[3]);
+            else tma_load_4d(sa + h * (64 * BK * 2), &tmA, fb, c[0], c[1], c[2], c[3]);
           }
         }
-        if (!p.b_mn) {  // box {64 k, bn rows}
-          c[0] = kb * BK; c[p.b_perm[0]] = nt * p.bn; c[p.b_perm[1]] = zi; c[p.b_perm[2]] = zo;
-          tma_load_4d(sb, &tmB, fb, c[0], c[1], c[2], c[3]);
+        if (!p.b_mn) {  // box {64 k, this CTA's B rows}
+          c[0] = kb * BK; c[p.b_perm[0]] = col0; c[p.b_perm[1]] = zi; c[p.b_perm[2]] = zo;
+          if (kPair) tma_load_4d_pair(sb, &tmB, fb, c[0], c[1], c[2], c[3]);
+          else tma_load_4d(sb, &tmB, fb, c[0], c[1], c[2], c[3]);
         } else {
           c[p.b_perm[0]] = kb * BK; c[p.b_perm[1]] = zi; c[p.b_perm[2]] = zo;
-          for (int h = 0; h < p.bn / 64; h++) {
-            c[0] = nt * p.bn + h * 64;
-            tma_load_4d(sb + h * (64 * BK * 2), &tmB, fb, c[0], c[1], c[2], c[3]);
+          for (int h = 0; h < bn_cta / 64; h++) {
+            c[0] = col0 + h * 64;
+            if (kPair) tma_load_4d_pair(sb + h * (64 * BK * 2), &tmB, fb, c[0], c[1], c[2], c[3]);
+            else tma_load_4d(sb + h * (64 * BK * 2), &tmB, fb, c[0], c[1], c[2], c[3]);
           }
         }
       }
     }
     if (!ok || *abort_flag) {
       // give up: let the copies already in flight land before the CTA leaves
-      const uint32_t n = it < (uint32_t)p.stages ? it : (uint32_t)p.stages;
+      const uint32_t n = !leader ? 0u : (it < (uint32_t)p.stages ? it : (uint32_t)p.stages);
+      if (!leader) {  // its copies are counted on the leader's barriers: give them time to land
+        const long long t0 = now_cycles();
+        while (now_cycles() - t0 < 2000000ll) {}
+      }
       for (uint32_t i = 0; i < n; i++) {
         const uint32_t j = it - 1 - i;
         const uint32_t fb = smem_u32(&full_bar[j % p.stages]);
@@ -404,7 +477,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         while (!mbar_try_wait(fb, (j / p.stages) & 1) && now_cycles() - t0 < 200000000ll) {}
       }
     }
-  } else if (warp == 1 && lane == 0) {
+  } else if (warp == 1 && lane == 0 && leader) {
     // ------------------------------- MMA issuer -------------------------------
     uint32_t it = 0, tile = 0;
     bool ok = true;
@@ -412,7 +485,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint32_t b_lbo = p.b_mn ? 64 * BK * 2 : 16;
     const uint32_t a_kstep = p.a_mn ? UMMA_K * 128 : UMMA_K * 2;  // bytes per 16-wide k step
     const uint32_t b_kstep = p.b_mn ? UMMA_K * 128 : UMMA_K * 2;
-    for (int w = blockIdx.x; w < p.total_work && ok; w += gridDim.x, tile++) {
+    for (int w = w_first; w < p.total_work && ok; w += w_step, tile++) {
       const int split = w / per_split;
       const int kb0 = split * p.kb_per_split;
       const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
@@ -430,15 +503,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         for (int k = 0; k < BK / UMMA_K; k++) {
           const uint64_t ad = make_smem_desc(sa + k * a_kstep, a_lbo);
           const uint64_t bd = make_smem_desc(sb + k * b_kstep, b_lbo);
-          tc_mma(d_tmem, ad, bd, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          if (kPair) tc_mma_pair(d_tmem, ad, bd, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          else tc_mma(d_tmem, ad, bd, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
         }
-        tc_commit(smem_u32(&empty_bar[s]));  // stage is free once these MMAs have read it
+        // the stage is free (in both CTAs) once these MMAs have read it
+        if (kPair) tc_commit_pair(smem_u32(&empty_bar[s])); else tc_commit(smem_u32(&empty_bar[s]));
       }
-      if (ok) tc_commit(smem_u32(&tfull_bar[acc]));  // accumulator complete
+      if (ok) {  // accumulator complete
+        if (kPair) tc_commit_pair(smem_u32(&tfull_bar[acc])); else tc_commit(smem_u32(&tfull_bar[acc]));
+      }
     }
     if (!ok || *abort_flag) {
       // make sure no MMA is still writing tensor memory before it is freed
-      tc_commit(smem_u32(&tfull_bar[0]));
+      if (kPair) tc_commit_pair(smem_u32(&tfull_bar[0])); else tc_commit(smem_u32(&tfull_bar[0]));
       const long long t0 = now_cycles();
       while (now_cycles() - t0 < 2000000ll) {}
     }
@@ -452,7 +529,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     uint8_t* stg = staging + (size_t)(warp - 2) * STAGING_BYTES;
     uint32_t tile = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < p.total_work && ok; w += gridDim.x, tile++) {
+    for (int w = w_first; w < p.total_work && ok; w += w_step, tile++) {
       const int split = w / per_split;
       int r = w - split * per_split;
       const int z = r / tiles_per_z;
@@ -462,7 +539,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const uint32_t acc = tile & 1, use = tile >> 1;
       if (!mbar_wait(smem_u32(&tfull_bar[acc]), use & 1, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      const int m_warp = mt * BM + q * 32;  // first row of this warp
+      const int m_warp = mt * mt_rows + (int)cta_rank * BM + q * 32;  // first row of this warp
       const int m = m_warp + lane;
       const long long zoff = zo * p.d_bo + zi * p.d_bi;
       const long long off0 = zoff + (long long)m * p.ldd;
@@ -497,7 +574,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // the accumulator is in registers now: hand it back before the slow part
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+        if (lane == 0) {
+        if (kPair && !leader) mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[acc]), 0));
+        else mbar_arrive(smem_u32(&tempty_bar[acc]));
+      }
         const int seq = (int)tile * 2 + 1;
         const int me = q * 2 + hsel, other = q * 2 + (hsel ^ 1);
         xmax[me * 32 + lane] = mx;
@@ -597,18 +677,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       // hand the accumulator back to the MMA warp
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&tempty_bar[acc]));
+      if (lane == 0) {
+        if (kPair && !leader) mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[acc]), 0));
+        else mbar_arrive(smem_u32(&tempty_bar[acc]));
+      }
       }
     }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (kPair) cluster_sync_all();  // neither CTA frees tensor memory while the other may still use it
   if (warp == 1) {
     __syncwarp();
     tc_fence_after();
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
-                 : "memory");
+    if (kPair)
+      asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
+                   : "memory");
+    else
+      asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS)
+                   : "memory");
   }
 }
 
@@ -733,15 +821,25 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   p.a_mn = (d.a_rs == 1 && d.a_ks != 1) ? 1 : 0;
   p.b_mn = (d.b_rs == 1 && d.b_ks != 1) ? 1 : 0;
   p.bn = d.N <= 64 ? 64 : (d.N <= 128 ? 128 : 256);
-  p.m_tiles = (d.M + BM - 1) / BM;
+  // Two CTAs per 256 x 256 tile: each SM then streams 64 instead of 96 bytes of operands per clock
+  // from L2 and has six instead of four stages in flight.  MSLT_GEMM_SINGLE_CTA=1 keeps one CTA per
+  // tile (for A/B measurements).
+  static const bool single_cta = getenv("MSLT_GEMM_SINGLE_CTA") && atoi(getenv("MSLT_GEMM_SINGLE_CTA")) == 1;
+  // Measured: the pair wins for row-contiguous (MN-major) operands and for deep contractions, and is
+  // on par or slightly behind for shallow k-contiguous products, which are bound by their epilogue.
+  const bool pair = !single_cta && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0 &&
+                    (p.a_mn || p.b_mn || d.K >= 2048);
+  const int tile_m = pair ? 2 * BM : BM;
+  p.m_tiles = (d.M + tile_m - 1) / tile_m;
   p.n_tiles = (d.N + p.bn - 1) / p.bn;
   p.kb_total = (d.K + BK - 1) / BK;
   const long long tiles = (long long)p.m_tiles * p.n_tiles * d.batch;
+  const int units = pair ? num_sms / 2 : num_sms;  // CTAs or CTA pairs that run concurrently
   int splits = 1;
   if (d.split_k > 1) {
     splits = d.split_k;
-  } else if (d.split_k == 0 && d.d_fp32 && d.accumulate && tiles < num_sms && p.kb_total >= 8) {
-    splits = (int)(num_sms / tiles);
+  } else if (d.split_k == 0 && d.d_fp32 && d.accumulate && tiles < units && p.kb_total >= 8) {
+    splits = (int)(units / tiles);
     const int max_by_k = p.kb_total / 4;  // keep at least four k blocks per split
     if (splits > max_by_k) splits = max_by_k;
     if (splits < 1) splits = 1;
@@ -760,7 +858,7 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
     snprintf(err, 256, "gemm: the softmax epilogue needs bf16 output rows of at most 128 columns");
     return MSLT_ERR_ARG;
   }
-  const int stage_bytes = A_STAGE_BYTES + p.bn * BK * 2;
+  const int stage_bytes = A_STAGE_BYTES + (pair ? p.bn / 2 : p.bn) * BK * 2;  // per CTA
   const int book_bytes = 256 + (d.act == 3 ? 64 + 2 * NUM_EPI_WARPS * 32 * 4 : 0);
   int stages = (smem_optin - NUM_EPI_WARPS * STAGING_BYTES - 1024 - book_bytes) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
@@ -774,7 +872,7 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   if (d.batch % d.hdiv) { snprintf(err, 256, "gemm: batch must be a multiple of hdiv"); return MSLT_ERR_ARG; }
   int rc = get_map(d.A, d.M, d.K, d.a_rs, d.a_ks, d.a_bo, d.a_bi, d.hdiv, nb, BM, &ma, err);
   if (rc) return rc;
-  rc = get_map(d.B, d.N, d.K, d.b_rs, d.b_ks, d.b_bo, d.b_bi, d.hdiv, nb, p.bn, &mb, err);
+  rc = get_map(d.B, d.N, d.K, d.b_rs, d.b_ks, d.b_bo, d.b_bi, d.hdiv, nb, pair ? p.bn / 2 : p.bn, &mb, err);
   if (rc) return rc;
   for (int i = 0; i < 3; i++) { p.a_perm[i] = ma.perm[i]; p.b_perm[i] = mb.perm[i]; }
 
@@ -789,21 +887,42 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
               al16(d.residual) && al16(d.bias)) ? 1 : 0;
   // instruction descriptor: fp32 accumulate, bf16 x bf16, operand majors, N and M of the tile
   p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
-            ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+            ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
 
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
     if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+      e = cudaFuncSetAttribute(gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    if (e == cudaSuccess)
+      e = cudaFuncSetAttribute(gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
     if (e != cudaSuccess) { snprintf(err, 256, "gemm: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
     attr_set = true;
   }
+  if (pair) {
+    const int clusters = p.total_work < units ? p.total_work : units;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3(2 * clusters);
+    cfg.blockDim = dim3(NUM_THREADS);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<false, true>, ma.map, mb.map, p);
+    if (e != cudaSuccess) { snprintf(err, 256, "gemm: cluster launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+    return 0;
+  }
   const int grid = p.total_work < num_sms ? p.total_work : num_sms;
   if (d.act == 3)
-    gemm_tc_kernel<true><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
+    gemm_tc_kernel<true, false><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
   else
-    gemm_tc_kernel<false><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
+    gemm_tc_kernel<false, false><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { snprintf(err, 256, "gemm: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
   return 0;
