@@ -827,8 +827,24 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   static const bool single_cta = getenv("MSLT_GEMM_SINGLE_CTA") && atoi(getenv("MSLT_GEMM_SINGLE_CTA")) == 1;
   // Measured: the pair wins for row-contiguous (MN-major) operands and for deep contractions, and is
   // on par or slightly behind for shallow k-contiguous products, which are bound by their epilogue.
-  const bool pair = !single_cta && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0 &&
-                    (p.a_mn || p.b_mn || d.K >= 2048);
+  bool pair = !single_cta && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0 &&
+              (p.a_mn || p.b_mn || d.K >= 2048);
+  // share of the SMs that the last wave of tiles keeps busy
+  auto wave_eff = [](long long work, int units_) {
+    const long long waves = (work + units_ - 1) / units_;
+    return (double)work / (double)(waves * units_);
+  };
+  const bool can_split = d.split_k != 1 && d.d_fp32 && d.accumulate;
+  if (p.bn == 256 && !can_split) {
+    // few large tiles leave SMs idle: 128-wide tiles on single CTAs may fill the machine better
+    const long long t256 = (long long)((d.M + (pair ? 2 * BM : BM) - 1) / (pair ? 2 * BM : BM)) *
+                           ((d.N + 255) / 256) * d.batch;
+    const long long t128 = (long long)((d.M + BM - 1) / BM) * ((d.N + 127) / 128) * d.batch;
+    if (wave_eff(t128, num_sms) > 1.25 * wave_eff(t256, pair ? num_sms / 2 : num_sms)) {
+      p.bn = 128;
+      pair = false;
+    }
+  }
   const int tile_m = pair ? 2 * BM : BM;
   p.m_tiles = (d.M + tile_m - 1) / tile_m;
   p.n_tiles = (d.N + p.bn - 1) / p.bn;
@@ -838,11 +854,14 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   int splits = 1;
   if (d.split_k > 1) {
     splits = d.split_k;
-  } else if (d.split_k == 0 && d.d_fp32 && d.accumulate && tiles < units && p.kb_total >= 8) {
-    splits = (int)(units / tiles);
-    const int max_by_k = p.kb_total / 4;  // keep at least four k blocks per split
-    if (splits > max_by_k) splits = max_by_k;
-    if (splits < 1) splits = 1;
+  } else if (d.split_k == 0 && can_split && tiles < 2 * units && p.kb_total >= 8) {
+    // the split count that fills the last wave best, with at least four k blocks per split
+    const int max_by_k = p.kb_total / 4;
+    double best = wave_eff(tiles, units);
+    for (int sp = 2; sp <= 16 && sp <= max_by_k; sp++) {
+      const double e = wave_eff(tiles * sp, units);
+      if (e > best + 0.04) { best = e; splits = sp; }
+    }
   }
   if (splits > 1 && !(d.d_fp32 && d.accumulate)) {
     snprintf(err, 256, "gemm: split_k needs an fp32 accumulating output");

@@ -70,31 +70,94 @@ __device__ __forceinline__ void ln_finish_row(float (&x)[LN_MAXE], int lane, int
   }
 }
 
-template <typename T>
-__global__ void __launch_bounds__(256) ln_fwd_kernel(const T* __restrict__ z,
-                                                     const float* __restrict__ gamma,
-                                                     const float* __restrict__ beta,
-                                                     T* __restrict__ y, float* __restrict__ stats,
-                                                     int rows, int H, float eps) {
+// One warp normalises ROWS consecutive rows at once: all their 16-byte loads are issued before
+// the first reduction, which keeps enough bytes in flight to approach HBM bandwidth, and gamma /
+// beta are fetched once per column vector for all ROWS rows.  NV = 16-byte vectors per lane.
+template <typename T, int NV, int ROWS>
+__global__ void __launch_bounds__(256)
+ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ gamma, const float* __restrict__ beta,
+              T* __restrict__ y, float* __restrict__ stats, int rows, int H, float eps) {
   constexpr int VN = VecT<T>::N;
-  constexpr int NV = LN_MAXE / VN;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  typedef typename VecT<T>::Raw Raw;
   const int lane = threadIdx.x & 31;
-  if (row >= rows) return;
-  float x[LN_MAXE];
-  const T* zr = z + (int64_t)row * H;
+  const int row0 = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * ROWS;
+  if (row0 >= rows) return;
+  Raw raw[ROWS][NV];
+#pragma unroll
+  for (int r = 0; r < ROWS; r++)
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (lane + 32 * i) * VN;
+      if (c < H && row0 + r < rows) raw[r][i] = VecT<T>::load_raw(z + (int64_t)(row0 + r) * H + c);
+    }
+  float mean[ROWS], rstd[ROWS];
+#pragma unroll
+  for (int r = 0; r < ROWS; r++) {
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      if ((lane + 32 * i) * VN < H && row0 + r < rows) {
+        float t[VN];
+        VecT<T>::unpack(raw[r][i], t);
+#pragma unroll
+        for (int e = 0; e < VN; e++) s += t[e];
+      }
+    }
+    mean[r] = s;
+  }
+#pragma unroll
+  for (int r = 0; r < ROWS; r++) mean[r] = warp_sum(mean[r]) / (float)H;
+#pragma unroll
+  for (int r = 0; r < ROWS; r++) {
+    float q = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      if ((lane + 32 * i) * VN < H && row0 + r < rows) {
+        float t[VN];
+        VecT<T>::unpack(raw[r][i], t);
+#pragma unroll
+        for (int e = 0; e < VN; e++) {
+          const float d = t[e] - mean[r];
+          q += d * d;
+        }
+      }
+    }
+    rstd[r] = q;
+  }
+#pragma unroll
+  for (int r = 0; r < ROWS; r++) rstd[r] = rsqrtf(warp_sum(rstd[r]) / (float)H + eps);
+  if (stats != nullptr && lane == 0) {
+#pragma unroll
+    for (int r = 0; r < ROWS; r++)
+      if (row0 + r < rows) {
+        stats[2 * (int64_t)(row0 + r)] = mean[r];
+        stats[2 * (int64_t)(row0 + r) + 1] = rstd[r];
+      }
+  }
 #pragma unroll
   for (int i = 0; i < NV; i++) {
     const int c = (lane + 32 * i) * VN;
-    float t[VN];
     if (c < H) {
-      VecT<T>::load(zr + c, t);
+      float g[VN], b[VN];
 #pragma unroll
-      for (int e = 0; e < VN; e++) x[i * VN + e] = t[e];
+      for (int e = 0; e < VN; e += 4) {
+        const float4 g4 = *reinterpret_cast<const float4*>(gamma + c + e);
+        const float4 b4 = *reinterpret_cast<const float4*>(beta + c + e);
+        g[e] = g4.x; g[e + 1] = g4.y; g[e + 2] = g4.z; g[e + 3] = g4.w;
+        b[e] = b4.x; b[e + 1] = b4.y; b[e + 2] = b4.z; b[e + 3] = b4.w;
+      }
+#pragma unroll
+      for (int r = 0; r < ROWS; r++) {
+        if (row0 + r < rows) {
+          float t[VN], o[VN];
+          VecT<T>::unpack(raw[r][i], t);
+#pragma unroll
+          for (int e = 0; e < VN; e++) o[e] = g[e] * ((t[e] - mean[r]) * rstd[r]) + b[e];
+          VecT<T>::store(y + (int64_t)(row0 + r) * H + c, o);
+        }
+      }
     }
   }
-  ln_finish_row<T>(x, lane, H, gamma, beta, y + (int64_t)row * H,
-                   stats ? stats + 2 * (int64_t)row : nullptr, eps);
 }
 
 // Embedding: z = word[token] + pos[s]; optional stash of z; then LayerNorm.
@@ -644,8 +707,18 @@ __global__ void f32_to_bf16_kernel(const float* __restrict__ src, bf16* __restri
 void launch_ln_fwd(bool bf, const void* z, const float* gamma, const float* beta, void* y,
                    float* stats, int rows, int H, float eps, cudaStream_t st) {
   if (rows <= 0) return;
-  DISPATCH_T(bf, (ln_fwd_kernel<T><<<div_up(rows, 8), 256, 0, st>>>(
-                     (const T*)z, gamma, beta, (T*)y, stats, rows, H, eps)));
+  const int vn = bf ? 8 : 4;
+  const int nv = (H + 32 * vn - 1) / (32 * vn);
+#define LN_FWD(NV, ROWS)                                                                             \
+  DISPATCH_T(bf, (ln_fwd_kernel<T, NV, ROWS><<<div_up(rows, 8 * ROWS), 256, 0, st>>>(                  \
+                     (const T*)z, gamma, beta, (T*)y, stats, rows, H, eps)))
+  if (nv <= 1) LN_FWD(1, 4);
+  else if (nv <= 2) LN_FWD(2, 4);
+  else if (nv <= 3) LN_FWD(3, 4);
+  else if (nv <= 4) LN_FWD(4, 4);
+  else if (nv <= 6) LN_FWD(6, 2);
+  else LN_FWD(8, 2);
+#undef LN_FWD
 }
 
 void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* pos,
