@@ -206,27 +206,24 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
   return d;
 }
 
-// erf on the FMA pipe only: the epilogue of a GELU tile is bound by the special-function unit
-// when erf costs a reciprocal and an exponential per element.  Odd polynomial x * P(x^2) of degree
-// 17, least-maximum-error fit on |x| <= 3 (absolute error below 3e-5 in fp32, far inside bf16
-// resolution); beyond that erf is +-1 to within 2.3e-5.
-__device__ __forceinline__ float erf_poly(float x) {
-  const float y = fminf(fmaxf(x, -3.0f), 3.0f);
-  const float t = y * y;
-  float p = 4.074212625e-08f;
-  p = fmaf(p, t, -1.944823467e-06f);
-  p = fmaf(p, t, 4.106053568e-05f);
-  p = fmaf(p, t, -5.110369647e-04f);
-  p = fmaf(p, t, 4.235427931e-03f);
-  p = fmaf(p, t, -2.510286290e-02f);
-  p = fmaf(p, t, 1.110793384e-01f);
-  p = fmaf(p, t, -3.753148786e-01f);
-  p = fmaf(p, t, 1.128268426e+00f);
-  p *= y;
-  return fabsf(x) >= 3.0f ? copysignf(1.0f, x) : p;
-}
+// GELU on the FMA pipe only: the epilogue of a GELU tile is bound by the special-function unit when
+// erf costs a reciprocal and an exponential per element.  gelu(u) = u * Phi(u) with
+// Phi(u) - 1/2 = u * Q(u^2), Q a degree-8 least-maximum-error fit on |u| <= 4 (gelu is off by less
+// than 3e-5 in fp32 there, far inside bf16 resolution); outside, the argument is clamped, which
+// leaves gelu(u) = u (1 - 3e-5) above and 3e-5 |u| below.
 __device__ __forceinline__ float gelu_fast(float u) {
-  return 0.5f * u * (1.0f + erf_poly(u * 0.70710678118654752f));
+  const float c = fminf(fmaxf(u, -4.0f), 4.0f);
+  const float t = c * c;
+  float q = 8.093845117e-11f;
+  q = fmaf(q, t, -7.032516570e-09f);
+  q = fmaf(q, t, 2.727248615e-07f);
+  q = fmaf(q, t, -6.317188128e-06f);
+  q = fmaf(q, t, 9.916073864e-05f);
+  q = fmaf(q, t, -1.135572678e-03f);
+  q = fmaf(q, t, 9.883344319e-03f);
+  q = fmaf(q, t, -6.642043264e-02f);
+  q = fmaf(q, t, 3.989280708e-01f);
+  return u * fmaf(q, c, 0.5f);
 }
 // GELU'(u) = Phi(u) + u phi(u), also on the FMA pipe: 0.5 + u * P(u^2) with a degree-17 odd
 // least-maximum-error fit on |u| <= 4 (absolute error below 1e-4); beyond that the derivative is
@@ -631,8 +628,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const long long off = off0 + n0;
         const bool fullv = p.vec_ok && (n0 + 32 <= p.N);
         const bool row_ok = m < p.M;
+        if (p.alpha != 1.0f) {
 #pragma unroll
-        for (int j = 0; j < 32; j++) v[j] *= p.alpha;
+          for (int j = 0; j < 32; j++) v[j] *= p.alpha;
+        }
         if (p.bias) {
           if (n0 + 32 <= p.N) {
 #pragma unroll
