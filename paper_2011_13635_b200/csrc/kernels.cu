@@ -559,6 +559,96 @@ cross_entropy_kernel(const float* __restrict__ logits, int64_t ldl, const int* _
   }
 }
 
+// The same for rows of up to 32768 logits, with the whole row held in the registers of a
+// 1024-thread block: the logits are read from HBM exactly once (eight independent 16-byte loads
+// per thread keep 128 KB in flight per SM) and one exponential per element is evaluated.
+constexpr int CE_REG_V4 = 8;  // float4 per thread
+
+template <typename T>
+__global__ void __launch_bounds__(1024)
+cross_entropy_regs_kernel(const float* __restrict__ logits, int64_t ldl, const int* __restrict__ rowlabel,
+                          const float* __restrict__ inv_n, T* __restrict__ dlogits, int64_t ldd,
+                          float* __restrict__ nll, int V) {
+  __shared__ float red[32];
+  __shared__ float bcast;
+  const int r = blockIdx.x, tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int label = rowlabel[r];
+  const float* lr = logits + (int64_t)r * ldl;
+  T* dr = dlogits ? dlogits + (int64_t)r * ldd : nullptr;
+  if (label < 0) {
+    if (tid == 0) nll[r] = 0.f;
+    if (dr != nullptr)
+      for (int64_t c = (int64_t)tid * 4; c < ldd; c += 1024 * 4) {
+#pragma unroll
+        for (int e = 0; e < 4; e++) dr[c + e] = from_f<T>(0.f);
+      }
+    return;
+  }
+  float x[CE_REG_V4][4];
+  float m = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < CE_REG_V4; i++) {
+    const int c = (tid + i * 1024) * 4;
+    float4 v = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+    if (c < ldl) v = *reinterpret_cast<const float4*>(lr + c);
+    x[i][0] = c + 0 < V ? v.x : -INFINITY;
+    x[i][1] = c + 1 < V ? v.y : -INFINITY;
+    x[i][2] = c + 2 < V ? v.z : -INFINITY;
+    x[i][3] = c + 3 < V ? v.w : -INFINITY;
+  }
+#pragma unroll
+  for (int i = 0; i < CE_REG_V4; i++)
+#pragma unroll
+    for (int e = 0; e < 4; e++) m = fmaxf(m, x[i][e]);
+  m = warp_max(m);
+  if (lane == 0) red[warp] = m;
+  __syncthreads();
+  if (warp == 0) {
+    float t = warp_max(red[lane]);
+    if (lane == 0) bcast = t;
+  }
+  __syncthreads();
+  m = bcast;
+  float s = 0.f;
+#pragma unroll
+  for (int i = 0; i < CE_REG_V4; i++)
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      x[i][e] = expf(x[i][e] - m);  // exp(-inf) = 0 for the padding
+      s += x[i][e];
+    }
+  s = warp_sum(s);
+  __syncthreads();  // bcast and red are reused
+  if (lane == 0) red[warp] = s;
+  __syncthreads();
+  if (warp == 0) {
+    float t = warp_sum(red[lane]);
+    if (lane == 0) {
+      bcast = t;
+      nll[r] = m + logf(t) - lr[label];
+    }
+  }
+  __syncthreads();
+  if (dr == nullptr) return;
+  const float scale = (*inv_n) / bcast;
+  const float inv = *inv_n;
+#pragma unroll
+  for (int i = 0; i < CE_REG_V4; i++) {
+    const int c = (tid + i * 1024) * 4;
+    if (c < ldd) {
+      T o[4];
+#pragma unroll
+      for (int e = 0; e < 4; e++) {
+        const float g = c + e < V ? x[i][e] * scale - (c + e == label ? inv : 0.f) : 0.f;
+        o[e] = from_f<T>(g);
+      }
+      if (sizeof(T) == 4) *reinterpret_cast<float4*>(dr + c) = *reinterpret_cast<const float4*>(o);
+      else *reinterpret_cast<uint2*>(dr + c) = *reinterpret_cast<const uint2*>(o);
+    }
+  }
+}
+
 __global__ void loss_reduce_kernel(const float* __restrict__ nll, int R,
                                    const float* __restrict__ inv_n, float* __restrict__ loss) {
   __shared__ float part[32];
@@ -784,8 +874,12 @@ void launch_cross_entropy(bool bf, const float* logits, int64_t ldl, const int* 
                           const float* inv_n, void* dlogits, int64_t ldd, float* nll, int R, int V,
                           cudaStream_t st) {
   if (R <= 0) return;
-  DISPATCH_T(bf, (cross_entropy_kernel<T><<<R, 256, 0, st>>>(logits, ldl, rowlabel, inv_n,
-                                                            (T*)dlogits, ldd, nll, V)));
+  if (ldl <= CE_REG_V4 * 1024 * 4)
+    DISPATCH_T(bf, (cross_entropy_regs_kernel<T><<<R, 1024, 0, st>>>(logits, ldl, rowlabel, inv_n,
+                                                                     (T*)dlogits, ldd, nll, V)));
+  else
+    DISPATCH_T(bf, (cross_entropy_kernel<T><<<R, 256, 0, st>>>(logits, ldl, rowlabel, inv_n,
+                                                              (T*)dlogits, ldd, nll, V)));
 }
 
 void launch_loss_reduce(const float* nll, int R, const float* inv_n, float* loss, cudaStream_t st) {
