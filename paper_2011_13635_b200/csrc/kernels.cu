@@ -361,42 +361,65 @@ softmax_fwd_kernel(const T* __restrict__ sc, T* __restrict__ p, const int* __res
 }
 
 // ds = p * (dp - sum_j dp * p) * scale, written over dp
-template <typename T>
+// A group of LPR lanes (16 or 32) owns a row; each group handles two rows per pass so that four
+// 16-byte loads per lane are in flight before the first reduction.  NV = vectors per lane.
+template <typename T, int LPR, int NV>
 __global__ void __launch_bounds__(256)
 softmax_bwd_kernel(T* __restrict__ dp, const T* __restrict__ p, int rows, int S, float scale) {
   constexpr int VN = VecT<T>::N;
-  constexpr int NV = SM_MAXE / VN;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= rows) return;
-  float a[SM_MAXE], b[SM_MAXE];
-  float dot = 0.f;
+  typedef typename VecT<T>::Raw Raw;
+  constexpr int GPW = 32 / LPR;  // groups per warp
+  constexpr int RPG = 2;         // rows per group and pass
+  const int lane = threadIdx.x & 31, gl = lane % LPR;
+  const int group = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * GPW + lane / LPR;
+  const int row0 = group * RPG;
+  if (row0 >= rows) return;   // whole groups leave together; shuffles below stay inside a group
+  const unsigned gmask = LPR == 32 ? 0xffffffffu : (0xffffu << (16 * (lane / 16)));
+  Raw ra[RPG][NV], rb[RPG][NV];
 #pragma unroll
-  for (int i = 0; i < NV; i++) {
-    const int c = (lane + 32 * i) * VN;
-    if (c < S) {
-      float t[VN], u[VN];
-      VecT<T>::load(dp + (int64_t)row * S + c, t);
-      VecT<T>::load(p + (int64_t)row * S + c, u);
+  for (int r = 0; r < RPG; r++)
 #pragma unroll
-      for (int e = 0; e < VN; e++) {
-        a[i * VN + e] = t[e];
-        b[i * VN + e] = u[e];
-        dot += t[e] * u[e];
+    for (int i = 0; i < NV; i++) {
+      const int c = (gl + LPR * i) * VN;
+      if (c < S && row0 + r < rows) {
+        ra[r][i] = VecT<T>::load_raw(dp + (int64_t)(row0 + r) * S + c);
+        rb[r][i] = VecT<T>::load_raw(p + (int64_t)(row0 + r) * S + c);
       }
     }
-  }
-  dot = warp_sum(dot);
+  float dot[RPG];
 #pragma unroll
-  for (int i = 0; i < NV; i++) {
-    const int c = (lane + 32 * i) * VN;
-    if (c < S) {
-      float o[VN];
+  for (int r = 0; r < RPG; r++) {
+    float d = 0.f;
 #pragma unroll
-      for (int e = 0; e < VN; e++) o[e] = b[i * VN + e] * (a[i * VN + e] - dot) * scale;
-      VecT<T>::store(dp + (int64_t)row * S + c, o);
+    for (int i = 0; i < NV; i++) {
+      if ((gl + LPR * i) * VN < S && row0 + r < rows) {
+        float a[VN], b[VN];
+        VecT<T>::unpack(ra[r][i], a);
+        VecT<T>::unpack(rb[r][i], b);
+#pragma unroll
+        for (int e = 0; e < VN; e++) d += a[e] * b[e];
+      }
     }
+    dot[r] = d;
   }
+#pragma unroll
+  for (int r = 0; r < RPG; r++)
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) dot[r] += __shfl_xor_sync(gmask, dot[r], o);
+#pragma unroll
+  for (int r = 0; r < RPG; r++)
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (gl + LPR * i) * VN;
+      if (c < S && row0 + r < rows) {
+        float a[VN], b[VN], o[VN];
+        VecT<T>::unpack(ra[r][i], a);
+        VecT<T>::unpack(rb[r][i], b);
+#pragma unroll
+        for (int e = 0; e < VN; e++) o[e] = b[e] * (a[e] - dot[r]) * scale;
+        VecT<T>::store(dp + (int64_t)(row0 + r) * S + c, o);
+      }
+    }
 }
 
 // ---------------------------------------------------------------------------------------
@@ -847,8 +870,16 @@ void launch_softmax_fwd(bool bf, const void* sc, void* p, const int* seq_lens, i
 void launch_softmax_bwd(bool bf, void* dp, const void* p, int rows, int S, float scale,
                         cudaStream_t st) {
   if (rows <= 0) return;
-  DISPATCH_T(bf, (softmax_bwd_kernel<T><<<div_up(rows, 8), 256, 0, st>>>((T*)dp, (const T*)p, rows,
-                                                                        S, scale)));
+  const int vn = bf ? 8 : 4;
+  const int nvec = (S + vn - 1) / vn;  // 16-byte vectors per row
+#define SM_BWD(LPR, NV)                                                                        \
+  DISPATCH_T(bf, (softmax_bwd_kernel<T, LPR, NV><<<div_up(rows, 8 * (32 / LPR) * 2), 256, 0, st>>>( \
+                     (T*)dp, (const T*)p, rows, S, scale)))
+  if (nvec <= 16) SM_BWD(16, 1);
+  else if (nvec <= 32) SM_BWD(32, 1);
+  else if (nvec <= 64) SM_BWD(32, 2);
+  else SM_BWD(32, 4);
+#undef SM_BWD
 }
 
 void launch_slots_prepare(const int* positions, const int* labels, const int* seq_lens, int B,
