@@ -112,7 +112,9 @@ def describe(cfg: I.StageConfig) -> dict:
                          f"{cfg.vocab}, seq {cfg.seq}, batch {cfg.batch} per GPU, {cfg.pred} MLM slots",
                 batch_per_gpu=cfg.batch, seq_len=cfg.seq, layers=cfg.layers, frozen=cfg.frozen,
                 trainable=cfg.trainable, parallelism="replicas only (no collective)",
-                l2="working set of one step (GBs of weights and activations) exceeds the 126 MB L2")
+                l2="working set of one step (GBs of weights and activations) exceeds the 126 MB L2",
+                launch="timed steps are replays of one mslt_step captured in a CUDA graph "
+                       "(--no-graph launches them one by one)")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -166,28 +168,45 @@ def run_reference(args, cfg):
 # ------------------------------------------------------------------------------------------------
 # our arm
 # ------------------------------------------------------------------------------------------------
-def make_model(cfg, torch):
+def make_model(cfg, torch, stream=None):
     from paper_2011_13635_b200.binding import Mslt
-    m = Mslt.from_config(cfg)
+    m = Mslt.from_config(cfg, stream=stream)
     m.set_params(I.make_weights(cfg, variant="bench"))
     m.mslt_set_trainable(cfg.trainable)
     m.mslt_set_optimizer(**I.ADAM_DEFAULTS)
     return m
 
 
-def time_steps(m, dev, torch, steps, warmup, sync_fn):
-    tok, lens, pos, lab = dev
-    for _ in range(warmup):
-        m.mslt_step(tok, lens, pos, lab, sync=False)
-    sync_fn()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+def capture_step(m, dev, torch):
+    """One mslt_step captured into a CUDA graph on the context's stream (after eager warm-up)."""
+    g = torch.cuda.CUDAGraph()
     before = m.launch_count
-    e0.record()
-    for _ in range(steps):
-        m.mslt_step(tok, lens, pos, lab, sync=False)
-    e1.record()
-    sync_fn()
-    return e0.elapsed_time(e1), m.launch_count - before
+    with torch.cuda.graph(g, stream=m.stream):
+        m.mslt_step(*dev, sync=False)
+    return g, m.launch_count - before
+
+
+def time_steps(m, dev, torch, steps, warmup, sync_fn, use_graph=True):
+    """(ms of the timed region, kernels launched in it).  The timed steps are replays of one
+    captured step unless use_graph is off; events are recorded on the context's stream."""
+    with torch.cuda.stream(m.stream):
+        for _ in range(warmup):
+            m.mslt_step(*dev, sync=False)
+        sync_fn()
+        graph, per_step = capture_step(m, dev, torch) if use_graph else (None, None)
+        sync_fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        before = m.launch_count
+        e0.record(m.stream)
+        for _ in range(steps):
+            if graph is not None:
+                graph.replay()
+            else:
+                m.mslt_step(*dev, sync=False)
+        e1.record(m.stream)
+        sync_fn()
+    launches = per_step * steps if graph is not None else m.launch_count - before
+    return e0.elapsed_time(e1), launches, graph
 
 
 def rank_seed(cfg, rank: int) -> int:
@@ -226,30 +245,40 @@ def run_ours(args, cfg):
     if cfg.varlen is None:
         host[1] = None
     pinned = [None if a is None else torch.from_numpy(a).pin_memory() for a in host]
-    dev = [None if a is None else a.cuda(non_blocking=True) for a in pinned]
-    m = make_model(cfg, torch)
-    loss0 = m.mslt_step(*dev)                       # also checks the device status word
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        dev = [None if a is None else a.cuda(non_blocking=True) for a in pinned]
+        m = make_model(cfg, torch, stream)
+        loss0 = m.mslt_step(*dev)                       # also checks the device status word
     if not np.isfinite(loss0):
         raise RuntimeError("non-finite loss")
 
     with ClockSampler(local) as clk:
-        ms, launches = time_steps(m, dev, torch, args.steps, args.warmup, sync)
+        ms, launches, graph = time_steps(m, dev, torch, args.steps, args.warmup, sync, args.graph)
     loss_end = m.mslt_read_loss()
     ms, value = aggregate(ms, cfg.batch, args.steps, world, dist, "cuda")
 
     # end to end: pinned host inputs copied in, loss read back, every step
     sync()
-    t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-    t0.record()
-    for _ in range(args.steps):
-        d = [None if a is None else a.cuda(non_blocking=True) for a in pinned]
-        m.mslt_step(*d)
-    t1.record()
-    sync()
+    with torch.cuda.stream(stream):
+        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+        t0.record(stream)
+        for _ in range(args.steps):
+            for d_, p_ in zip(dev, pinned):
+                if d_ is not None:
+                    d_.copy_(p_, non_blocking=True)
+            if graph is not None:
+                graph.replay()
+                m.mslt_read_loss()
+            else:
+                m.mslt_step(*dev)
+        t1.record(stream)
+        sync()
     _, e2e_value = aggregate(t0.elapsed_time(t1), cfg.batch, args.steps, world, dist, "cuda")
     e2e = dict(value=e2e_value, unit=UNIT,
                h2d_bytes_per_step=int(sum(a.nbytes for a in host if a is not None)),
                d2h_bytes_per_step=16)
+    del graph
 
     line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
                 warmup=args.warmup, ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak",
@@ -263,8 +292,9 @@ def run_ours(args, cfg):
         m.mslt_set_timing(2)
         m.mslt_get_kernel_profile()
         n_prof = max(1, min(args.steps, 5))
-        for _ in range(n_prof):
-            m.mslt_step(*dev, sync=False)
+        with torch.cuda.stream(stream):
+            for _ in range(n_prof):
+                m.mslt_step(*dev, sync=False)
         torch.cuda.synchronize()
         prof = m.mslt_get_kernel_profile()
         phases = m.mslt_get_timings()
@@ -298,9 +328,10 @@ def run_ours(args, cfg):
         torch.cuda.empty_cache()
         if world == 1 and args.ratio and cfg.name == "base_stage":
             full = I.CONFIGS["base_full"]
-            mf = make_model(full, torch)
+            mf = make_model(full, torch, stream)
             k = max(3, min(args.steps, 10))
-            ms_f, _ = time_steps(mf, dev, torch, k, 3, sync)
+            ms_f, _, gf = time_steps(mf, dev, torch, k, 3, sync, args.graph)
+            del gf
             line["stage_vs_full"] = dict(
                 staged_ms=ms / args.steps, full_ms=ms_f / k, ratio=(ms / args.steps) / (ms_f / k),
                 note="step time of 9 frozen + 3 trainable layers over all 12 trainable, same shapes, "
@@ -324,6 +355,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seqs", type=int, default=8, help="sequences in the oracle's timed sample")
     ap.add_argument("--no-ratio", dest="ratio", action="store_false")
+    ap.add_argument("--no-graph", dest="graph", action="store_false",
+                    help="launch every timed step eagerly instead of replaying one captured step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = I.CONFIGS[args.config]

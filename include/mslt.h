@@ -119,7 +119,10 @@ int mslt_set_optimizer(mslt_ctx* ctx, const mslt_opt* opt);
  *   loss_out        host float or NULL.  Non-NULL: the stream is synchronised and the loss
  *                   and the device status word are read back (an out-of-range index or a
  *                   kernel wait that ran out gives MSLT_ERR_DEVICE).  NULL: nothing is
- *                   synchronised; use mslt_read_loss later.
+ *                   synchronised; use mslt_read_loss later.  In this form the call only enqueues
+ *                   kernels and memsets on the context's stream (the Adam step count lives in
+ *                   device memory), so after one ordinary step it may be captured into a CUDA
+ *                   graph by the caller and replayed on the same buffers.
  */
 int mslt_step(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens,
               const int32_t* d_mlm_positions, const int32_t* d_mlm_labels, int32_t B, int32_t S,

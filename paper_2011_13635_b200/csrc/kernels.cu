@@ -752,10 +752,22 @@ __global__ void embed_scatter_kernel(const T* __restrict__ dz, const int* __rest
 // ---------------------------------------------------------------------------------------
 // Adam with decoupled weight decay over a table of chunks of the trainable slice.
 // ---------------------------------------------------------------------------------------
+// Advances the step count kept in device memory and forms the bias corrections 1 / (1 - beta^t)
+// there, so that a captured step (CUDA graph) replays with the right values.
+__global__ void adam_tick_kernel(int* __restrict__ t, float* __restrict__ bc, float beta1, float beta2,
+                                 int bias_correction) {
+  const int n = *t + 1;
+  *t = n;
+  bc[0] = bias_correction ? (float)(1.0 / (1.0 - pow((double)beta1, (double)n))) : 1.f;
+  bc[1] = bias_correction ? (float)(1.0 / (1.0 - pow((double)beta2, (double)n))) : 1.f;
+}
+
 __global__ void __launch_bounds__(256)
 adam_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ w,
             const float* __restrict__ g, float* __restrict__ m, float* __restrict__ v,
-            bf16* __restrict__ wb, AdamHyper h) {
+            bf16* __restrict__ wb, AdamHyper h, const float* __restrict__ bc) {
+  h.bc1 = bc[0];
+  h.bc2 = bc[1];
   const AdamChunk ch = chunks[blockIdx.x];
   const float decay = h.weight_decay * ch.decay;
   for (int i = threadIdx.x * 4; i < ch.count; i += 256 * 4) {
@@ -936,9 +948,11 @@ void launch_embed_scatter(bool bf, const void* dz, const int* tokens, float* dwo
 }
 
 void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,
-                 void* wb, const AdamHyper& h, cudaStream_t st) {
+                 void* wb, const AdamHyper& h, int* t_dev, float* bc_dev, int bias_correction,
+                 cudaStream_t st) {
+  adam_tick_kernel<<<1, 1, 0, st>>>(t_dev, bc_dev, h.beta1, h.beta2, bias_correction);
   if (n_chunks <= 0) return;
-  adam_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, g, m, v, (bf16*)wb, h);
+  adam_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, g, m, v, (bf16*)wb, h, bc_dev);
 }
 
 void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st) {

@@ -15,7 +15,7 @@ struct AdamChunk {
 struct AdamHyper {
   float lr, beta1, beta2, eps, weight_decay;
   float omb1, omb2;  // 1 - beta, formed in double on the host
-  float bc1, bc2;    // bias corrections 1 / (1 - beta^t), or 1
+  float bc1, bc2;    // bias corrections 1 / (1 - beta^t), or 1: filled on the device
 };
 
 void launch_ln_fwd(bool bf, const void* z, const float* gamma, const float* beta, void* y,
@@ -46,8 +46,11 @@ void launch_colsum(bool bf, const void* x, int64_t ld, int rows, int N, float* o
                    cudaStream_t st);
 void launch_embed_scatter(bool bf, const void* dz, const int* tokens, float* dword, float* dpos,
                           int rows, int S, int H, int V, cudaStream_t st);
+// t_dev: step count in device memory (incremented here); bc_dev: two floats that receive the bias
+// corrections of this step
 void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,
-                 void* wb, const AdamHyper& h, cudaStream_t st);
+                 void* wb, const AdamHyper& h, int* t_dev, float* bc_dev, int bias_correction,
+                 cudaStream_t st);
 // d[i] *= gelu'(u[i]); n a multiple of the vector width
 void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st);
 void launch_f32_to_bf16(const float* src, void* dst, int64_t n, cudaStream_t st);

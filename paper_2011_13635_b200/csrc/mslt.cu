@@ -68,7 +68,8 @@ struct LayerBuf {
 
 struct Workspace {
   size_t bytes = 0;
-  int* scalars;  // [0] status, [1] n_valid, [2] inv_n (float), [3] loss (float)
+  int* scalars;  // [0] status, [1] n_valid, [2] inv_n (float), [3] loss (float), [4] Adam step count,
+                 // [5], [6] Adam bias corrections (float)
   int *rowsrc, *rowlabel;
   AdamChunk* chunks;
   int64_t max_chunks;
@@ -265,12 +266,18 @@ int rebuild_chunks(mslt_ctx* c) {
   c->n_chunks = (int)h.size();
   CUDA_TRY(cudaStreamSynchronize(c->st));
   if (!h.empty())
-    CUDA_TRY(cudaMemcpy(c->ws.chunks, h.data(), h.size() * sizeof(AdamChunk), cudaMemcpyHostToDevice));
+  {
+    // In-stream copy, then wait: a plain cudaMemcpy from pageable memory may return while its DMA is
+    // still in flight, and a non-blocking stream does not wait for it.
+    CUDA_TRY(cudaMemcpyAsync(c->ws.chunks, h.data(), h.size() * sizeof(AdamChunk), cudaMemcpyHostToDevice, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+  }
   return 0;
 }
 
 int reset_optimizer(mslt_ctx* c) {
   c->t_step = 0;
+  CUDA_TRY(cudaMemsetAsync(c->ws.scalars + 4, 0, 12, c->st));
   CUDA_TRY(cudaMemsetAsync(c->m, 0, c->n_elems * 4, c->st));
   CUDA_TRY(cudaMemsetAsync(c->v, 0, c->n_elems * 4, c->st));
   return rebuild_chunks(c);
@@ -544,7 +551,8 @@ int finish(mslt_ctx* c, float* loss_out) {
   if (!loss_out) return 0;
   int h[4];
   CUDA_TRY(cudaStreamSynchronize(c->st));
-  CUDA_TRY(cudaMemcpy(h, c->ws.scalars, 16, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpyAsync(h, c->ws.scalars, 16, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(cudaStreamSynchronize(c->st));
   memcpy(loss_out, &h[3], 4);
   if (h[0] != 0)
     return fail(MSLT_ERR_DEVICE, "device status 0x%x (1: kernel wait ran out, 2: token id, 4: MLM "
@@ -739,9 +747,9 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   h.weight_decay = c->opt.weight_decay;
   h.omb1 = (float)(1.0 - (double)c->opt.beta1);
   h.omb2 = (float)(1.0 - (double)c->opt.beta2);
-  h.bc1 = c->opt.bias_correction ? (float)(1.0 / (1.0 - pow((double)c->opt.beta1, (double)c->t_step))) : 1.f;
-  h.bc2 = c->opt.bias_correction ? (float)(1.0 / (1.0 - pow((double)c->opt.beta2, (double)c->t_step))) : 1.f;
-  KL(PC_ADAM, 30.0 * c->n_chunks * kAdamChunk, launch_adam(w.chunks, c->n_chunks, c->master, c->grad, c->m, c->v, c->wb, h, c->st));
+  h.bc1 = h.bc2 = 1.f;  // formed on the device from the step count kept there
+  KL(PC_ADAM, 30.0 * c->n_chunks * kAdamChunk, launch_adam(w.chunks, c->n_chunks, c->master, c->grad, c->m, c->v, c->wb, h, w.scalars + 4,
+                 (float*)(w.scalars + 5), c->opt.bias_correction, c->st));
   mark(c, 5);
   if (c->timing && c->have_events) {
     CUDA_TRY(cudaEventSynchronize(c->ev[5]));
@@ -839,7 +847,8 @@ int mslt_get_param(mslt_ctx* c, const char* name, float* dst, size_t n) {
   TRY(lookup(c, name, n, &t));
   if (!dst) return fail(MSLT_ERR_ARG, "null pointer");
   CUDA_TRY(cudaStreamSynchronize(c->st));
-  CUDA_TRY(cudaMemcpy(dst, c->master + t->offset, n * 4, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpyAsync(dst, c->master + t->offset, n * 4, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(cudaStreamSynchronize(c->st));
   return 0;
 }
 
@@ -848,7 +857,10 @@ int mslt_set_param(mslt_ctx* c, const char* name, const float* src, size_t n) {
   TRY(lookup(c, name, n, &t));
   if (!src) return fail(MSLT_ERR_ARG, "null pointer");
   CUDA_TRY(cudaStreamSynchronize(c->st));
-  CUDA_TRY(cudaMemcpy(c->master + t->offset, src, n * 4, cudaMemcpyHostToDevice));
+  // in the context's stream, so that the conversion kernel below is ordered after the copy even
+  // when that stream does not synchronise with the default stream
+  CUDA_TRY(cudaMemcpyAsync(c->master + t->offset, src, n * 4, cudaMemcpyHostToDevice, c->st));
+  CUDA_TRY(cudaStreamSynchronize(c->st));
   if (c->bf) {
     KL(PC_OTHER, 6.0 * n, launch_f32_to_bf16(c->master + t->offset, c->wb + t->offset * 2, (int64_t)n, c->st));
     CUDA_TRY(cudaStreamSynchronize(c->st));
@@ -865,7 +877,8 @@ int mslt_get_param_raw(mslt_ctx* c, const char* name, void* dst, size_t bytes) {
   if (bytes != want) return fail(MSLT_ERR_ARG, "tensor '%s' needs %zu raw bytes, got %zu", name, want, bytes);
   CUDA_TRY(cudaStreamSynchronize(c->st));
   const void* src = b ? (const void*)(c->wb + t->offset * 2) : (const void*)(c->master + t->offset);
-  CUDA_TRY(cudaMemcpy(dst, src, bytes, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(cudaStreamSynchronize(c->st));
   return 0;
 }
 
@@ -875,7 +888,8 @@ int mslt_get_grad(mslt_ctx* c, const char* name, float* dst, size_t n) {
   if (!dst) return fail(MSLT_ERR_ARG, "null pointer");
   if (!is_trainable(c, *t)) return fail(MSLT_ERR_STATE, "tensor '%s' is frozen: it has no gradient", name);
   CUDA_TRY(cudaStreamSynchronize(c->st));
-  CUDA_TRY(cudaMemcpy(dst, c->grad + t->offset, n * 4, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpyAsync(dst, c->grad + t->offset, n * 4, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(cudaStreamSynchronize(c->st));
   return 0;
 }
 
@@ -885,7 +899,8 @@ int mslt_get_opt_state(mslt_ctx* c, const char* name, int32_t which, float* dst,
   if (!dst || which < 0 || which > 1) return fail(MSLT_ERR_ARG, "bad argument");
   if (!is_trainable(c, *t)) return fail(MSLT_ERR_STATE, "tensor '%s' is frozen: it has no optimizer state", name);
   CUDA_TRY(cudaStreamSynchronize(c->st));
-  CUDA_TRY(cudaMemcpy(dst, (which ? c->v : c->m) + t->offset, n * 4, cudaMemcpyDeviceToHost));
+  CUDA_TRY(cudaMemcpyAsync(dst, (which ? c->v : c->m) + t->offset, n * 4, cudaMemcpyDeviceToHost, c->st));
+  CUDA_TRY(cudaStreamSynchronize(c->st));
   return 0;
 }
 
@@ -946,7 +961,8 @@ int mslt_op_gemm(const mslt_gemm_desc* d, void* cuda_stream, int32_t* d_status) 
   CUDA_TRY(cudaStreamSynchronize(st));
   if (d_status) {
     int h = 0;
-    CUDA_TRY(cudaMemcpy(&h, d_status, 4, cudaMemcpyDeviceToHost));
+    CUDA_TRY(cudaMemcpyAsync(&h, d_status, 4, cudaMemcpyDeviceToHost, st));
+    CUDA_TRY(cudaStreamSynchronize(st));
     if (h) return fail(MSLT_ERR_DEVICE, "device status 0x%x: a kernel wait ran out", h);
   }
   return 0;

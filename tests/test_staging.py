@@ -152,3 +152,37 @@ def test_error_paths_return_codes():
     assert m.mslt_step(d_tok, None, d_pos, none) == 0.0
     assert not m.mslt_get_grad("head.transform.weight").any()
     m.close()
+
+
+def test_captured_step_replays_like_eager_steps():
+    """mslt_step without loss read-back only enqueues work, so it can be captured in a CUDA graph:
+    replays advance Adam's step count on the device and match eagerly launched steps."""
+    import torch
+    cfg = CFG16
+    tok, lens, pos, lab = I.make_batch(cfg)
+    res = []
+    for use_graph in (False, True):
+        stream = torch.cuda.Stream()
+        with torch.cuda.stream(stream):
+            from paper_2011_13635_b200.binding import Mslt
+            m = Mslt.from_config(cfg, stream=stream)
+            m.set_params(I.make_weights(cfg, variant="parity"))
+            m.mslt_set_trainable(cfg.trainable)
+            m.mslt_set_optimizer(lr=1e-3)
+            d = PT.to_cuda(torch, tok, pos, lab)
+            m.mslt_step(d[0], None, d[1], d[2])                 # step 1, eager on both sides
+            if use_graph:
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=stream):
+                    m.mslt_step(d[0], None, d[1], d[2], sync=False)
+                g.replay(); g.replay()                          # steps 2 and 3 (capture runs nothing)
+            else:
+                for _ in range(2):
+                    m.mslt_step(d[0], None, d[1], d[2], sync=False)
+            loss = m.mslt_read_loss()
+            res.append((loss, m.mslt_get_param("layer.3.ffn1.weight"), m.mslt_get_opt_state("head.ln.gamma", 1)))
+            m.close()
+    (l0, w0, v0), (l1, w1, v1) = res
+    assert abs(l0 - l1) < 1e-3 * abs(l0)
+    assert PT.max_rel(w1, w0) < 1e-3                            # atomics reorder sums, nothing more
+    assert PT.max_rel(v1, v0) < 1e-2
