@@ -304,58 +304,86 @@ ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z, const float* __
 // ---------------------------------------------------------------------------------------
 // Scaled masked softmax over the last axis of [rows, S]; key j valid iff j < len(sequence).
 // ---------------------------------------------------------------------------------------
-constexpr int SM_MAXE = 16;  // S <= 512
-
-template <typename T>
+// A group of LPR lanes (16 or 32) owns a row and handles two rows per pass, so that several 16-byte
+// loads per lane are in flight before the first reduction.  NV = vectors per lane.
+template <typename T, int LPR, int NV>
 __global__ void __launch_bounds__(256)
 softmax_fwd_kernel(const T* __restrict__ sc, T* __restrict__ p, const int* __restrict__ seq_lens,
                    int rows, int S, int rows_per_seq, float scale) {
   constexpr int VN = VecT<T>::N;
-  constexpr int NV = SM_MAXE / VN;
-  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const int lane = threadIdx.x & 31;
-  if (row >= rows) return;
-  int len = seq_lens ? seq_lens[row / rows_per_seq] : S;
-  len = min(max(len, 1), S);
-  float x[SM_MAXE];
-  float mx = -INFINITY;
+  typedef typename VecT<T>::Raw Raw;
+  constexpr int GPW = 32 / LPR;
+  constexpr int RPG = 2;
+  const int lane = threadIdx.x & 31, gl = lane % LPR;
+  const int group = (blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5)) * GPW + lane / LPR;
+  const int row0 = group * RPG;
+  if (row0 >= rows) return;   // whole groups leave together; shuffles below stay inside a group
+  const unsigned gmask = LPR == 32 ? 0xffffffffu : (0xffffu << (16 * (lane / 16)));
+  Raw raw[RPG][NV];
+  int len[RPG];
 #pragma unroll
-  for (int i = 0; i < NV; i++) {
-    const int c = (lane + 32 * i) * VN;
-    if (c < S) {
-      float t[VN];
-      VecT<T>::load(sc + (int64_t)row * S + c, t);
+  for (int r = 0; r < RPG; r++) {
+    const int row = min(row0 + r, rows - 1);
+    const int l = seq_lens ? seq_lens[row / rows_per_seq] : S;
+    len[r] = min(max(l, 1), S);
 #pragma unroll
-      for (int e = 0; e < VN; e++) {
-        const float v = (c + e < len) ? t[e] * scale : -INFINITY;
-        x[i * VN + e] = v;
-        mx = fmaxf(mx, v);
-      }
+    for (int i = 0; i < NV; i++) {
+      const int c = (gl + LPR * i) * VN;
+      if (c < S && row0 + r < rows) raw[r][i] = VecT<T>::load_raw(sc + (int64_t)(row0 + r) * S + c);
     }
   }
-  mx = warp_max(mx);
-  float s = 0.f;
+  float x[RPG][NV][VN];
+  float mx[RPG], sum[RPG];
 #pragma unroll
-  for (int i = 0; i < NV; i++) {
-    const int c = (lane + 32 * i) * VN;
-    if (c < S) {
+  for (int r = 0; r < RPG; r++) {
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (gl + LPR * i) * VN;
+      float t[VN];
+      if (c < S && row0 + r < rows) VecT<T>::unpack(raw[r][i], t);
 #pragma unroll
       for (int e = 0; e < VN; e++) {
-        const float v = (c + e < len) ? expf(x[i * VN + e] - mx) : 0.f;
-        x[i * VN + e] = v;
+        const float v = (c + e < len[r] && row0 + r < rows) ? t[e] * scale : -INFINITY;
+        x[r][i][e] = v;
+        m = fmaxf(m, v);
+      }
+    }
+    mx[r] = m;
+  }
+#pragma unroll
+  for (int r = 0; r < RPG; r++)
+#pragma unroll
+    for (int o = LPR / 2; o > 0; o >>= 1) mx[r] = fmaxf(mx[r], __shfl_xor_sync(gmask, mx[r], o));
+#pragma unroll
+  for (int r = 0; r < RPG; r++) {
+    float s = 0.f;
+#pragma unroll
+    for (int i = 0; i < NV; i++)
+#pragma unroll
+      for (int e = 0; e < VN; e++) {
+        const float v = x[r][i][e] == -INFINITY ? 0.f : expf(x[r][i][e] - mx[r]);
+        x[r][i][e] = v;
         s += v;
       }
-    }
+    sum[r] = s;
   }
-  const float inv = 1.0f / warp_sum(s);
 #pragma unroll
-  for (int i = 0; i < NV; i++) {
-    const int c = (lane + 32 * i) * VN;
-    if (c < S) {
-      float o[VN];
+  for (int r = 0; r < RPG; r++)
 #pragma unroll
-      for (int e = 0; e < VN; e++) o[e] = x[i * VN + e] * inv;
-      VecT<T>::store(p + (int64_t)row * S + c, o);
+    for (int o = LPR / 2; o > 0; o >>= 1) sum[r] += __shfl_xor_sync(gmask, sum[r], o);
+#pragma unroll
+  for (int r = 0; r < RPG; r++) {
+    const float inv = 1.0f / sum[r];
+#pragma unroll
+    for (int i = 0; i < NV; i++) {
+      const int c = (gl + LPR * i) * VN;
+      if (c < S && row0 + r < rows) {
+        float o[VN];
+#pragma unroll
+        for (int e = 0; e < VN; e++) o[e] = x[r][i][e] * inv;
+        VecT<T>::store(p + (int64_t)(row0 + r) * S + c, o);
+      }
     }
   }
 }
@@ -875,8 +903,16 @@ void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, c
 void launch_softmax_fwd(bool bf, const void* sc, void* p, const int* seq_lens, int rows, int S,
                         int rows_per_seq, float scale, cudaStream_t st) {
   if (rows <= 0) return;
-  DISPATCH_T(bf, (softmax_fwd_kernel<T><<<div_up(rows, 8), 256, 0, st>>>(
-                     (const T*)sc, (T*)p, seq_lens, rows, S, rows_per_seq, scale)));
+  const int vn = bf ? 8 : 4;
+  const int nvec = (S + vn - 1) / vn;  // 16-byte vectors per row
+#define SM_FWD(LPR, NV)                                                                        \
+  DISPATCH_T(bf, (softmax_fwd_kernel<T, LPR, NV><<<div_up(rows, 8 * (32 / LPR) * 2), 256, 0, st>>>( \
+                     (const T*)sc, (T*)p, seq_lens, rows, S, rows_per_seq, scale)))
+  if (nvec <= 16) SM_FWD(16, 1);
+  else if (nvec <= 32) SM_FWD(32, 1);
+  else if (nvec <= 64) SM_FWD(32, 2);
+  else SM_FWD(32, 4);
+#undef SM_FWD
 }
 
 void launch_softmax_bwd(bool bf, void* dp, const void* p, int rows, int S, float scale,
