@@ -235,6 +235,36 @@ int mslt_op_cross_entropy(int32_t dtype, const float* d_logits, int64_t ldl, con
                           void* d_scratch, size_t scratch_bytes, void* cuda_stream);
 
 /*
+ * The fused memory-bound kernels of the step one at a time, for per-kernel tests and bandwidth
+ * measurements.  dtype 0: rows of float, dtype 1: rows of bf16; statistics, gains, biases and
+ * column sums are fp32.  All pointers are device pointers, rows are contiguous (row length a
+ * multiple of 8; rows 16-byte aligned).  sync != 0 synchronises the stream before returning.
+ *
+ * LayerNorm of the encoder (post-LN BERT, Section 4.1): y = gamma * (z - mean) / sqrt(var + eps) +
+ * beta over rows of H <= 1024 elements, biased variance; d_stats (may be NULL) receives
+ * {mean, 1/sqrt(var + eps)} per row.  The backward call takes those statistics and returns dz and
+ * ADDS the column sums dgamma += sum dy * xhat, dbeta += sum dy (the caller zeroes them).
+ */
+int mslt_op_layernorm(int32_t dtype, const void* d_z, const float* d_gamma, const float* d_beta, void* d_y,
+                      float* d_stats, int32_t rows, int32_t H, float eps, void* cuda_stream, int32_t sync);
+int mslt_op_layernorm_bwd(int32_t dtype, const void* d_dy, const void* d_z, const float* d_stats,
+                          const float* d_gamma, void* d_dz, float* d_dgamma, float* d_dbeta, int32_t rows,
+                          int32_t H, void* cuda_stream, int32_t sync);
+/* Scaled masked softmax of attention over rows of S <= 512 scores: row r belongs to sequence
+ * r / rows_per_seq; key j is valid iff j < d_seq_lens[sequence] (NULL: all valid); masked
+ * probabilities are exactly 0.  May run in place.  The backward call overwrites dp with
+ * p * (dp - sum_j dp * p) * scale. */
+int mslt_op_softmax(int32_t dtype, const void* d_scores, void* d_probs, const int32_t* d_seq_lens,
+                    int32_t rows, int32_t S, int32_t rows_per_seq, float scale, void* cuda_stream,
+                    int32_t sync);
+int mslt_op_softmax_bwd(int32_t dtype, void* d_dp, const void* d_probs, int32_t rows, int32_t S, float scale,
+                        void* cuda_stream, int32_t sync);
+/* Bias gradient: d_out[n] += sum over rows of x[row, n] (leading dimension ld, N a multiple of 8;
+ * fp32 atomic adds, order not fixed). */
+int mslt_op_colsum(int32_t dtype, const void* d_x, int64_t ld, int32_t rows, int32_t N, float* d_out,
+                   void* cuda_stream, int32_t sync);
+
+/*
  * mslt_op_cross_entropy without any device allocation by anybody.  (The paper has no counterpart
  * of this call; it exists for the integration below.)
  *

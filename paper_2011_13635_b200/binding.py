@@ -54,7 +54,8 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_kernel_profile",
            "mslt_last_error",
            "mslt_op_gemm", "mslt_op_gemm_enqueue", "mslt_op_cross_entropy",
-           "mslt_op_cross_entropy_scratch_bytes", "mslt_op_cross_entropy_noalloc"]
+           "mslt_op_cross_entropy_scratch_bytes", "mslt_op_cross_entropy_noalloc", "mslt_op_layernorm",
+           "mslt_op_layernorm_bwd", "mslt_op_softmax", "mslt_op_softmax_bwd", "mslt_op_colsum"]
 
 lib.mslt_last_error.restype = C.c_char_p
 lib.mslt_last_error.argtypes = [C.c_void_p]
@@ -97,6 +98,14 @@ lib.mslt_op_cross_entropy.argtypes = [C.c_int32, C.c_void_p, C.c_int64, C.c_void
 
 lib.mslt_op_cross_entropy_noalloc.argtypes = [C.c_int32, C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_int32,
                                               C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p]
+
+
+_P = C.c_void_p
+lib.mslt_op_layernorm.argtypes = [C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
+lib.mslt_op_layernorm_bwd.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, _P, C.c_int32]
+lib.mslt_op_softmax.argtypes = [C.c_int32, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
+lib.mslt_op_softmax_bwd.argtypes = [C.c_int32, _P, _P, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
+lib.mslt_op_colsum.argtypes = [C.c_int32, _P, C.c_int64, C.c_int32, C.c_int32, _P, _P, C.c_int32]
 
 
 class MsltError(RuntimeError):
@@ -144,6 +153,42 @@ def mslt_op_cross_entropy_noalloc(dtype: int, logits, labels, V: int, dlogits, l
     _check(lib.mslt_op_cross_entropy_noalloc(dtype, logits.data_ptr(), logits.stride(0), labels.data_ptr(), R,
                                              V, _ptr(dlogits), 0 if dlogits is None else dlogits.stride(0),
                                              loss.data_ptr(), C.c_void_p(stream)))
+
+
+def _dt(t) -> int:
+    import torch
+    return 1 if t.dtype == torch.bfloat16 else 0
+
+
+def mslt_op_layernorm(z, gamma, beta, y, stats, eps: float, stream: int, sync: bool = True) -> None:
+    """z, y [rows, H] float or bf16; gamma, beta fp32 [H]; stats fp32 [rows, 2] or None: CUDA tensors."""
+    _check(lib.mslt_op_layernorm(_dt(z), z.data_ptr(), gamma.data_ptr(), beta.data_ptr(), y.data_ptr(),
+                                 _ptr(stats), z.shape[0], z.shape[1], eps, C.c_void_p(stream), int(sync)))
+
+
+def mslt_op_layernorm_bwd(dy, z, stats, gamma, dz, dgamma, dbeta, stream: int, sync: bool = True) -> None:
+    _check(lib.mslt_op_layernorm_bwd(_dt(z), dy.data_ptr(), z.data_ptr(), stats.data_ptr(), gamma.data_ptr(),
+                                     dz.data_ptr(), dgamma.data_ptr(), dbeta.data_ptr(), z.shape[0],
+                                     z.shape[1], C.c_void_p(stream), int(sync)))
+
+
+def mslt_op_softmax(scores, probs, seq_lens, rows_per_seq: int, scale: float, stream: int,
+                    sync: bool = True) -> None:
+    """scores, probs [rows, S] (may be the same tensor); seq_lens int32 [rows / rows_per_seq] or None."""
+    _check(lib.mslt_op_softmax(_dt(scores), scores.data_ptr(), probs.data_ptr(), _ptr(seq_lens),
+                               scores.shape[0], scores.shape[1], rows_per_seq, scale, C.c_void_p(stream),
+                               int(sync)))
+
+
+def mslt_op_softmax_bwd(dp, probs, scale: float, stream: int, sync: bool = True) -> None:
+    _check(lib.mslt_op_softmax_bwd(_dt(dp), dp.data_ptr(), probs.data_ptr(), dp.shape[0], dp.shape[1], scale,
+                                   C.c_void_p(stream), int(sync)))
+
+
+def mslt_op_colsum(x, n: int, out, stream: int, sync: bool = True) -> None:
+    """out[:n] += x[:, :n].sum(0); x [rows, ld] float or bf16, out fp32."""
+    _check(lib.mslt_op_colsum(_dt(x), x.data_ptr(), x.stride(0), x.shape[0], n, out.data_ptr(),
+                              C.c_void_p(stream), int(sync)))
 
 
 class Mslt:

@@ -90,26 +90,16 @@ ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ gamma, const fl
       const int c = (lane + 32 * i) * VN;
       if (c < H && row0 + r < rows) raw[r][i] = VecT<T>::load_raw(z + (int64_t)(row0 + r) * H + c);
     }
+  // One reduction round for both moments: sums of (x - x0) and (x - x0)^2 with x0 the first element
+  // of the row, which keeps the subtraction var = E[d^2] - E[d]^2 well conditioned (x0 lies within
+  // the spread of the row).
   float mean[ROWS], rstd[ROWS];
 #pragma unroll
   for (int r = 0; r < ROWS; r++) {
-    float s = 0.f;
-#pragma unroll
-    for (int i = 0; i < NV; i++) {
-      if ((lane + 32 * i) * VN < H && row0 + r < rows) {
-        float t[VN];
-        VecT<T>::unpack(raw[r][i], t);
-#pragma unroll
-        for (int e = 0; e < VN; e++) s += t[e];
-      }
-    }
-    mean[r] = s;
-  }
-#pragma unroll
-  for (int r = 0; r < ROWS; r++) mean[r] = warp_sum(mean[r]) / (float)H;
-#pragma unroll
-  for (int r = 0; r < ROWS; r++) {
-    float q = 0.f;
+    float first[VN];
+    VecT<T>::unpack(raw[r][0], first);
+    const float x0 = __shfl_sync(0xffffffffu, first[0], 0);
+    float s1 = 0.f, s2 = 0.f;
 #pragma unroll
     for (int i = 0; i < NV; i++) {
       if ((lane + 32 * i) * VN < H && row0 + r < rows) {
@@ -117,15 +107,33 @@ ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ gamma, const fl
         VecT<T>::unpack(raw[r][i], t);
 #pragma unroll
         for (int e = 0; e < VN; e++) {
-          const float d = t[e] - mean[r];
-          q += d * d;
+          const float d = t[e] - x0;
+          s1 += d;
+          s2 = fmaf(d, d, s2);
         }
       }
     }
-    rstd[r] = q;
+    mean[r] = s1;
+    rstd[r] = s2;
   }
 #pragma unroll
-  for (int r = 0; r < ROWS; r++) rstd[r] = rsqrtf(warp_sum(rstd[r]) / (float)H + eps);
+  for (int o = 16; o > 0; o >>= 1) {
+#pragma unroll
+    for (int r = 0; r < ROWS; r++) {
+      mean[r] += __shfl_xor_sync(0xffffffffu, mean[r], o);
+      rstd[r] += __shfl_xor_sync(0xffffffffu, rstd[r], o);
+    }
+  }
+#pragma unroll
+  for (int r = 0; r < ROWS; r++) {
+    float first[VN];
+    VecT<T>::unpack(raw[r][0], first);
+    const float x0 = __shfl_sync(0xffffffffu, first[0], 0);
+    const float m1 = mean[r] / (float)H;
+    const float var = fmaxf(rstd[r] / (float)H - m1 * m1, 0.f);
+    mean[r] = x0 + m1;
+    rstd[r] = rsqrtf(var + eps);
+  }
   if (stats != nullptr && lane == 0) {
 #pragma unroll
     for (int r = 0; r < ROWS; r++)
@@ -362,7 +370,7 @@ softmax_fwd_kernel(const T* __restrict__ sc, T* __restrict__ p, const int* __res
     for (int i = 0; i < NV; i++)
 #pragma unroll
       for (int e = 0; e < VN; e++) {
-        const float v = x[r][i][e] == -INFINITY ? 0.f : expf(x[r][i][e] - mx[r]);
+        const float v = x[r][i][e] == -INFINITY ? 0.f : __expf(x[r][i][e] - mx[r]);
         x[r][i][e] = v;
         s += v;
       }
@@ -863,12 +871,12 @@ void launch_ln_fwd(bool bf, const void* z, const float* gamma, const float* beta
   const int vn = bf ? 8 : 4;
   const int nv = (H + 32 * vn - 1) / (32 * vn);
 #define LN_FWD(NV, ROWS)                                                                             \
-  DISPATCH_T(bf, (ln_fwd_kernel<T, NV, ROWS><<<div_up(rows, 8 * ROWS), 256, 0, st>>>(                  \
+  DISPATCH_T(bf, (ln_fwd_kernel<T, NV, ROWS><<<div_up(rows, 4 * ROWS), 128, 0, st>>>(                  \
                      (const T*)z, gamma, beta, (T*)y, stats, rows, H, eps)))
   if (nv <= 1) LN_FWD(1, 4);
-  else if (nv <= 2) LN_FWD(2, 4);
-  else if (nv <= 3) LN_FWD(3, 4);
-  else if (nv <= 4) LN_FWD(4, 4);
+  else if (nv <= 2) LN_FWD(2, 2);
+  else if (nv <= 3) LN_FWD(3, 2);
+  else if (nv <= 4) LN_FWD(4, 2);
   else if (nv <= 6) LN_FWD(6, 2);
   else LN_FWD(8, 2);
 #undef LN_FWD

@@ -82,6 +82,24 @@ int run_ce(int dtype, const float* logits, int64_t ldl, const int32_t* labels, i
   return 0;
 }
 
+int finish_op(const char* what, cudaStream_t st, int sync) {
+  cudaError_t e = cudaGetLastError();
+  if (e == cudaSuccess && sync) e = cudaStreamSynchronize(st);
+  if (e != cudaSuccess) return op_fail(MSLT_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+  return 0;
+}
+
+int check_rows(const char* what, int dtype, int rows, int width, int width_mult, int width_max) {
+  if (dtype != 0 && dtype != 1) return op_fail(MSLT_ERR_ARG, "%s: dtype must be 0 or 1", what);
+  if (rows < 1) return op_fail(MSLT_ERR_ARG, "%s: rows must be >= 1", what);
+  if (width < 1 || width % width_mult || width > width_max)
+    return op_fail(MSLT_ERR_ARG, "%s: row length must be a multiple of %d and <= %d", what, width_mult, width_max);
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0)
+    return op_fail(MSLT_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  return 0;
+}
+
 // ---- allocation-free variant ------------------------------------------------------------------
 // Scratch for mslt_op_cross_entropy_noalloc lives in the library image, so the call needs no
 // cudaMalloc.  Every GPU that loads the library holds these bytes until the process exits.
@@ -146,6 +164,65 @@ int mslt_op_cross_entropy(int32_t dtype, const float* d_logits, int64_t ldl, con
                    ce_scratch_bytes(R));
   return run_ce(dtype, d_logits, ldl, d_labels, R, V, d_dlogits, ldd, d_loss, d_scratch,
                 (cudaStream_t)cuda_stream);
+}
+
+}  // extern "C"
+
+extern "C" {
+
+int mslt_op_layernorm(int32_t dtype, const void* d_z, const float* d_gamma, const float* d_beta, void* d_y,
+                      float* d_stats, int32_t rows, int32_t H, float eps, void* cuda_stream, int32_t sync) {
+  if (!d_z || !d_gamma || !d_beta || !d_y) return op_fail(MSLT_ERR_ARG, "layernorm: null pointer");
+  int rc = check_rows("layernorm", dtype, rows, H, 8, 1024);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  launch_ln_fwd(dtype == 1, d_z, d_gamma, d_beta, d_y, d_stats, rows, H, eps, st);
+  return finish_op("layernorm", st, sync);
+}
+
+int mslt_op_layernorm_bwd(int32_t dtype, const void* d_dy, const void* d_z, const float* d_stats,
+                          const float* d_gamma, void* d_dz, float* d_dgamma, float* d_dbeta, int32_t rows,
+                          int32_t H, void* cuda_stream, int32_t sync) {
+  if (!d_dy || !d_z || !d_stats || !d_gamma || !d_dz || !d_dgamma || !d_dbeta)
+    return op_fail(MSLT_ERR_ARG, "layernorm_bwd: null pointer");
+  int rc = check_rows("layernorm_bwd", dtype, rows, H, 8, 1024);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  launch_ln_bwd(dtype == 1, d_dy, d_z, d_stats, d_gamma, d_dz, d_dgamma, d_dbeta, rows, H, st);
+  return finish_op("layernorm_bwd", st, sync);
+}
+
+int mslt_op_softmax(int32_t dtype, const void* d_scores, void* d_probs, const int32_t* d_seq_lens,
+                    int32_t rows, int32_t S, int32_t rows_per_seq, float scale, void* cuda_stream,
+                    int32_t sync) {
+  if (!d_scores || !d_probs) return op_fail(MSLT_ERR_ARG, "softmax: null pointer");
+  int rc = check_rows("softmax", dtype, rows, S, 8, 512);
+  if (rc) return rc;
+  if (rows_per_seq < 1) return op_fail(MSLT_ERR_ARG, "softmax: rows_per_seq must be >= 1");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  launch_softmax_fwd(dtype == 1, d_scores, d_probs, d_seq_lens, rows, S, rows_per_seq, scale, st);
+  return finish_op("softmax", st, sync);
+}
+
+int mslt_op_softmax_bwd(int32_t dtype, void* d_dp, const void* d_probs, int32_t rows, int32_t S, float scale,
+                        void* cuda_stream, int32_t sync) {
+  if (!d_dp || !d_probs) return op_fail(MSLT_ERR_ARG, "softmax_bwd: null pointer");
+  int rc = check_rows("softmax_bwd", dtype, rows, S, 8, 512);
+  if (rc) return rc;
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  launch_softmax_bwd(dtype == 1, d_dp, d_probs, rows, S, scale, st);
+  return finish_op("softmax_bwd", st, sync);
+}
+
+int mslt_op_colsum(int32_t dtype, const void* d_x, int64_t ld, int32_t rows, int32_t N, float* d_out,
+                   void* cuda_stream, int32_t sync) {
+  if (!d_x || !d_out) return op_fail(MSLT_ERR_ARG, "colsum: null pointer");
+  int rc = check_rows("colsum", dtype, rows, N, 8, 1 << 30);
+  if (rc) return rc;
+  if (ld < N || ld % 8) return op_fail(MSLT_ERR_ARG, "colsum: ld must be a multiple of 8 and >= N");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  launch_colsum(dtype == 1, d_x, ld, rows, N, d_out, st);
+  return finish_op("colsum", st, sync);
 }
 
 }  // extern "C"

@@ -46,3 +46,111 @@ def test_cross_entropy_matches_oracle(dtype, R, V):
     loss, _ = run_cross_entropy(Bd.mslt_op_cross_entropy, dtype, logits, labels, V, want_grad=False,
                                 scratch=scratch)
     assert abs(loss - want_loss) / want_loss < 1e-5
+
+
+def _t(x, dtype):
+    import torch
+    return torch.from_numpy(np.ascontiguousarray(x, dtype=np.float32)).cuda().to(
+        torch.bfloat16 if dtype == 1 else torch.float32)
+
+
+def _stream():
+    import torch
+    return torch.cuda.current_stream().cuda_stream
+
+
+@pytest.mark.parametrize("dtype", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("rows,H", [(5, 128), (37, 192), (130, 768), (64, 1024), (9, 320)])
+def test_layernorm_forward_and_backward_match_oracle(dtype, rows, H):
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    rng = np.random.default_rng(rows * H)
+    z = _t(rng.standard_normal((rows, H)) * 2 + 0.5, dtype)
+    gamma = (1 + 0.1 * rng.standard_normal(H)).astype(np.float32)
+    beta = (0.1 * rng.standard_normal(H)).astype(np.float32)
+    dy = _t(rng.standard_normal((rows, H)), dtype)
+    d_g, d_b = torch.from_numpy(gamma).cuda(), torch.from_numpy(beta).cuda()
+    y = torch.empty_like(z)
+    stats = torch.empty((rows, 2), device="cuda")
+    Bd.mslt_op_layernorm(z, d_g, d_b, y, stats, 1e-12, _stream())
+    z64, dy64 = z.double().cpu().numpy(), dy.double().cpu().numpy()
+    y_ref, xhat, rstd = O.layer_norm(z64, gamma.astype(np.float64), beta.astype(np.float64), 1e-12)
+    tol = 2e-5 if dtype == 0 else 6e-3
+    assert np.abs(y.double().cpu().numpy() - y_ref).max() / np.abs(y_ref).max() < tol
+    st = stats.cpu().numpy()
+    np.testing.assert_allclose(st[:, 0], z64.mean(-1), atol=1e-5)
+    np.testing.assert_allclose(st[:, 1], rstd[:, 0], rtol=1e-5)
+    # without statistics (frozen layers)
+    y2 = torch.empty_like(z)
+    Bd.mslt_op_layernorm(z, d_g, d_b, y2, None, 1e-12, _stream())
+    assert torch.equal(y, y2)
+    # backward
+    dz = torch.empty_like(z)
+    dgam = torch.zeros(H, device="cuda"); dbet = torch.zeros(H, device="cuda")
+    Bd.mslt_op_layernorm_bwd(dy, z, stats, d_g, dz, dgam, dbet, _stream())
+    dz_ref, dg_ref, db_ref = O.layer_norm_backward(dy64, xhat, rstd, gamma.astype(np.float64))
+    assert np.abs(dz.double().cpu().numpy() - dz_ref).max() / np.abs(dz_ref).max() < tol
+    assert np.abs(dgam.cpu().numpy() - dg_ref).max() / np.abs(dg_ref).max() < 1e-4
+    assert np.abs(dbet.cpu().numpy() - db_ref).max() / np.abs(db_ref).max() < 1e-4
+    # the column sums are accumulated: a second call doubles them
+    Bd.mslt_op_layernorm_bwd(dy, z, stats, d_g, dz, dgam, dbet, _stream())
+    assert np.abs(dbet.cpu().numpy() - 2 * db_ref).max() / np.abs(db_ref).max() < 2e-4
+
+
+@pytest.mark.parametrize("dtype", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("S", [8, 64, 72, 128, 512])
+def test_softmax_forward_and_backward_match_oracle(dtype, S):
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    B, A = 3, 2
+    rng = np.random.default_rng(S)
+    sc = _t(rng.standard_normal((B * A * S, S)) * 3, dtype)
+    lens = np.array([S, max(1, S // 3), 1], dtype=np.int32)
+    d_lens = torch.from_numpy(lens).cuda()
+    p = torch.empty_like(sc)
+    Bd.mslt_op_softmax(sc, p, d_lens, A * S, 0.125, _stream())
+    sc64 = sc.double().cpu().numpy().reshape(B, A, S, S)
+    p_ref = O.masked_softmax(sc64 * 0.125, lens).reshape(B * A * S, S)
+    got = p.double().cpu().numpy()
+    tol = 2e-6 if dtype == 0 else 4e-3
+    assert np.abs(got - p_ref).max() < tol
+    assert np.all(got[p_ref == 0] == 0)
+    # in place
+    sc2 = sc.clone()
+    Bd.mslt_op_softmax(sc2, sc2, d_lens, A * S, 0.125, _stream())
+    assert torch.equal(sc2, p)
+    # backward
+    dp = _t(rng.standard_normal((B * A * S, S)), dtype)
+    dp64 = dp.double().cpu().numpy()
+    ref = O.softmax_backward(dp64, got) * 0.125
+    Bd.mslt_op_softmax_bwd(dp, p, 0.125, _stream())
+    assert np.abs(dp.double().cpu().numpy() - ref).max() / np.abs(ref).max() < (2e-5 if dtype == 0 else 6e-3)
+
+
+@pytest.mark.parametrize("dtype", [0, 1], ids=["fp32", "bf16"])
+@pytest.mark.parametrize("rows,N,ld", [(7, 8, 8), (300, 768, 768), (1000, 1040, 1048), (64, 30528, 30528)])
+def test_colsum_matches_numpy(dtype, rows, N, ld):
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    rng = np.random.default_rng(rows + N)
+    x = _t(rng.standard_normal((rows, ld)), dtype)
+    out = torch.full((ld,), 0.5, device="cuda")
+    Bd.mslt_op_colsum(x, N, out, _stream())
+    ref = 0.5 + x.double().cpu().numpy()[:, :N].sum(0)
+    got = out.cpu().numpy()
+    assert np.abs(got[:N] - ref).max() < 1e-4 * max(1.0, np.abs(ref).max())
+    assert np.all(got[N:] == 0.5)                   # nothing past N is touched
+
+
+def test_op_argument_checks():
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    z = torch.zeros((4, 100), device="cuda")        # row length not a multiple of 8
+    g = torch.zeros(100, device="cuda")
+    with pytest.raises(Bd.MsltError) as ei:
+        Bd.mslt_op_layernorm(z, g, g, z, None, 1e-12, _stream())
+    assert ei.value.code == -1
+    s = torch.zeros((4, 1024), device="cuda")       # row longer than the softmax kernels hold
+    with pytest.raises(Bd.MsltError) as ei:
+        Bd.mslt_op_softmax(s, s, None, 4, 1.0, _stream())
+    assert ei.value.code == -1
