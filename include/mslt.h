@@ -220,6 +220,16 @@ int mslt_op_gemm(const mslt_gemm_desc* desc, void* cuda_stream, int32_t* d_statu
 int mslt_op_gemm_enqueue(const mslt_gemm_desc* desc, void* cuda_stream, int32_t* d_status);
 
 /*
+ * Test hook for the failure path.  Every wait inside the tensor-core kernel is bounded; when one
+ * runs out the CTA sets bit 0 of the status word, drains, frees its tensor memory and returns, and
+ * the host call reports MSLT_ERR_DEVICE.  After mslt_debug_starve_next_gemm(1) the NEXT dtype-1
+ * contraction (and only that one) runs with a producer that issues no copies and a wait limit of
+ * about 20 ms, so this path can be exercised without faulting or hanging the GPU; its output is
+ * garbage.  The context and the device stay usable.
+ */
+int mslt_debug_starve_next_gemm(int32_t on);
+
+/*
  * The loss kernel alone (MLM objective, Section 4.1; mean over the valid slots as in the step):
  * for every row r of fp32 logits [R, ldl] with label in [0, V): nll = logsumexp - logit[label];
  * *d_loss = sum nll / n_valid; d_dlogits (may be NULL) [R, ldd] receives

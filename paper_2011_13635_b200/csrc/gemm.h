@@ -16,6 +16,10 @@ int gemm_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* err
 int gemm_simt_launch(const mslt_gemm_desc& d, cudaStream_t st, char* err);
 int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* err);
 
+// Test hook: the next tensor-core launch gets a producer that issues no copies and a wait limit of
+// about 20 ms, so that its first wait runs out and the give-up path is exercised.
+void gemm_tc_starve_next(int on);
+
 // Kernels launched by the GEMM front end since the library was loaded (for launch accounting).
 int64_t gemm_launches();
 

@@ -21,6 +21,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 #include <string>
 #include <unordered_map>
@@ -41,7 +42,7 @@ constexpr int NUM_EPI_WARPS = 8;
 constexpr int NUM_THREADS = 64 + 32 * NUM_EPI_WARPS;
 constexpr int STAGING_BYTES = 4096;  // per epilogue warp
 constexpr uint32_t TMEM_COLS = 512;
-constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // about 2 s of SM clock
+constexpr long long WAIT_LIMIT_CYCLES = 4000000000ll;  // about 2 s of SM clock (the default limit)
 
 struct TcParams {
   int M, N, K, batch, hdiv;
@@ -57,6 +58,8 @@ struct TcParams {
   bf16* aux;
   const bf16* residual;
   const int* seq_lens;  // act 3: valid keys per outer batch index, or null
+  long long wait_limit; // SM cycles a wait may take before the CTA gives up
+  int starve;           // test hook: the producer issues no copies, so the first wait runs out
   int* status;
   uint32_t idesc;
 };
@@ -97,7 +100,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     if (mbar_try_wait(bar, parity)) return true;
     if ((++spins & 255u) == 0u) {
       if (*abort_flag) return false;
-      if (now_cycles() - t0 > WAIT_LIMIT_CYCLES) {
+      if (now_cycles() - t0 > *reinterpret_cast<volatile long long*>(abort_flag + 1)) {
         *abort_flag = 1;
         atomicOr(status, ST_WAIT_TIMEOUT);
         return false;
@@ -336,7 +339,7 @@ __device__ __forceinline__ bool pair_sync(volatile int* flags, int me, int other
     while (flags[other] < seq) {
       if ((++spins & 255u) == 0u) {
         if (*abort_flag) { ok = 0; break; }
-        if (now_cycles() - t0 > WAIT_LIMIT_CYCLES) {
+        if (now_cycles() - t0 > *reinterpret_cast<volatile long long*>(abort_flag + 1)) {
           *abort_flag = 1;
           atomicOr(status, ST_WAIT_TIMEOUT);
           ok = 0;
@@ -395,6 +398,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       mbar_init(smem_u32(&tempty_bar[a]), kPair ? 2 * NUM_EPI_WARPS : NUM_EPI_WARPS);
     }
     *abort_flag = 0;
+    *reinterpret_cast<volatile long long*>(abort_flag + 1) = p.wait_limit;  // read by every bounded wait
     if (kSoftmax)
       for (int i = 0; i < NUM_EPI_WARPS; i++) xflag[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -421,7 +425,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int tiles_per_z = p.m_tiles * p.n_tiles;
   const int per_split = tiles_per_z * p.batch;
 
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && !p.starve) {
     // ------------------------------- TMA producer -------------------------------
     uint32_t it = 0;
     bool ok = true;
@@ -816,6 +820,9 @@ int get_map(const void* ptr, long long rows, long long K, long long rs, long lon
 
 }  // namespace
 
+static std::atomic<int> g_starve_next{0};
+void gemm_tc_starve_next(int on) { g_starve_next.store(on ? 1 : 0); }
+
 int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* err) {
   static int num_sms = 0;
   static int smem_optin = 0;
@@ -911,6 +918,11 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   p.d_fp32 = d.d_fp32; p.accumulate = d.accumulate; p.alpha = d.alpha; p.bias = d.bias; p.act = d.act;
   p.aux = (bf16*)d.aux; p.residual = (const bf16*)d.residual; p.status = status;
   p.seq_lens = d.seq_lens;
+  p.wait_limit = WAIT_LIMIT_CYCLES;
+  if (g_starve_next.exchange(0)) {  // armed by mslt_debug_starve_next_gemm
+    p.starve = 1;
+    p.wait_limit = 40000000ll;  // about 20 ms
+  }
   // 16-byte vector access in the epilogue needs every row segment to start on a 16-byte boundary
   // in each of the buffers it touches (bf16 ones are the stricter case: 8 elements)
   auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };

@@ -932,6 +932,11 @@ int mslt_get_timings(mslt_ctx* c, float* ms, int32_t n) {
   return 0;
 }
 
+int mslt_debug_starve_next_gemm(int32_t on) {
+  gemm_tc_starve_next(on);
+  return 0;
+}
+
 static int check_gemm_desc(const mslt_gemm_desc* d) {
   if (!d || !d->A || !d->B || !d->D) return fail(MSLT_ERR_ARG, "null pointer");
   if (d->M < 1 || d->N < 1 || d->K < 1 || d->batch < 1 || d->hdiv < 1)

@@ -188,3 +188,33 @@ def test_bf16_softmax_epilogue(S):
     assert np.abs(got - ref).max() < 6e-3
     assert np.all(got[ref == 0] == 0)                  # masked keys are exactly zero
     np.testing.assert_allclose(got.sum(-1), 1.0, atol=2e-2)
+
+
+def test_wait_that_runs_out_is_reported_and_leaves_the_device_usable():
+    """Failure path without a fault: the producer of one launch issues no copies, the first wait
+    runs out after ~20 ms, the kernel drains and returns, and the call reports MSLT_ERR_DEVICE."""
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    M = N = 128
+    K = 64
+    a = torch.randn((M, K), device="cuda").to(torch.bfloat16)
+    b = torch.randn((N, K), device="cuda").to(torch.bfloat16)
+    out = torch.zeros((M, N), device="cuda", dtype=torch.bfloat16)
+    d = Bd.GemmDesc()
+    d.dtype, d.M, d.N, d.K, d.batch, d.hdiv, d.alpha = 1, M, N, K, 1, 1, 1.0
+    d.A, d.a_rs, d.a_ks = a.data_ptr(), K, 1
+    d.B, d.b_rs, d.b_ks = b.data_ptr(), K, 1
+    d.D, d.ldd = out.data_ptr(), N
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    Bd.lib.mslt_debug_starve_next_gemm(1)
+    with pytest.raises(Bd.MsltError) as ei:
+        Bd.mslt_op_gemm(d, stream, status)
+    assert ei.value.code == -5
+    assert int(status.item()) & 1
+    # the hook disarms itself: the same call now succeeds and is correct
+    status.zero_()
+    Bd.mslt_op_gemm(d, stream, status)
+    ref = a.double() @ b.double().t()
+    assert (out.double() - ref).abs().max() / ref.abs().max() < 6e-3
+    assert int(status.item()) == 0
