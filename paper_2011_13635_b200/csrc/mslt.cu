@@ -79,7 +79,7 @@ struct Workspace {
   char* z0;
   float* st0;
   char *hm, *ut, *gt, *tm, *dlogits, *dtm, *dgt, *dhm;
-  float *hst, *logits, *nll;
+  float *hst, *logits, *nll, *dtm32;
   char *dxa, *dxb, *dz2, *dg, *dy, *dz1, *dc, *dp, *dqkv;
 };
 
@@ -214,6 +214,7 @@ void plan_workspace(const mslt_arch& a, const std::vector<Tensor>& tensors, char
   w.dlogits = take(R * Vp * E);
   w.nll = (float*)take(R * 4);
   w.dtm = take(R * H * E); w.dgt = take(R * H * E); w.dhm = take(R * H * E);
+  w.dtm32 = (float*)take(R * H * 4);
   w.dxa = take(T * H * E); w.dxb = take(T * H * E); w.dz2 = take(T * H * E);
   w.dg = take(T * F * E); w.dy = take(T * H * E); w.dz1 = take(T * H * E);
   w.dc = take(T * H * E); w.dp = take(P2 * E); w.dqkv = take(T * 3 * H * E);
@@ -506,8 +507,17 @@ int head_backward(mslt_ctx* c, int B, int S, int P, bool full) {
     Lin g(c, R, H, V);
     g.d.A = w.dlogits; g.d.a_rs = Vp; g.d.a_ks = 1;
     g.d.B = Wc(c, toff(c, -1, "emb.word")); g.d.b_rs = 1; g.d.b_ks = H;
-    g.d.D = w.dtm; g.d.ldd = H;
-    TRY(run_gemm(c, g.d));
+    if (c->bf) {
+      // few output tiles, a contraction over the whole vocabulary: split it across the machine
+      // with fp32 partial sums, then round once to bf16
+      CUDA_TRY(cudaMemsetAsync(w.dtm32, 0, (size_t)R * H * 4, c->st));
+      g.d.D = w.dtm32; g.d.ldd = H; g.d.d_fp32 = 1; g.d.accumulate = 1;
+      TRY(run_gemm(c, g.d));
+      KL(PC_OTHER, 6.0 * R * H, launch_f32_to_bf16(w.dtm32, w.dtm, (int64_t)R * H, c->st));
+    } else {
+      g.d.D = w.dtm; g.d.ldd = H;
+      TRY(run_gemm(c, g.d));
+    }
   }
   if (full) {  // the shared word embedding moves only while every layer is trainable
     Lin g(c, V, H, R);
