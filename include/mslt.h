@@ -230,6 +230,12 @@ int mslt_op_gemm_enqueue(const mslt_gemm_desc* desc, void* cuda_stream, int32_t*
 int mslt_debug_starve_next_gemm(int32_t on);
 
 /*
+ * Memory-safety check for tests: every buffer the library carves out of the workspace is followed
+ * by a 256-byte guard band that no kernel may write and that is zero from mslt_create on.  Counts
+ * the guard bands that are no longer zero (*bad_out, host; 0 = no stray write).  Synchronises. */
+int mslt_debug_check_guards(mslt_ctx* ctx, int32_t* bad_out);
+
+/*
  * The loss kernel alone (MLM objective, Section 4.1; mean over the valid slots as in the step):
  * for every row r of fp32 logits [R, ldl] with label in [0, V): nll = logsumexp - logit[label];
  * *d_loss = sum nll / n_valid; d_dlogits (may be NULL) [R, ldd] receives

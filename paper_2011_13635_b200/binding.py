@@ -56,7 +56,7 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_op_gemm", "mslt_op_gemm_enqueue", "mslt_op_cross_entropy",
            "mslt_op_cross_entropy_scratch_bytes", "mslt_op_cross_entropy_noalloc", "mslt_op_layernorm",
            "mslt_op_layernorm_bwd", "mslt_op_softmax", "mslt_op_softmax_bwd", "mslt_op_colsum",
-           "mslt_debug_starve_next_gemm"]
+           "mslt_debug_starve_next_gemm", "mslt_debug_check_guards"]
 
 lib.mslt_last_error.restype = C.c_char_p
 lib.mslt_last_error.argtypes = [C.c_void_p]
@@ -103,6 +103,7 @@ lib.mslt_op_cross_entropy_noalloc.argtypes = [C.c_int32, C.c_void_p, C.c_int64, 
 
 _P = C.c_void_p
 lib.mslt_debug_starve_next_gemm.argtypes = [C.c_int32]
+lib.mslt_debug_check_guards.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
 lib.mslt_op_layernorm.argtypes = [C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
 lib.mslt_op_layernorm_bwd.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, _P, C.c_int32]
 lib.mslt_op_softmax.argtypes = [C.c_int32, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
@@ -335,6 +336,12 @@ class Mslt:
         out = np.empty(shape, dtype=np.float32)
         _check(lib.mslt_get_opt_state(self.h, name.encode(), which, out.ctypes.data, out.size))
         return out
+
+    def mslt_debug_check_guards(self) -> int:
+        """Number of workspace guard bands that a kernel has written into (0 = none)."""
+        bad = C.c_int32()
+        _check(lib.mslt_debug_check_guards(self.h, C.byref(bad)))
+        return bad.value
 
     def mslt_set_timing(self, level: int):
         _check(lib.mslt_set_timing(self.h, int(level)))

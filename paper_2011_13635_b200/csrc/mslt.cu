@@ -68,6 +68,7 @@ struct LayerBuf {
 
 struct Workspace {
   size_t bytes = 0;
+  std::vector<size_t> guards;  // byte offsets of the 256-byte guard bands that follow every buffer
   int* scalars;  // [0] status, [1] n_valid, [2] inv_n (float), [3] loss (float), [4] Adam step count,
                  // [5], [6] Adam bias corrections (float)
   int *rowsrc, *rowlabel;
@@ -179,9 +180,14 @@ constexpr int64_t kAdamChunk = 8192;
 void plan_workspace(const mslt_arch& a, const std::vector<Tensor>& tensors, char* base,
                     Workspace& w) {
   size_t off = 0;
+  // every buffer is followed by a 256-byte guard band that no kernel may touch (it stays zero
+  // from creation on; mslt_debug_check_guards looks for stray writes)
+  w.guards.clear();
   auto take = [&](size_t bytes) -> char* {
     char* p = base ? base + off : nullptr;
     off += (bytes + 255) / 256 * 256;
+    w.guards.push_back(off);
+    off += 256;
     return p;
   };
   const int64_t E = a.dtype == 1 ? 2 : 4;
@@ -939,6 +945,22 @@ int mslt_get_timings(mslt_ctx* c, float* ms, int32_t n) {
   if (!c || !ms || n < 5) return fail(MSLT_ERR_ARG, "need room for 5 floats");
   if (!c->have_events) return fail(MSLT_ERR_STATE, "no timed step has run");
   for (int i = 0; i < 5; i++) ms[i] = c->phase_ms[i];
+  return 0;
+}
+
+int mslt_debug_check_guards(mslt_ctx* c, int32_t* bad_out) {
+  if (!c || !bad_out) return fail(MSLT_ERR_ARG, "null pointer");
+  CUDA_TRY(cudaStreamSynchronize(c->st));
+  const char* base = (const char*)c->ws.scalars;  // the first buffer of the workspace
+  std::vector<uint64_t> host(32);
+  int bad = 0;
+  for (size_t off : c->ws.guards) {
+    CUDA_TRY(cudaMemcpyAsync(host.data(), base + off, 256, cudaMemcpyDeviceToHost, c->st));
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (uint64_t v : host)
+      if (v != 0) { bad++; break; }
+  }
+  *bad_out = bad;
   return 0;
 }
 

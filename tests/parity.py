@@ -112,6 +112,7 @@ def compare_step(m, oracle, cfg, batch, tol, report=None):
     for n in frozen:
         assert np.array_equal(m.mslt_get_param(n), raw_frozen[n][0]), ("frozen master moved", n)
         assert np.array_equal(m.mslt_get_param_raw(n), raw_frozen[n][1]), ("frozen copy moved", n)
+    assert m.mslt_debug_check_guards() == 0, "a kernel wrote outside its workspace buffer"
     if report is not None:
         report.append(dict(loss_gpu=loss_g, loss_oracle=loss_o, rel_loss=rel_loss, **worst))
     return loss_g, loss_o, worst

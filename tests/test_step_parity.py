@@ -108,4 +108,5 @@ def test_forward_matches_oracle(cfg):
     m.mslt_set_optimizer(lr=0.0)
     loss = m.mslt_step(d_tok, d_lens, d_pos, d_lab)
     assert abs(loss - nll.mean()) / nll.mean() < 1e-5
+    assert m.mslt_debug_check_guards() == 0
     m.close()
