@@ -178,7 +178,8 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
+// 32 consecutive accumulator columns of this lane's row, as 16 (even, odd) column pairs
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, float2 (&w)[16]) {
   uint32_t r[32];
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -193,8 +194,9 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float (&v)[32]) {
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 #pragma unroll
-  for (int i = 0; i < 32; i++) v[i] = __uint_as_float(r[i]);
+  for (int i = 0; i < 16; i++) w[i] = make_float2(__uint_as_float(r[2 * i]), __uint_as_float(r[2 * i + 1]));
 }
+__device__ __forceinline__ float2 splat2(float c) { return make_float2(c, c); }
 
 // Shared-memory matrix descriptor for a 128-byte-swizzled tile whose rows are 128 bytes apart and
 // whose 8-row groups are 1024 bytes apart.  lbo_bytes: distance between 64-element column blocks
@@ -210,40 +212,52 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr, uint32_t lbo_b
 }
 
 // GELU on the FMA pipe only: the epilogue of a GELU tile is bound by the special-function unit when
-// erf costs a reciprocal and an exponential per element.  gelu(u) = u * Phi(u) with
-// Phi(u) - 1/2 = u * Q(u^2), Q a degree-8 least-maximum-error fit on |u| <= 4 (gelu is off by less
-// than 3e-5 in fp32 there, far inside bf16 resolution); outside, the argument is clamped, which
-// leaves gelu(u) = u (1 - 3e-5) above and 3e-5 |u| below.
-__device__ __forceinline__ float gelu_fast(float u) {
-  const float c = fminf(fmaxf(u, -4.0f), 4.0f);
-  const float t = c * c;
-  float q = 8.093845117e-11f;
-  q = fmaf(q, t, -7.032516570e-09f);
-  q = fmaf(q, t, 2.727248615e-07f);
-  q = fmaf(q, t, -6.317188128e-06f);
-  q = fmaf(q, t, 9.916073864e-05f);
-  q = fmaf(q, t, -1.135572678e-03f);
-  q = fmaf(q, t, 9.883344319e-03f);
-  q = fmaf(q, t, -6.642043264e-02f);
-  q = fmaf(q, t, 3.989280708e-01f);
-  return u * fmaf(q, c, 0.5f);
+// erf costs a reciprocal and an exponential per element, and by instruction issue after that, so
+// the polynomials below run on the packed two-wide fp32 instructions (fma.rn.f32x2), two columns
+// per instruction.  gelu(u) = u * Phi(u) with Phi(u) - 1/2 = u * Q(u^2), Q a degree-8
+// least-maximum-error fit on |u| <= 4 (gelu is off by less than 3e-5 in fp32 there, far inside bf16
+// resolution).  Outside, u^2 is clamped to 16 and Phi saturates to [0, 1], which gives gelu(u) = u
+// above and 0 below (the exact values differ from those by less than 2e-4).
+__device__ __forceinline__ float2 gelu_fast2(float2 u) {
+  float2 t = __fmul2_rn(u, u);
+  t.x = fminf(t.x, 16.0f);
+  t.y = fminf(t.y, 16.0f);
+  float2 q = splat2(8.093845117e-11f);
+  q = __ffma2_rn(q, t, splat2(-7.032516570e-09f));
+  q = __ffma2_rn(q, t, splat2(2.727248615e-07f));
+  q = __ffma2_rn(q, t, splat2(-6.317188128e-06f));
+  q = __ffma2_rn(q, t, splat2(9.916073864e-05f));
+  q = __ffma2_rn(q, t, splat2(-1.135572678e-03f));
+  q = __ffma2_rn(q, t, splat2(9.883344319e-03f));
+  q = __ffma2_rn(q, t, splat2(-6.642043264e-02f));
+  q = __ffma2_rn(q, t, splat2(3.989280708e-01f));
+  float2 phi;
+  phi.x = __saturatef(fmaf(q.x, u.x, 0.5f));
+  phi.y = __saturatef(fmaf(q.y, u.y, 0.5f));
+  return __fmul2_rn(u, phi);
 }
 // GELU'(u) = Phi(u) + u phi(u), also on the FMA pipe: 0.5 + u * P(u^2) with a degree-17 odd
 // least-maximum-error fit on |u| <= 4 (absolute error below 1e-4); beyond that the derivative is
 // 0 or 1 to within 5e-4.  The result multiplies a gradient that is then rounded to bf16.
-__device__ __forceinline__ float gelu_grad_fast(float u) {
-  const float t = u * u;
-  float p = 9.837601957e-10f;
-  p = fmaf(p, t, -8.257008028e-08f);
-  p = fmaf(p, t, 3.042579986e-06f);
-  p = fmaf(p, t, -6.523749948e-05f);
-  p = fmaf(p, t, 9.104776309e-04f);
-  p = fmaf(p, t, -8.736754371e-03f);
-  p = fmaf(p, t, 5.852845753e-02f);
-  p = fmaf(p, t, -2.649477277e-01f);
-  p = fmaf(p, t, 7.976755055e-01f);
-  p = fmaf(p, u, 0.5f);
-  return fabsf(u) >= 4.0f ? (u > 0.f ? 1.0f : 0.0f) : p;
+__device__ __forceinline__ float2 gelu_grad_fast2(float2 u) {
+  const float2 t = __fmul2_rn(u, u);
+  float2 p = splat2(9.837601957e-10f);
+  p = __ffma2_rn(p, t, splat2(-8.257008028e-08f));
+  p = __ffma2_rn(p, t, splat2(3.042579986e-06f));
+  p = __ffma2_rn(p, t, splat2(-6.523749948e-05f));
+  p = __ffma2_rn(p, t, splat2(9.104776309e-04f));
+  p = __ffma2_rn(p, t, splat2(-8.736754371e-03f));
+  p = __ffma2_rn(p, t, splat2(5.852845753e-02f));
+  p = __ffma2_rn(p, t, splat2(-2.649477277e-01f));
+  p = __ffma2_rn(p, t, splat2(7.976755055e-01f));
+  p = __ffma2_rn(p, u, splat2(0.5f));
+  // step(u) without a second comparison: u * 2^100 saturated to [0, 1]
+  p.x = fabsf(u.x) >= 4.0f ? __saturatef(u.x * 1.2676506e30f) : p.x;
+  p.y = fabsf(u.y) >= 4.0f ? __saturatef(u.y * 1.2676506e30f) : p.y;
+  return p;
+}
+__device__ __forceinline__ float2 bf162_to_f2(uint32_t h) {
+  return make_float2(__uint_as_float(h << 16), __uint_as_float(h & 0xffff0000u));
 }
 
 // Staging buffer of one epilogue warp: 32 rows of 128 bytes.  Lane r writes its row as 16-byte
@@ -258,7 +272,7 @@ __device__ __forceinline__ uint32_t slot_b16(int r, int c) {  // c in 0..3: 4 pi
 
 // Writes a 32 x 32 chunk (lane = row, v = its 32 columns) to `base` (row-major, leading dimension
 // ldd, element (m_warp + row, n0 + col)) with coalesced 16-byte stores.
-__device__ __forceinline__ void stage_store_bf16(uint8_t* stg, int lane, const float (&v)[32], bf16* base,
+__device__ __forceinline__ void stage_store_bf16(uint8_t* stg, int lane, const float2 (&w)[16], bf16* base,
                                                  long long ldd, int m_warp, int n0, int M, int N,
                                                  int vec_ok) {
 #pragma unroll
@@ -266,7 +280,7 @@ __device__ __forceinline__ void stage_store_bf16(uint8_t* stg, int lane, const f
     uint4 pk;
     __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
 #pragma unroll
-    for (int e = 0; e < 4; e++) h[e] = __floats2bfloat162_rn(v[8 * c + 2 * e], v[8 * c + 2 * e + 1]);
+    for (int e = 0; e < 4; e++) h[e] = __float22bfloat162_rn(w[4 * c + e]);
     *reinterpret_cast<uint4*>(stg + slot_b16(lane, c)) = pk;
   }
   __syncwarp();
@@ -290,13 +304,13 @@ __device__ __forceinline__ void stage_store_bf16(uint8_t* stg, int lane, const f
   __syncwarp();
 }
 
-__device__ __forceinline__ void stage_store_f32(uint8_t* stg, int lane, const float (&v)[32], float* base,
+__device__ __forceinline__ void stage_store_f32(uint8_t* stg, int lane, const float2 (&w)[16], float* base,
                                                 long long ldd, int m_warp, int n0, int M, int N, int vec_ok,
                                                 int accumulate) {
 #pragma unroll
   for (int c = 0; c < 8; c++)
     *reinterpret_cast<float4*>(stg + slot_f32(lane, c)) =
-        make_float4(v[4 * c], v[4 * c + 1], v[4 * c + 2], v[4 * c + 3]);
+        make_float4(w[2 * c].x, w[2 * c].y, w[2 * c + 1].x, w[2 * c + 1].y);
   __syncwarp();
 #pragma unroll
   for (int it = 0; it < 8; it++) {
@@ -427,8 +441,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
   if (warp == 0 && lane == 0 && !p.starve) {
     // ------------------------------- TMA producer -------------------------------
-    uint32_t it = 0;
+    // Ring position kept as (stage, phase) counters and tile coordinates kept in scalars: the loop
+    // body is a wait, a handful of adds and the copies, so one thread keeps the ring full.
+    uint32_t it = 0, s = 0, ph = 0;
     bool ok = true;
+    // which coordinate slot carries k: slot 0 for a k-contiguous operand, else the permuted one
+    const int ak = p.a_mn ? p.a_perm[0] : 0, bk = p.b_mn ? p.b_perm[0] : 0;
+    const int da0 = ak == 0 ? BK : 0, da1 = ak == 1 ? BK : 0, da2 = ak == 2 ? BK : 0, da3 = ak == 3 ? BK : 0;
+    const int db0 = bk == 0 ? BK : 0, db1 = bk == 1 ? BK : 0, db2 = bk == 2 ? BK : 0, db3 = bk == 3 ? BK : 0;
+    const uint32_t smem0 = smem_u32(smem);
+    const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+    const uint32_t tx_bytes = kPair ? 2 * stage_bytes : stage_bytes;
+    const int a_boxes = p.a_mn ? BM / 64 : 1, b_boxes = p.b_mn ? bn_cta / 64 : 1;
     for (int w = w_first; w < p.total_work && ok; w += w_step) {
       const int split = w / per_split;
       int r = w - split * per_split;
@@ -438,43 +462,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int zo = z / p.hdiv, zi = z - zo * p.hdiv;
       const int kb0 = split * p.kb_per_split;
       const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
+      const int row0 = mt * mt_rows + (int)cta_rank * BM;
+      const int col0 = nt * p.bn + (int)cta_rank * bn_cta;
+      int ca[4], cb[4];
+      if (!p.a_mn) { ca[0] = kb0 * BK; ca[p.a_perm[0]] = row0; }
+      else         { ca[0] = row0; ca[p.a_perm[0]] = kb0 * BK; }
+      ca[p.a_perm[1]] = zi; ca[p.a_perm[2]] = zo;
+      if (!p.b_mn) { cb[0] = kb0 * BK; cb[p.b_perm[0]] = col0; }
+      else         { cb[0] = col0; cb[p.b_perm[0]] = kb0 * BK; }
+      cb[p.b_perm[1]] = zi; cb[p.b_perm[2]] = zo;
+      int a0 = ca[0], a1 = ca[1], a2 = ca[2], a3 = ca[3];
+      int b0 = cb[0], b1 = cb[1], b2 = cb[2], b3 = cb[3];
       for (int kb = kb0; kb < kb1; kb++, it++) {
-        const uint32_t s = it % p.stages, round = it / p.stages;
-        if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
-        const uint32_t fb_own = smem_u32(&full_bar[s]);
+        if (!mbar_wait(empty0 + s * 8, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+        const uint32_t fb_own = full0 + s * 8;
         // pair mode: both CTAs' copies are counted on the leader's barrier
         const uint32_t fb = kPair ? mapa_u32(fb_own, 0) : fb_own;
-        if (leader) mbar_expect_tx(fb_own, kPair ? 2 * stage_bytes : stage_bytes);
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        if (leader) mbar_expect_tx(fb_own, tx_bytes);
+        const uint32_t sa = smem0 + s * (uint32_t)stage_bytes;
         const uint32_t sb = sa + A_STAGE_BYTES;
-        const int row0 = mt * mt_rows + (int)cta_rank * BM;
-        const int col0 = nt * p.bn + (int)cta_rank * bn_cta;
-        int c[4];
-        if (!p.a_mn) {  // box {64 k, 128 rows}
-          c[0] = kb * BK; c[p.a_perm[0]] = row0; c[p.a_perm[1]] = zi; c[p.a_perm[2]] = zo;
-          if (kPair) tma_load_4d_pair(sa, &tmA, fb, c[0], c[1], c[2], c[3]);
-          else tma_load_4d(sa, &tmA, fb, c[0], c[1], c[2], c[3]);
-        } else {        // two boxes {64 rows, 64 k}
-          c[p.a_perm[0]] = kb * BK; c[p.a_perm[1]] = zi; c[p.a_perm[2]] = zo;
-#pragma unroll
-          for (int h = 0; h < BM / 64; h++) {
-            c[0] = row0 + h * 64;
-            if (kPair) tma_load_4d_pair(sa + h * (64 * BK * 2), &tmA, fb, c[0], c[1], c[2], c[3]);
-            else tma_load_4d(sa + h * (64 * BK * 2), &tmA, fb, c[0], c[1], c[2], c[3]);
-          }
+        // k-contiguous operand: one box {64 k, rows}; row-contiguous: boxes {64 rows, 64 k}
+        for (int h = 0; h < a_boxes; h++) {
+          if (kPair) tma_load_4d_pair(sa + h * (64 * BK * 2), &tmA, fb, a0 + h * 64, a1, a2, a3);
+          else tma_load_4d(sa + h * (64 * BK * 2), &tmA, fb, a0 + h * 64, a1, a2, a3);
         }
-        if (!p.b_mn) {  // box {64 k, this CTA's B rows}
-          c[0] = kb * BK; c[p.b_perm[0]] = col0; c[p.b_perm[1]] = zi; c[p.b_perm[2]] = zo;
-          if (kPair) tma_load_4d_pair(sb, &tmB, fb, c[0], c[1], c[2], c[3]);
-          else tma_load_4d(sb, &tmB, fb, c[0], c[1], c[2], c[3]);
-        } else {
-          c[p.b_perm[0]] = kb * BK; c[p.b_perm[1]] = zi; c[p.b_perm[2]] = zo;
-          for (int h = 0; h < bn_cta / 64; h++) {
-            c[0] = col0 + h * 64;
-            if (kPair) tma_load_4d_pair(sb + h * (64 * BK * 2), &tmB, fb, c[0], c[1], c[2], c[3]);
-            else tma_load_4d(sb + h * (64 * BK * 2), &tmB, fb, c[0], c[1], c[2], c[3]);
-          }
+        for (int h = 0; h < b_boxes; h++) {
+          if (kPair) tma_load_4d_pair(sb + h * (64 * BK * 2), &tmB, fb, b0 + h * 64, b1, b2, b3);
+          else tma_load_4d(sb + h * (64 * BK * 2), &tmB, fb, b0 + h * 64, b1, b2, b3);
         }
+        a0 += da0; a1 += da1; a2 += da2; a3 += da3;
+        b0 += db0; b1 += db1; b2 += db2; b3 += db3;
+        if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
       }
     }
     if (!ok || *abort_flag) {
@@ -493,12 +511,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
   } else if (warp == 1 && lane == 0 && leader) {
     // ------------------------------- MMA issuer -------------------------------
-    uint32_t it = 0, tile = 0;
+    // One thread feeds the tensor core, so its loop is kept short: ring position as counters,
+    // descriptors as a constant high word plus a low word that only gains the stage and k offsets.
+    uint32_t tile = 0, s = 0, ph = 0;
     bool ok = true;
     const uint32_t a_lbo = p.a_mn ? 64 * BK * 2 : 16;
     const uint32_t b_lbo = p.b_mn ? 64 * BK * 2 : 16;
-    const uint32_t a_kstep = p.a_mn ? UMMA_K * 128 : UMMA_K * 2;  // bytes per 16-wide k step
-    const uint32_t b_kstep = p.b_mn ? UMMA_K * 128 : UMMA_K * 2;
+    const uint32_t a_kstep = (p.a_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4;  // 16-byte units per 16-wide k step
+    const uint32_t b_kstep = (p.b_mn ? UMMA_K * 128 : UMMA_K * 2) >> 4;
+    const uint64_t a_desc0 = make_smem_desc(smem_u32(smem), a_lbo);
+    const uint64_t b_desc0 = make_smem_desc(smem_u32(smem) + A_STAGE_BYTES, b_lbo);
+    const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), b_hi = (uint32_t)(b_desc0 >> 32);
+    const uint32_t a_lo0 = (uint32_t)a_desc0, b_lo0 = (uint32_t)b_desc0;
+    const uint32_t stage_units = (uint32_t)stage_bytes >> 4;
+    const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
     for (int w = w_first; w < p.total_work && ok; w += w_step, tile++) {
       const int split = w / per_split;
       const int kb0 = split * p.kb_per_split;
@@ -507,21 +533,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       if (!mbar_wait(smem_u32(&tempty_bar[acc]), (use & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + acc * 256;
-      for (int kb = kb0; kb < kb1; kb++, it++) {
-        const uint32_t s = it % p.stages, round = it / p.stages;
-        if (!mbar_wait(smem_u32(&full_bar[s]), round & 1, abort_flag, p.status)) { ok = false; break; }
+      uint32_t accum = 0;
+      for (int kb = kb0; kb < kb1; kb++) {
+        if (!mbar_wait(full0 + s * 8, ph, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t sb = sa + A_STAGE_BYTES;
+        const uint32_t a_lo = a_lo0 + s * stage_units, b_lo = b_lo0 + s * stage_units;
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; k++) {
-          const uint64_t ad = make_smem_desc(sa + k * a_kstep, a_lbo);
-          const uint64_t bd = make_smem_desc(sb + k * b_kstep, b_lbo);
-          if (kPair) tc_mma_pair(d_tmem, ad, bd, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
-          else tc_mma(d_tmem, ad, bd, p.idesc, (kb > kb0 || k > 0) ? 1u : 0u);
+          const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo + k * a_kstep);
+          const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo + k * b_kstep);
+          if (kPair) tc_mma_pair(d_tmem, ad, bd, p.idesc, accum);
+          else tc_mma(d_tmem, ad, bd, p.idesc, accum);
+          accum = 1;
         }
         // the stage is free (in both CTAs) once these MMAs have read it
-        if (kPair) tc_commit_pair(smem_u32(&empty_bar[s])); else tc_commit(smem_u32(&empty_bar[s]));
+        if (kPair) tc_commit_pair(empty0 + s * 8); else tc_commit(empty0 + s * 8);
+        if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
       }
       if (ok) {  // accumulator complete
         if (kPair) tc_commit_pair(smem_u32(&tfull_bar[acc])); else tc_commit(smem_u32(&tfull_bar[acc]));
@@ -566,23 +593,25 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         len = min(max(len, 1), p.N);
         const int c0 = hsel, c1 = hsel + 2;
         const bool h0 = c0 * 32 < p.N && c0 < p.bn / 32, h1 = c1 * 32 < p.N && c1 < p.bn / 32;
-        float v0[32], v1[32];
+        float2 v0[16], v1[16];
         float mx = -INFINITY;
         const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
         if (h0) {
           tc_ld32(trow + c0 * 32, v0);
 #pragma unroll
-          for (int j = 0; j < 32; j++) {
-            v0[j] = (c0 * 32 + j < len) ? v0[j] * p.alpha : -INFINITY;
-            mx = fmaxf(mx, v0[j]);
+          for (int j = 0; j < 16; j++) {
+            v0[j].x = (c0 * 32 + 2 * j < len) ? v0[j].x * p.alpha : -INFINITY;
+            v0[j].y = (c0 * 32 + 2 * j + 1 < len) ? v0[j].y * p.alpha : -INFINITY;
+            mx = fmaxf(mx, fmaxf(v0[j].x, v0[j].y));
           }
         }
         if (h1) {
           tc_ld32(trow + c1 * 32, v1);
 #pragma unroll
-          for (int j = 0; j < 32; j++) {
-            v1[j] = (c1 * 32 + j < len) ? v1[j] * p.alpha : -INFINITY;
-            mx = fmaxf(mx, v1[j]);
+          for (int j = 0; j < 16; j++) {
+            v1[j].x = (c1 * 32 + 2 * j < len) ? v1[j].x * p.alpha : -INFINITY;
+            v1[j].y = (c1 * 32 + 2 * j + 1 < len) ? v1[j].y * p.alpha : -INFINITY;
+            mx = fmaxf(mx, fmaxf(v1[j].x, v1[j].y));
           }
         }
         // the accumulator is in registers now: hand it back before the slow part
@@ -600,11 +629,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         float sum = 0.f;
         if (h0) {
 #pragma unroll
-          for (int j = 0; j < 32; j++) { v0[j] = __expf(v0[j] - mx); sum += v0[j]; }
+          for (int j = 0; j < 16; j++) {
+            v0[j].x = __expf(v0[j].x - mx);
+            v0[j].y = __expf(v0[j].y - mx);
+            sum += v0[j].x + v0[j].y;
+          }
         }
         if (h1) {
 #pragma unroll
-          for (int j = 0; j < 32; j++) { v1[j] = __expf(v1[j] - mx); sum += v1[j]; }
+          for (int j = 0; j < 16; j++) {
+            v1[j].x = __expf(v1[j].x - mx);
+            v1[j].y = __expf(v1[j].y - mx);
+            sum += v1[j].x + v1[j].y;
+          }
         }
         xsum[me * 32 + lane] = sum;
         if (!pair_sync(xflag, me, other, seq + 1, lane, abort_flag, p.status)) { ok = false; break; }
@@ -612,13 +649,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const float inv = 1.0f / sum;
         if (h0) {
 #pragma unroll
-          for (int j = 0; j < 32; j++) v0[j] *= inv;
+          for (int j = 0; j < 16; j++) v0[j] = __fmul2_rn(v0[j], splat2(inv));
           stage_store_bf16(stg, lane, v0, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, c0 * 32, p.M, p.N,
                            p.vec_ok);
         }
         if (h1) {
 #pragma unroll
-          for (int j = 0; j < 32; j++) v1[j] *= inv;
+          for (int j = 0; j < 16; j++) v1[j] = __fmul2_rn(v1[j], splat2(inv));
           stage_store_bf16(stg, lane, v1, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, c1 * 32, p.M, p.N,
                            p.vec_ok);
         }
@@ -627,60 +664,72 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       for (int cidx = hsel; cidx < p.bn / 32; cidx += 2) {
         const int n0 = n_base + cidx * 32;
         if (n0 >= p.N) break;  // uniform over the warp
-        float v[32];
+        float2 v[16];
         tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256 + cidx * 32, v);
         const long long off = off0 + n0;
         const bool fullv = p.vec_ok && (n0 + 32 <= p.N);
         const bool row_ok = m < p.M;
         if (p.alpha != 1.0f) {
+          const float2 a2 = splat2(p.alpha);
 #pragma unroll
-          for (int j = 0; j < 32; j++) v[j] *= p.alpha;
+          for (int j = 0; j < 16; j++) v[j] = __fmul2_rn(v[j], a2);
         }
         if (p.bias) {
           if (n0 + 32 <= p.N) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              const float4 b4 = *reinterpret_cast<const float4*>(p.bias + n0 + j);
-              v[j] += b4.x; v[j + 1] += b4.y; v[j + 2] += b4.z; v[j + 3] += b4.w;
+            for (int j = 0; j < 16; j += 2) {
+              const float4 b4 = *reinterpret_cast<const float4*>(p.bias + n0 + 2 * j);
+              v[j] = __fadd2_rn(v[j], make_float2(b4.x, b4.y));
+              v[j + 1] = __fadd2_rn(v[j + 1], make_float2(b4.z, b4.w));
             }
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; j++)
-              if (n0 + j < p.N) v[j] += p.bias[n0 + j];
+            for (int j = 0; j < 16; j++) {
+              if (n0 + 2 * j < p.N) v[j].x += p.bias[n0 + 2 * j];
+              if (n0 + 2 * j + 1 < p.N) v[j].y += p.bias[n0 + 2 * j + 1];
+            }
           }
         }
         if (p.act == 1) {
           if (p.aux) stage_store_bf16(stg, lane, v, p.aux + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
 #pragma unroll
-          for (int j = 0; j < 32; j++) v[j] = gelu_fast(v[j]);
+          for (int j = 0; j < 16; j++) v[j] = gelu_fast2(v[j]);
         } else if (p.act == 2 && row_ok) {
           if (fullv) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              float t[8];
-              VecT<bf16>::load(p.aux + off + j, t);
-#pragma unroll
-              for (int e = 0; e < 8; e++) v[j + e] *= gelu_grad_fast(t[e]);
+            for (int j = 0; j < 16; j += 4) {
+              const uint4 raw = *reinterpret_cast<const uint4*>(p.aux + off + 2 * j);
+              v[j] = __fmul2_rn(v[j], gelu_grad_fast2(bf162_to_f2(raw.x)));
+              v[j + 1] = __fmul2_rn(v[j + 1], gelu_grad_fast2(bf162_to_f2(raw.y)));
+              v[j + 2] = __fmul2_rn(v[j + 2], gelu_grad_fast2(bf162_to_f2(raw.z)));
+              v[j + 3] = __fmul2_rn(v[j + 3], gelu_grad_fast2(bf162_to_f2(raw.w)));
             }
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; j++)
-              if (n0 + j < p.N) v[j] *= gelu_grad_fast(__bfloat162float(p.aux[off + j]));
+            for (int j = 0; j < 16; j++) {
+              float2 u = make_float2(0.f, 0.f);
+              if (n0 + 2 * j < p.N) u.x = __bfloat162float(p.aux[off + 2 * j]);
+              if (n0 + 2 * j + 1 < p.N) u.y = __bfloat162float(p.aux[off + 2 * j + 1]);
+              v[j] = __fmul2_rn(v[j], gelu_grad_fast2(u));
+            }
           }
         }
         if (p.residual && row_ok) {
           if (fullv) {
 #pragma unroll
-            for (int j = 0; j < 32; j += 8) {
-              float t[8];
-              VecT<bf16>::load(p.residual + off + j, t);
-#pragma unroll
-              for (int e = 0; e < 8; e++) v[j + e] += t[e];
+            for (int j = 0; j < 16; j += 4) {
+              const uint4 raw = *reinterpret_cast<const uint4*>(p.residual + off + 2 * j);
+              v[j] = __fadd2_rn(v[j], bf162_to_f2(raw.x));
+              v[j + 1] = __fadd2_rn(v[j + 1], bf162_to_f2(raw.y));
+              v[j + 2] = __fadd2_rn(v[j + 2], bf162_to_f2(raw.z));
+              v[j + 3] = __fadd2_rn(v[j + 3], bf162_to_f2(raw.w));
             }
           } else {
 #pragma unroll
-            for (int j = 0; j < 32; j++)
-              if (n0 + j < p.N) v[j] += __bfloat162float(p.residual[off + j]);
+            for (int j = 0; j < 16; j++) {
+              if (n0 + 2 * j < p.N) v[j].x += __bfloat162float(p.residual[off + 2 * j]);
+              if (n0 + 2 * j + 1 < p.N) v[j].y += __bfloat162float(p.residual[off + 2 * j + 1]);
+            }
           }
         }
         if (p.d_fp32)
