@@ -198,6 +198,38 @@ __device__ __forceinline__ void tc_ld32(uint32_t taddr, float2 (&w)[16]) {
 }
 __device__ __forceinline__ float2 splat2(float c) { return make_float2(c, c); }
 
+// The same read split in two, so that the next chunk's read is in flight while this chunk is worked
+// on: after tc_ld32_issue the registers are not valid until tc_ld32_wait has returned.  The wait
+// names the registers as in/out operands so that no use of them can be scheduled above it.
+__device__ __forceinline__ void tc_ld32_issue(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+        "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+        "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+        "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_ld32_wait(uint32_t (&r)[32]) {
+  asm volatile("tcgen05.wait::ld.sync.aligned;"
+               : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                 "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]),
+                 "+r"(r[15])
+               :
+               : "memory");
+  // the second half of the registers is tied to the same point in the instruction stream
+  asm volatile(""
+               : "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]),
+                 "+r"(r[23]), "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]),
+                 "+r"(r[30]), "+r"(r[31])
+               :
+               : "memory");
+}
+
 // Shared-memory matrix descriptor for a 128-byte-swizzled tile whose rows are 128 bytes apart and
 // whose 8-row groups are 1024 bytes apart.  lbo_bytes: distance between 64-element column blocks
 // of an MN-major operand (ignored by the hardware for K-major swizzled tiles).
@@ -260,14 +292,12 @@ __device__ __forceinline__ float2 bf162_to_f2(uint32_t h) {
   return make_float2(__uint_as_float(h << 16), __uint_as_float(h & 0xffff0000u));
 }
 
-// Staging buffer of one epilogue warp: 32 rows of 128 bytes.  Lane r writes its row as 16-byte
-// pieces; the slot functions permute the pieces so that both this row-per-lane write and the
-// row-segment-per-quarter-warp read that follows are free of bank conflicts.
-__device__ __forceinline__ uint32_t slot_f32(int r, int c) {  // c in 0..7: 8 pieces of 4 floats
-  return (uint32_t)(r * 128 + ((c ^ (r & 7)) << 4));
-}
-__device__ __forceinline__ uint32_t slot_b16(int r, int c) {  // c in 0..3: 4 pieces of 8 bf16
-  return (uint32_t)(r * 128 + (((c + ((r & 1) << 2)) ^ ((r >> 1) & 3)) << 4));
+// Staging buffer of one epilogue warp: 32 rows of 64 bytes (2 KB).  Lane r writes its row as four
+// 16-byte pieces; the slot function permutes the pieces so that both this
+// row-per-lane write and the row-segment-per-quarter-warp read that follows are free of bank
+// conflicts.  Bytes 2048.. of the warp's 4 KB hold the bias values of the warp's columns.
+__device__ __forceinline__ uint32_t slot_b16(int r, int c) {  // c in 0..3: pieces of 8 bf16 or 4 floats
+  return (uint32_t)(r * 64 + ((c ^ ((r >> 1) & 3)) << 4));
 }
 
 // Writes a 32 x 32 chunk (lane = row, v = its 32 columns) to `base` (row-major, leading dimension
@@ -304,39 +334,44 @@ __device__ __forceinline__ void stage_store_bf16(uint8_t* stg, int lane, const f
   __syncwarp();
 }
 
+// fp32 output: the same 2 KB transposer, used twice for 16 columns each.
 __device__ __forceinline__ void stage_store_f32(uint8_t* stg, int lane, const float2 (&w)[16], float* base,
                                                 long long ldd, int m_warp, int n0, int M, int N, int vec_ok,
                                                 int accumulate) {
 #pragma unroll
-  for (int c = 0; c < 8; c++)
-    *reinterpret_cast<float4*>(stg + slot_f32(lane, c)) =
-        make_float4(w[2 * c].x, w[2 * c].y, w[2 * c + 1].x, w[2 * c + 1].y);
-  __syncwarp();
+  for (int half = 0; half < 2; half++) {
 #pragma unroll
-  for (int it = 0; it < 8; it++) {
-    const int row = it * 4 + (lane >> 3), c = lane & 7;
-    const float4 val = *reinterpret_cast<const float4*>(stg + slot_f32(row, c));
-    const int mm = m_warp + row, nn = n0 + c * 4;
-    if (mm < M && nn < N) {
-      float* dst = base + (long long)mm * ldd + nn;
-      if (vec_ok && nn + 4 <= N) {
-        if (accumulate)
-          asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(val.x), "f"(val.y),
-                       "f"(val.z), "f"(val.w)
-                       : "memory");
-        else
-          *reinterpret_cast<float4*>(dst) = val;
-      } else {
-        const float e4[4] = {val.x, val.y, val.z, val.w};
+    for (int c = 0; c < 4; c++)
+      *reinterpret_cast<float4*>(stg + slot_b16(lane, c)) =
+          make_float4(w[8 * half + 2 * c].x, w[8 * half + 2 * c].y, w[8 * half + 2 * c + 1].x,
+                      w[8 * half + 2 * c + 1].y);
+    __syncwarp();
 #pragma unroll
-        for (int e = 0; e < 4; e++)
-          if (nn + e < N) {
-            if (accumulate) atomicAdd(dst + e, e4[e]); else dst[e] = e4[e];
-          }
+    for (int it = 0; it < 4; it++) {
+      const int row = it * 8 + (lane >> 2), c = lane & 3;
+      const float4 val = *reinterpret_cast<const float4*>(stg + slot_b16(row, c));
+      const int mm = m_warp + row, nn = n0 + half * 16 + c * 4;
+      if (mm < M && nn < N) {
+        float* dst = base + (long long)mm * ldd + nn;
+        if (vec_ok && nn + 4 <= N) {
+          if (accumulate)
+            asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst), "f"(val.x), "f"(val.y),
+                         "f"(val.z), "f"(val.w)
+                         : "memory");
+          else
+            *reinterpret_cast<float4*>(dst) = val;
+        } else {
+          const float e4[4] = {val.x, val.y, val.z, val.w};
+#pragma unroll
+          for (int e = 0; e < 4; e++)
+            if (nn + e < N) {
+              if (accumulate) atomicAdd(dst + e, e4[e]); else dst[e] = e4[e];
+            }
+        }
       }
     }
+    __syncwarp();
   }
-  __syncwarp();
 }
 
 // Hand-over between the two epilogue warps of a TMEM lane quarter: publish my sequence number
@@ -367,12 +402,78 @@ __device__ __forceinline__ bool pair_sync(volatile int* flags, int me, int other
   return ok != 0;
 }
 
+// Epilogue flavours.  Each is its own kernel instantiation: one kernel with every flavour behind
+// run-time branches measured 2-3x slower per chunk (register pressure and jumps across large code
+// blocks), which made shallow contractions wait for their epilogue.
+enum : int {
+  EPI_STORE = 0,   // bf16 out = alpha * acc + bias
+  EPI_RESIDUAL,    // bf16 out = alpha * acc + bias + residual row
+  EPI_GELU,        // bf16 out = gelu(alpha * acc + bias)
+  EPI_GELU_AUX,    // the same, and the pre-activation goes to aux
+  EPI_DGELU,       // bf16 out = (alpha * acc + bias) * gelu'(aux)
+  EPI_F32,         // fp32 out (stored, or added to what is there) = alpha * acc + bias
+  EPI_GENERIC,     // every other combination the descriptor allows, and unaligned buffers
+  EPI_SOFTMAX,     // masked row softmax (its own epilogue)
+  EPI_COUNT
+};
+
+// One 32 x 32 chunk of a specialised flavour: a = this lane's 32 accumulator columns, bias_c = the
+// chunk's bias values in shared memory (zeros without a bias), x = this lane's 32 bf16 values of
+// the row-shaped extra operand (EPI_RESIDUAL, EPI_DGELU).
+template <int kMode>
+__device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)[32], const uint4 (&x)[4],
+                                          const float* bias_c, uint8_t* stg, int lane, long long zoff,
+                                          int m_warp, int n0) {
+  float2 v[16];
+  const float2 al = splat2(p.alpha);
+  const float4* b4 = reinterpret_cast<const float4*>(bias_c);
+#pragma unroll
+  for (int j = 0; j < 8; j++) {
+    const float4 t = b4[j];
+    v[2 * j] = __ffma2_rn(make_float2(__uint_as_float(a[4 * j]), __uint_as_float(a[4 * j + 1])), al,
+                          make_float2(t.x, t.y));
+    v[2 * j + 1] = __ffma2_rn(make_float2(__uint_as_float(a[4 * j + 2]), __uint_as_float(a[4 * j + 3])), al,
+                              make_float2(t.z, t.w));
+  }
+  if constexpr (kMode == EPI_GELU_AUX)
+    stage_store_bf16(stg, lane, v, p.aux + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
+  if constexpr (kMode == EPI_GELU || kMode == EPI_GELU_AUX) {
+#pragma unroll
+    for (int j = 0; j < 16; j++) v[j] = gelu_fast2(v[j]);
+  }
+  if constexpr (kMode == EPI_DGELU) {
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      v[4 * j] = __fmul2_rn(v[4 * j], gelu_grad_fast2(bf162_to_f2(x[j].x)));
+      v[4 * j + 1] = __fmul2_rn(v[4 * j + 1], gelu_grad_fast2(bf162_to_f2(x[j].y)));
+      v[4 * j + 2] = __fmul2_rn(v[4 * j + 2], gelu_grad_fast2(bf162_to_f2(x[j].z)));
+      v[4 * j + 3] = __fmul2_rn(v[4 * j + 3], gelu_grad_fast2(bf162_to_f2(x[j].w)));
+    }
+  }
+  if constexpr (kMode == EPI_RESIDUAL) {
+#pragma unroll
+    for (int j = 0; j < 4; j++) {
+      v[4 * j] = __fadd2_rn(v[4 * j], bf162_to_f2(x[j].x));
+      v[4 * j + 1] = __fadd2_rn(v[4 * j + 1], bf162_to_f2(x[j].y));
+      v[4 * j + 2] = __fadd2_rn(v[4 * j + 2], bf162_to_f2(x[j].z));
+      v[4 * j + 3] = __fadd2_rn(v[4 * j + 3], bf162_to_f2(x[j].w));
+    }
+  }
+  if constexpr (kMode == EPI_F32)
+    stage_store_f32(stg, lane, v, reinterpret_cast<float*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok,
+                    p.accumulate);
+  else
+    stage_store_bf16(stg, lane, v, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
+}
+
 // ---- the kernel ---------------------------------------------------------------------------------
 // 10 warps are allocated registers as 12, which caps a thread at 168 registers
-template <bool kSoftmax, bool kPair>
+template <int kMode, bool kPair>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const TcParams p) {
+  constexpr bool kSoftmax = kMode == EPI_SOFTMAX;
+  constexpr bool kHasX = kMode == EPI_RESIDUAL || kMode == EPI_DGELU;
   extern __shared__ uint8_t smem_raw[];
   // tiles need 1024-byte alignment for the 128-byte swizzle pattern
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -568,6 +669,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int q = warp & 3;              // TMEM lane quarter this warp may read
     const int hsel = (warp - 2) >> 2;    // which of the two warps of the quarter
     uint8_t* stg = staging + (size_t)(warp - 2) * STAGING_BYTES;
+    float* bias_s = reinterpret_cast<float*>(stg + 2048);  // bias of this warp's columns, chunk by chunk
     uint32_t tile = 0;
     bool ok = true;
     for (int w = w_first; w < p.total_work && ok; w += w_step, tile++) {
@@ -578,14 +680,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int mt = r / p.n_tiles, nt = r - mt * p.n_tiles;
       const int zo = z / p.hdiv, zi = z - zo * p.hdiv;
       const uint32_t acc = tile & 1, use = tile >> 1;
-      if (!mbar_wait(smem_u32(&tfull_bar[acc]), use & 1, abort_flag, p.status)) { ok = false; break; }
-      tc_fence_after();
       const int m_warp = mt * mt_rows + (int)cta_rank * BM + q * 32;  // first row of this warp
       const int m = m_warp + lane;
       const long long zoff = zo * p.d_bo + zi * p.d_bi;
       const long long off0 = zoff + (long long)m * p.ldd;
       const int n_base = nt * p.bn;
       if constexpr (kSoftmax) {
+        if (!mbar_wait(smem_u32(&tfull_bar[acc]), use & 1, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
         // Scaled masked softmax over whole rows (one n-tile of at most 128 columns holds a row).
         // Each warp keeps its (up to) two 32-column chunks in registers; the two warps of a
         // quarter exchange row maxima and row sums through shared memory.
@@ -661,33 +763,63 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         continue;
       } else {
-      for (int cidx = hsel; cidx < p.bn / 32; cidx += 2) {
-        const int n0 = n_base + cidx * 32;
-        if (n0 >= p.N) break;  // uniform over the warp
-        float2 v[16];
-        tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256 + cidx * 32, v);
+      // Software pipeline over this warp's 32-column chunks (cidx = hsel, hsel + 2, ...): the
+      // TMEM read of the next chunk and the global loads it needs (GELU' argument or residual
+      // row) are issued before the current chunk is worked on.
+      const int nch = p.bn >> 6;
+      const bool row_ok = m < p.M;
+      const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
+      // the row-shaped extra operand, if any
+      const bf16* xsrc = kMode == EPI_GENERIC ? (p.act == 2 ? p.aux : p.residual)
+                       : kMode == EPI_DGELU ? p.aux : kMode == EPI_RESIDUAL ? p.residual : nullptr;
+      auto chunk_n0 = [&](int i) { return n_base + (hsel + 2 * i) * 32; };
+      auto chunk_ok = [&](int i) { return i < nch && chunk_n0(i) < p.N; };
+      auto prefetch_x = [&](int i, uint4 (&x)[4]) {
+        const int n0 = chunk_n0(i);
+        if ((kHasX && row_ok) || (kMode == EPI_GENERIC && xsrc && row_ok && p.vec_ok && n0 + 32 <= p.N)) {
+          const uint4* src = reinterpret_cast<const uint4*>(xsrc + off0 + n0);
+#pragma unroll
+          for (int j = 0; j < 4; j++) x[j] = src[j];
+        }
+      };
+      auto release_acc = [&]() {  // every TMEM read of this tile has returned
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) {
+          if (kPair && !leader) mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[acc]), 0));
+          else mbar_arrive(smem_u32(&tempty_bar[acc]));
+        }
+      };
+      auto process = [&](uint32_t (&a)[32], uint4 (&x)[4], int i, bool has_next) {
+        const int n0 = chunk_n0(i);
+        if constexpr (kMode != EPI_GENERIC) {
+          uint4 xc[4];
+          if constexpr (kHasX) {
+#pragma unroll
+            for (int j = 0; j < 4; j++) xc[j] = x[j];
+            // the extra operand of the next chunk travels while this chunk is worked on
+            if (has_next) prefetch_x(i + 1, x);
+          }
+          epi_chunk<kMode>(p, a, xc, bias_s + i * 32, stg, lane, zoff, m_warp, n0);
+          return;
+        }
         const long long off = off0 + n0;
         const bool fullv = p.vec_ok && (n0 + 32 <= p.N);
-        const bool row_ok = m < p.M;
+        float2 v[16];
+#pragma unroll
+        for (int j = 0; j < 16; j++) v[j] = make_float2(__uint_as_float(a[2 * j]), __uint_as_float(a[2 * j + 1]));
         if (p.alpha != 1.0f) {
           const float2 a2 = splat2(p.alpha);
 #pragma unroll
           for (int j = 0; j < 16; j++) v[j] = __fmul2_rn(v[j], a2);
         }
-        if (p.bias) {
-          if (n0 + 32 <= p.N) {
+        if (p.bias) {  // this warp's bias values were put in shared memory at the start of the tile
+          const float4* b4 = reinterpret_cast<const float4*>(bias_s + i * 32);
 #pragma unroll
-            for (int j = 0; j < 16; j += 2) {
-              const float4 b4 = *reinterpret_cast<const float4*>(p.bias + n0 + 2 * j);
-              v[j] = __fadd2_rn(v[j], make_float2(b4.x, b4.y));
-              v[j + 1] = __fadd2_rn(v[j + 1], make_float2(b4.z, b4.w));
-            }
-          } else {
-#pragma unroll
-            for (int j = 0; j < 16; j++) {
-              if (n0 + 2 * j < p.N) v[j].x += p.bias[n0 + 2 * j];
-              if (n0 + 2 * j + 1 < p.N) v[j].y += p.bias[n0 + 2 * j + 1];
-            }
+          for (int j = 0; j < 8; j++) {
+            const float4 t = b4[j];
+            v[2 * j] = __fadd2_rn(v[2 * j], make_float2(t.x, t.y));
+            v[2 * j + 1] = __fadd2_rn(v[2 * j + 1], make_float2(t.z, t.w));
           }
         }
         if (p.act == 1) {
@@ -697,12 +829,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         } else if (p.act == 2 && row_ok) {
           if (fullv) {
 #pragma unroll
-            for (int j = 0; j < 16; j += 4) {
-              const uint4 raw = *reinterpret_cast<const uint4*>(p.aux + off + 2 * j);
-              v[j] = __fmul2_rn(v[j], gelu_grad_fast2(bf162_to_f2(raw.x)));
-              v[j + 1] = __fmul2_rn(v[j + 1], gelu_grad_fast2(bf162_to_f2(raw.y)));
-              v[j + 2] = __fmul2_rn(v[j + 2], gelu_grad_fast2(bf162_to_f2(raw.z)));
-              v[j + 3] = __fmul2_rn(v[j + 3], gelu_grad_fast2(bf162_to_f2(raw.w)));
+            for (int j = 0; j < 4; j++) {
+              v[4 * j] = __fmul2_rn(v[4 * j], gelu_grad_fast2(bf162_to_f2(x[j].x)));
+              v[4 * j + 1] = __fmul2_rn(v[4 * j + 1], gelu_grad_fast2(bf162_to_f2(x[j].y)));
+              v[4 * j + 2] = __fmul2_rn(v[4 * j + 2], gelu_grad_fast2(bf162_to_f2(x[j].z)));
+              v[4 * j + 3] = __fmul2_rn(v[4 * j + 3], gelu_grad_fast2(bf162_to_f2(x[j].w)));
             }
           } else {
 #pragma unroll
@@ -715,14 +846,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         }
         if (p.residual && row_ok) {
-          if (fullv) {
+          if (fullv && p.act != 2) {
 #pragma unroll
-            for (int j = 0; j < 16; j += 4) {
-              const uint4 raw = *reinterpret_cast<const uint4*>(p.residual + off + 2 * j);
-              v[j] = __fadd2_rn(v[j], bf162_to_f2(raw.x));
-              v[j + 1] = __fadd2_rn(v[j + 1], bf162_to_f2(raw.y));
-              v[j + 2] = __fadd2_rn(v[j + 2], bf162_to_f2(raw.z));
-              v[j + 3] = __fadd2_rn(v[j + 3], bf162_to_f2(raw.w));
+            for (int j = 0; j < 4; j++) {
+              v[4 * j] = __fadd2_rn(v[4 * j], bf162_to_f2(x[j].x));
+              v[4 * j + 1] = __fadd2_rn(v[4 * j + 1], bf162_to_f2(x[j].y));
+              v[4 * j + 2] = __fadd2_rn(v[4 * j + 2], bf162_to_f2(x[j].z));
+              v[4 * j + 3] = __fadd2_rn(v[4 * j + 3], bf162_to_f2(x[j].w));
             }
           } else {
 #pragma unroll
@@ -732,19 +862,41 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             }
           }
         }
+        // the extra operand of the next chunk travels while this chunk is stored
+        if (has_next) prefetch_x(i + 1, x);
         if (p.d_fp32)
           stage_store_f32(stg, lane, v, reinterpret_cast<float*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N,
                           p.vec_ok, p.accumulate);
         else
           stage_store_bf16(stg, lane, v, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N,
                            p.vec_ok);
+      };
+      // before the accumulator is ready: bias values of this warp's columns to shared memory,
+      // first chunk's extra operand on its way
+      uint32_t a0[32];
+      uint4 x[4];
+      const bool c0ok = chunk_ok(0);
+      if (kMode != EPI_GENERIC || p.bias) {
+        for (int i = 0; i < nch; i++) {
+          const int n = chunk_n0(i) + lane;
+          bias_s[i * 32 + lane] = (p.bias && n < p.N) ? p.bias[n] : 0.f;
+        }
+        __syncwarp();
       }
-      // hand the accumulator back to the MMA warp
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) {
-        if (kPair && !leader) mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[acc]), 0));
-        else mbar_arrive(smem_u32(&tempty_bar[acc]));
+      if (c0ok) prefetch_x(0, x);
+      if (!mbar_wait(smem_u32(&tfull_bar[acc]), use & 1, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      if (c0ok) {
+        for (int i = 0;; i++) {
+          const bool v1 = chunk_ok(i + 1);
+          tc_ld32_issue(trow + (hsel + 2 * i) * 32, a0);
+          tc_ld32_wait(a0);
+          if (!v1) release_acc();
+          process(a0, x, i, v1);
+          if (!v1) break;
+        }
+      } else {
+        release_acc();
       }
       }
     }
@@ -895,8 +1047,9 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   static const bool single_cta = getenv("MSLT_GEMM_SINGLE_CTA") && atoi(getenv("MSLT_GEMM_SINGLE_CTA")) == 1;
   // Measured: the pair wins for row-contiguous (MN-major) operands and for deep contractions, and is
   // on par or slightly behind for shallow k-contiguous products, which are bound by their epilogue.
+  static const bool force_pair = getenv("MSLT_GEMM_SINGLE_CTA") && atoi(getenv("MSLT_GEMM_SINGLE_CTA")) == 2;
   bool pair = !single_cta && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0 &&
-              (p.a_mn || p.b_mn || d.K >= 2048);
+              (force_pair || p.a_mn || p.b_mn || d.K >= 2048);
   // share of the SMs that the last wave of tiles keeps busy
   auto wave_eff = [](long long work, int units_) {
     const long long waves = (work + units_ - 1) / units_;
@@ -949,6 +1102,8 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   const int book_bytes = 256 + (d.act == 3 ? 64 + 2 * NUM_EPI_WARPS * 32 * 4 : 0);
   int stages = (smem_optin - NUM_EPI_WARPS * STAGING_BYTES - 1024 - book_bytes) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
+  static const int stage_cap = getenv("MSLT_GEMM_STAGES") ? atoi(getenv("MSLT_GEMM_STAGES")) : 0;
+  if (stage_cap >= 2 && stages > stage_cap) stages = stage_cap;
   if (stages < 2) { snprintf(err, 256, "gemm: not enough shared memory"); return MSLT_ERR_CUDA; }
   p.stages = stages;
   const size_t smem_bytes = (size_t)stages * stage_bytes + NUM_EPI_WARPS * STAGING_BYTES + 1024 + book_bytes;
@@ -981,41 +1136,58 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
             ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
 
+  // epilogue flavour: a specialised kernel where one fits, the general one otherwise
+  int mode = EPI_GENERIC;
+  const bool x_ok = p.vec_ok && d.N % 32 == 0;  // row-shaped extra operands are read 16 bytes at a time
+  if (d.act == 3) mode = EPI_SOFTMAX;
+  else if (d.d_fp32) { if (d.act == 0 && !d.residual) mode = EPI_F32; }
+  else if (d.act == 0 && !d.residual) mode = EPI_STORE;
+  else if (d.act == 0 && d.residual && x_ok) mode = EPI_RESIDUAL;
+  else if (d.act == 1 && !d.residual) mode = d.aux ? EPI_GELU_AUX : EPI_GELU;
+  else if (d.act == 2 && d.aux && !d.residual && x_ok) mode = EPI_DGELU;
+  static const bool generic_only = getenv("MSLT_GEMM_GENERIC_EPILOGUE") && atoi(getenv("MSLT_GEMM_GENERIC_EPILOGUE")) == 1;
+  if (generic_only && mode != EPI_SOFTMAX) mode = EPI_GENERIC;
+
+  typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const TcParams);
+  static const KernelFn kernels[EPI_COUNT][2] = {
+      {gemm_tc_kernel<EPI_STORE, false>, gemm_tc_kernel<EPI_STORE, true>},
+      {gemm_tc_kernel<EPI_RESIDUAL, false>, gemm_tc_kernel<EPI_RESIDUAL, true>},
+      {gemm_tc_kernel<EPI_GELU, false>, gemm_tc_kernel<EPI_GELU, true>},
+      {gemm_tc_kernel<EPI_GELU_AUX, false>, gemm_tc_kernel<EPI_GELU_AUX, true>},
+      {gemm_tc_kernel<EPI_DGELU, false>, gemm_tc_kernel<EPI_DGELU, true>},
+      {gemm_tc_kernel<EPI_F32, false>, gemm_tc_kernel<EPI_F32, true>},
+      {gemm_tc_kernel<EPI_GENERIC, false>, gemm_tc_kernel<EPI_GENERIC, true>},
+      {gemm_tc_kernel<EPI_SOFTMAX, false>, nullptr}};
   static bool attr_set = false;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
-    if (e == cudaSuccess)
-      e = cudaFuncSetAttribute(gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
-    if (e != cudaSuccess) { snprintf(err, 256, "gemm: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+    for (int mo = 0; mo < EPI_COUNT; mo++)
+      for (int pr = 0; pr < 2; pr++) {
+        if (!kernels[mo][pr]) continue;
+        cudaError_t e = cudaFuncSetAttribute((const void*)kernels[mo][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+        if (e != cudaSuccess) { snprintf(err, 256, "gemm: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+      }
     attr_set = true;
   }
+  const KernelFn fn = kernels[mode][pair ? 1 : 0];
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.dynamicSmemBytes = smem_bytes;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
   if (pair) {
     const int clusters = p.total_work < units ? p.total_work : units;
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof(cfg));
     cfg.gridDim = dim3(2 * clusters);
-    cfg.blockDim = dim3(NUM_THREADS);
-    cfg.dynamicSmemBytes = smem_bytes;
-    cfg.stream = st;
-    cudaLaunchAttribute attr[1];
     attr[0].id = cudaLaunchAttributeClusterDimension;
     attr[0].val.clusterDim.x = 2;
     attr[0].val.clusterDim.y = 1;
     attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    cudaError_t e = cudaLaunchKernelEx(&cfg, gemm_tc_kernel<false, true>, ma.map, mb.map, p);
-    if (e != cudaSuccess) { snprintf(err, 256, "gemm: cluster launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
-    return 0;
+  } else {
+    cfg.gridDim = dim3(p.total_work < num_sms ? p.total_work : num_sms);
   }
-  const int grid = p.total_work < num_sms ? p.total_work : num_sms;
-  if (d.act == 3)
-    gemm_tc_kernel<true, false><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
-  else
-    gemm_tc_kernel<false, false><<<grid, NUM_THREADS, smem_bytes, st>>>(ma.map, mb.map, p);
-  cudaError_t e = cudaGetLastError();
+  cudaError_t e = cudaLaunchKernelEx(&cfg, fn, ma.map, mb.map, p);
   if (e != cudaSuccess) { snprintf(err, 256, "gemm: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
   return 0;
 }
