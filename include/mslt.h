@@ -280,6 +280,19 @@ int mslt_op_softmax_bwd(int32_t dtype, void* d_dp, const void* d_probs, int32_t 
 int mslt_op_colsum(int32_t dtype, const void* d_x, int64_t ld, int32_t rows, int32_t N, float* d_out,
                    void* cuda_stream, int32_t sync);
 
+/* Attention of one encoder layer in a single kernel (the paper defers the encoder to BERT,
+ * Section 4.1: scaled dot-product attention with a key-padding mask), bf16 only, head width 64,
+ * 1 <= S <= 128:  probs[b,h,i,:] = softmax over the valid keys j < d_seq_lens[b] (NULL: all S) of
+ * scale * q_i . k_j, masked probabilities exactly 0;  ctx[b,i,h,:] = sum_j probs[b,h,i,j] v_j with
+ * probs rounded to bf16 first.  d_qkv: device, [B*S, 3*heads*64] row-major, columns = queries |
+ * keys | values, head h in columns h*64.. of each; d_probs: device, [B, heads, S, S] or NULL (not
+ * written); d_ctx: device, [B*S, heads*64].  All buffers 16-byte aligned and caller-owned.
+ * d_status: device int32 that receives bit 0 if a bounded wait ran out (returned as
+ * MSLT_ERR_DEVICE when sync != 0).  Other shapes are rejected with MSLT_ERR_ARG. */
+int mslt_op_attention(const void* d_qkv, void* d_probs, void* d_ctx, const int32_t* d_seq_lens, int32_t B,
+                      int32_t S, int32_t heads, float scale, int32_t* d_status, void* cuda_stream,
+                      int32_t sync);
+
 /*
  * mslt_op_cross_entropy without any device allocation by anybody.  (The paper has no counterpart
  * of this call; it exists for the integration below.)

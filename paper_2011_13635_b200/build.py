@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmslt.so")
-SOURCES = ["mslt.cu", "gemm.cu", "gemm_simt.cu", "gemm_tc.cu", "kernels.cu", "ops.cu"]
+SOURCES = ["mslt.cu", "gemm.cu", "gemm_simt.cu", "gemm_tc.cu", "attn_tc.cu", "kernels.cu", "ops.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

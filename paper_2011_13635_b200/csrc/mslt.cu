@@ -306,6 +306,28 @@ bool getenv_cuda_cores() {
   return v;
 }
 
+// true when attention runs as two batched products with a separate softmax (for A/B measurements)
+bool getenv_unfused_attention() {
+  static const bool v = getenv("MSLT_UNFUSED_ATTENTION") && atoi(getenv("MSLT_UNFUSED_ATTENTION")) == 1;
+  return v;
+}
+
+// scores, masked softmax and context of one layer in one kernel (bf16, head width 64, S <= 128)
+int run_attention(mslt_ctx* c, const void* qkv, void* probs, void* ctx, const int* seq_lens, int B, int S,
+                  int A, int d, float scale) {
+  char err[256] = "";
+  const bool prof = c->profile && c->prec.size() * 2 + 2 <= c->pev.size();
+  if (prof) cudaEventRecord(c->pev[2 * c->prec.size()], c->st);
+  int rc = attn_fwd_launch(qkv, probs, ctx, seq_lens, B, S, A, d, scale, c->ws.scalars, c->st, err);
+  if (prof) {
+    cudaEventRecord(c->pev[2 * c->prec.size() + 1], c->st);
+    c->prec.push_back({1, 4.0 * B * A * (double)S * S * d});
+  }
+  if (rc) return fail(rc, "%s", err);
+  c->launches++;
+  return 0;
+}
+
 int run_gemm(mslt_ctx* c, const mslt_gemm_desc& d) {
   if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) return 0;
   char err[256] = "";
@@ -395,28 +417,33 @@ int layer_forward(mslt_ctx* c, int l, const void* x, LayerBuf& b, void* out, boo
   const float scale = 1.0f / sqrtf((float)d);
   TRY(linear_fwd(c, x, T, H, toff(c, l, "qkv.weight"), toff(c, l, "qkv.bias"), 3 * H, b.qkv, 0,
                  nullptr, nullptr));
-  {  // scores[b,h,i,j] = q_i . k_j / sqrt(d)
-    Lin g(c, S, S, d);
-    g.d.batch = B * A; g.d.hdiv = A; g.d.alpha = scale;
-    g.d.A = b.qkv; g.d.a_rs = 3 * H; g.d.a_ks = 1; g.d.a_bo = (int64_t)S * 3 * H; g.d.a_bi = d;
-    g.d.B = b.qkv + (int64_t)H * E; g.d.b_rs = 3 * H; g.d.b_ks = 1; g.d.b_bo = (int64_t)S * 3 * H; g.d.b_bi = d;
-    g.d.D = b.p; g.d.ldd = S; g.d.d_bo = (int64_t)A * S * S; g.d.d_bi = (int64_t)S * S;
-    // rows of at most 128 keys fit one tile: the tensor-core kernel applies the masked softmax
-    // in its epilogue and writes probabilities straight away
-    const bool fused = c->bf && S <= 128 && !getenv_cuda_cores();
-    if (fused) { g.d.act = 3; g.d.seq_lens = seq_lens; }
-    TRY(run_gemm(c, g.d));
-    if (!fused)
-      KL(PC_SOFTMAX_FWD, 2.0 * B * A * S * S * c->esz,
-         launch_softmax_fwd(c->bf, b.p, b.p, seq_lens, B * A * S, S, A * S, 1.0f, c->st));
-  }
-  {  // context[b,i,h,:] = sum_j p[b,h,i,j] v_j
-    Lin g(c, S, d, S);
-    g.d.batch = B * A; g.d.hdiv = A;
-    g.d.A = b.p; g.d.a_rs = S; g.d.a_ks = 1; g.d.a_bo = (int64_t)A * S * S; g.d.a_bi = (int64_t)S * S;
-    g.d.B = b.qkv + (int64_t)2 * H * E; g.d.b_rs = 1; g.d.b_ks = 3 * H; g.d.b_bo = (int64_t)S * 3 * H; g.d.b_bi = d;
-    g.d.D = b.c; g.d.ldd = H; g.d.d_bo = (int64_t)S * H; g.d.d_bi = d;
-    TRY(run_gemm(c, g.d));
+  if (c->bf && S <= 128 && d == 64 && !getenv_cuda_cores() && !getenv_unfused_attention()) {
+    // the probabilities go to memory only where the backward pass will read them
+    TRY(run_attention(c, b.qkv, save ? b.p : nullptr, b.c, seq_lens, B, S, A, d, scale));
+  } else {
+    {  // scores[b,h,i,j] = q_i . k_j / sqrt(d)
+      Lin g(c, S, S, d);
+      g.d.batch = B * A; g.d.hdiv = A; g.d.alpha = scale;
+      g.d.A = b.qkv; g.d.a_rs = 3 * H; g.d.a_ks = 1; g.d.a_bo = (int64_t)S * 3 * H; g.d.a_bi = d;
+      g.d.B = b.qkv + (int64_t)H * E; g.d.b_rs = 3 * H; g.d.b_ks = 1; g.d.b_bo = (int64_t)S * 3 * H; g.d.b_bi = d;
+      g.d.D = b.p; g.d.ldd = S; g.d.d_bo = (int64_t)A * S * S; g.d.d_bi = (int64_t)S * S;
+      // rows of at most 128 keys fit one tile: the tensor-core kernel applies the masked softmax
+      // in its epilogue and writes probabilities straight away
+      const bool fused = c->bf && S <= 128 && !getenv_cuda_cores();
+      if (fused) { g.d.act = 3; g.d.seq_lens = seq_lens; }
+      TRY(run_gemm(c, g.d));
+      if (!fused)
+        KL(PC_SOFTMAX_FWD, 2.0 * B * A * S * S * c->esz,
+           launch_softmax_fwd(c->bf, b.p, b.p, seq_lens, B * A * S, S, A * S, 1.0f, c->st));
+    }
+    {  // context[b,i,h,:] = sum_j p[b,h,i,j] v_j
+      Lin g(c, S, d, S);
+      g.d.batch = B * A; g.d.hdiv = A;
+      g.d.A = b.p; g.d.a_rs = S; g.d.a_ks = 1; g.d.a_bo = (int64_t)A * S * S; g.d.a_bi = (int64_t)S * S;
+      g.d.B = b.qkv + (int64_t)2 * H * E; g.d.b_rs = 1; g.d.b_ks = 3 * H; g.d.b_bo = (int64_t)S * 3 * H; g.d.b_bi = d;
+      g.d.D = b.c; g.d.ldd = H; g.d.d_bo = (int64_t)S * H; g.d.d_bi = d;
+      TRY(run_gemm(c, g.d));
+    }
   }
   TRY(linear_fwd(c, b.c, T, H, toff(c, l, "out.weight"), toff(c, l, "out.bias"), H, b.z1, 0, nullptr, x));
   KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_ln_fwd(c->bf, b.z1, Wv(c, toff(c, l, "ln1.gamma")), Wv(c, toff(c, l, "ln1.beta")), b.y,

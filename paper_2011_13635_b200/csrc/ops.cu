@@ -6,6 +6,7 @@
 
 #include "../../include/mslt.h"
 #include "common.cuh"
+#include "gemm.h"
 #include "kernels.h"
 
 using namespace mslt;
@@ -190,6 +191,31 @@ int mslt_op_layernorm_bwd(int32_t dtype, const void* d_dy, const void* d_z, cons
   cudaStream_t st = (cudaStream_t)cuda_stream;
   launch_ln_bwd(dtype == 1, d_dy, d_z, d_stats, d_gamma, d_dz, d_dgamma, d_dbeta, rows, H, st);
   return finish_op("layernorm_bwd", st, sync);
+}
+
+int mslt_op_attention(const void* d_qkv, void* d_probs, void* d_ctx, const int32_t* d_seq_lens, int32_t B,
+                      int32_t S, int32_t heads, float scale, int32_t* d_status, void* cuda_stream,
+                      int32_t sync) {
+  if (!d_qkv || !d_ctx || !d_status) return op_fail(MSLT_ERR_ARG, "attention: null pointer");
+  if (((uintptr_t)d_qkv | (uintptr_t)d_ctx | (uintptr_t)d_probs) & 15)
+    return op_fail(MSLT_ERR_ARG, "attention: buffers must be 16-byte aligned");
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1)
+    return op_fail(MSLT_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char err[256] = "";
+  int rc = attn_fwd_launch(d_qkv, d_probs, d_ctx, d_seq_lens, B, S, heads, 64, scale, d_status, st, err);
+  if (rc) return op_fail(rc, "%s", err);
+  if (sync) {
+    rc = finish_op("attention", st, 1);
+    if (rc) return rc;
+    int h = 0;
+    if (cudaMemcpy(&h, d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return op_fail(MSLT_ERR_CUDA, "attention: reading the status word failed");
+    if (h & 1) return op_fail(MSLT_ERR_DEVICE, "attention: a bounded wait ran out on the device");
+    return 0;
+  }
+  return finish_op("attention", st, 0);
 }
 
 int mslt_op_softmax(int32_t dtype, const void* d_scores, void* d_probs, const int32_t* d_seq_lens,

@@ -154,3 +154,56 @@ def test_op_argument_checks():
     with pytest.raises(Bd.MsltError) as ei:
         Bd.mslt_op_softmax(s, s, None, 4, 1.0, _stream())
     assert ei.value.code == -1
+
+
+@pytest.mark.parametrize("B,S,A,masked", [(2, 128, 2, False), (3, 128, 12, True), (2, 100, 3, True),
+                                          (5, 64, 2, True), (1, 24, 1, False), (37, 128, 12, True)])
+@pytest.mark.parametrize("want_probs", [True, False], ids=["probs", "noprobs"])
+def test_fused_attention_matches_oracle(B, S, A, masked, want_probs):
+    """Scores, masked softmax and context in one kernel against the oracle's definition
+    (einsum, masked_softmax, einsum) on the same bf16-rounded inputs."""
+    import math
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    d, H = 64, A * 64
+    rng = np.random.default_rng(B * 1000 + S + A)
+    qkv = torch.from_numpy((rng.standard_normal((B * S, 3 * H)) * 1.5).astype(np.float32)).cuda().bfloat16()
+    lens = rng.integers(1, S + 1, size=B).astype(np.int32) if masked else np.full(B, S, np.int32)
+    if masked:
+        lens[0] = S
+        lens[-1] = 1 if B > 1 else S
+    d_lens = torch.from_numpy(lens).cuda() if masked else None
+    probs = torch.full((B, A, S, S), 7.0, device="cuda", dtype=torch.bfloat16) if want_probs else None
+    ctx = torch.full((B * S, H), 7.0, device="cuda", dtype=torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scale = 1.0 / math.sqrt(d)
+    for _ in range(2):   # twice: the second call must not depend on what the first left behind
+        Bd.mslt_op_attention(qkv, probs, ctx, d_lens, B, S, A, scale, status, _stream())
+    assert int(status.item()) == 0
+    x = qkv.float().cpu().numpy().astype(np.float64).reshape(B, S, 3, A, d)
+    q, k, v = (x[:, :, i].transpose(0, 2, 1, 3) for i in range(3))          # [B, A, S, d]
+    p_ref = O.masked_softmax(np.einsum("bhid,bhjd->bhij", q, k) * scale, lens)
+    c_ref = np.einsum("bhij,bhjd->bhid", p_ref, v).transpose(0, 2, 1, 3).reshape(B * S, H)
+    if want_probs:
+        got = probs.float().cpu().numpy()
+        assert np.abs(got - p_ref).max() < 6e-3                              # bf16 resolution at p <= 1
+        for b in range(B):
+            assert not got[b, :, :, lens[b]:].any()                          # masked keys exactly 0
+    # rows at padded query positions are unspecified: compare valid rows only
+    got = ctx.float().cpu().numpy().reshape(B, S, H)
+    ref = c_ref.reshape(B, S, H)
+    for b in range(B):
+        err = np.abs(got[b, :lens[b]] - ref[b, :lens[b]]).max()
+        assert err / np.abs(ref[b, :lens[b]]).max() < 1.5e-2, (b, err)
+
+
+def test_fused_attention_rejects_other_shapes():
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    qkv = torch.zeros((256, 192), device="cuda", dtype=torch.bfloat16)
+    ctx = torch.zeros((256, 64), device="cuda", dtype=torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(Bd.MsltError):
+        Bd.mslt_op_attention(qkv, None, ctx, None, 1, 256, 1, 0.125, status, _stream())
+    with pytest.raises(Bd.MsltError):
+        Bd.mslt_op_attention(qkv, None, ctx, None, 0, 128, 1, 0.125, status, _stream())
