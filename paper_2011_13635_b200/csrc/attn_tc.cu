@@ -4,14 +4,17 @@
 // when the backward pass needs them.  Unfused, the two products are bound by HBM traffic (about
 // 32 flop per byte at head width 64); fused, a layer's attention reads Q, K, V once and writes the
 // context once.
-//   warp 0   : TMA producer: the Q, K and V tiles of a (sequence, head) item, three items deep.
+//   warp 0   : TMA producer: the Q, K and V tiles of a (sequence, head) item, four items deep.
 //   warp 1   : one thread issues tcgen05.mma: S = Q K^T into one of two 128-column accumulators,
-//              and, once the epilogue warps have put P into shared memory, C = P V.
-//   warps 2-9: scaled masked softmax on the accumulator (two warps per 32-row quarter, each half
-//              of the columns; row maxima and sums exchanged through shared memory), P written as
-//              the bf16 A operand of the second product (128-byte swizzle, by hand) and, for
-//              layers that run backward, to global memory; then the context tile is read back
-//              from tensor memory and stored.
+//              and, once a softmax group has put P into shared memory, C = P V into one of two
+//              64-column accumulators.
+//   warps 2-5, 6-9: two softmax groups that take alternate items, so that the exponentials of one
+//              item overlap the second product and the stores of the other.  A thread owns one
+//              query row: it reads the row's 128 scores from tensor memory, applies scale and
+//              mask, forms max, exponentials and sum with no exchange between threads, writes the
+//              normalised row as the bf16 A operand of the second product (128-byte swizzle, by
+//              hand, over the item's dead Q and K tiles) and, for layers that run backward, to
+//              global memory; then reads the context tile back from tensor memory and stores it.
 // P is rounded to bf16 before the second product, exactly as when it is stored and read back.
 // Every wait is bounded: when one runs out the CTA raises a status bit, drains and returns.
 #include <atomic>
@@ -23,13 +26,13 @@ namespace mslt {
 
 namespace {
 
-constexpr int AT_STAGES = 3;
+constexpr int AT_STAGES = 4;
 constexpr int AT_TILE_BYTES = 128 * 64 * 2;          // one of Q, K, V: 16 KB
 constexpr int AT_STAGE_BYTES = 3 * AT_TILE_BYTES;    // 48 KB
-constexpr int AT_P_BYTES = 128 * 128 * 2;            // probabilities as an MMA operand: 32 KB
 constexpr int AT_STAGING = 2048;                     // per epilogue warp
 constexpr uint32_t AT_TMEM_COLS = 512;
-constexpr uint32_t AT_O_COL = 256;                   // context accumulator after the two score buffers
+constexpr uint32_t AT_O_COL = 256;                   // two context accumulators after the two score buffers
+constexpr int AT_GROUP_WARPS = 4;                    // warps of a softmax group
 
 struct AttnParams {
   int S, heads, items;
@@ -46,25 +49,27 @@ struct AttnParams {
   uint32_t idesc_s, idesc_o;
 };
 
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* p_smem = smem + AT_STAGES * AT_STAGE_BYTES;
-  uint8_t* staging = p_smem + AT_P_BYTES;
+  uint8_t* staging = smem + AT_STAGES * AT_STAGE_BYTES;
   uint64_t* bars = (uint64_t*)(staging + NUM_EPI_WARPS * AT_STAGING);
   uint64_t* full_bar = bars;                 // [AT_STAGES] tiles of an item have landed
   uint64_t* empty_bar = bars + AT_STAGES;    // [AT_STAGES] both products of an item have read them
   uint64_t* sfull_bar = bars + 2 * AT_STAGES;      // [2] scores complete
   uint64_t* sempty_bar = bars + 2 * AT_STAGES + 2; // [2] scores read by every epilogue warp
-  uint64_t* pready_bar = bars + 2 * AT_STAGES + 4; // probabilities in shared memory
-  uint64_t* ofull_bar = bars + 2 * AT_STAGES + 5;  // context complete
-  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * AT_STAGES + 6);
+  uint64_t* pready_bar = bars + 2 * AT_STAGES + 4; // [2] probabilities of a group's item in shared memory
+  uint64_t* ofull_bar = bars + 2 * AT_STAGES + 6;  // [2] context of a group's item complete
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * AT_STAGES + 8);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
-  volatile int* xflag = (volatile int*)((uint8_t*)bars + 256);
-  float* xmax = (float*)((uint8_t*)bars + 256 + 64);
-  float* xsum = xmax + NUM_EPI_WARPS * 32;
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
@@ -74,13 +79,12 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
     }
     for (int a = 0; a < 2; a++) {
       mbar_init(smem_u32(&sfull_bar[a]), 1);
-      mbar_init(smem_u32(&sempty_bar[a]), NUM_EPI_WARPS);
+      mbar_init(smem_u32(&sempty_bar[a]), AT_GROUP_WARPS);
+      mbar_init(smem_u32(&pready_bar[a]), AT_GROUP_WARPS);
+      mbar_init(smem_u32(&ofull_bar[a]), 1);
     }
-    mbar_init(smem_u32(pready_bar), NUM_EPI_WARPS);
-    mbar_init(smem_u32(ofull_bar), 1);
     *abort_flag = 0;
     *reinterpret_cast<volatile long long*>(abort_flag + 1) = p.wait_limit;
-    for (int i = 0; i < NUM_EPI_WARPS; i++) xflag[i] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
@@ -133,26 +137,25 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   } else if (warp == 1 && lane == 0) {
     // ------------------------------- MMA issuer -------------------------------
     bool ok = true;
-    const uint32_t p_desc_lo = (uint32_t)make_smem_desc(smem_u32(p_smem), 16);
-    const uint32_t hi_k = (uint32_t)(make_smem_desc(0, 16) >> 32);
-    const uint32_t hi_mn = (uint32_t)(make_smem_desc(0, 64 * BK * 2) >> 32);
-    const uint32_t lbo_mn_lo = (uint32_t)make_smem_desc(0, 64 * BK * 2);  // low word carries the LBO field
-    auto issue_pv = [&](int j) {  // C = P V of item j
-      const uint32_t s = (uint32_t)(j % AT_STAGES);
-      const uint32_t sv = smem_u32(smem + (size_t)s * AT_STAGE_BYTES + 2 * AT_TILE_BYTES);
-      const uint32_t v_lo = lbo_mn_lo | ((sv & 0x3FFFFu) >> 4);
+    const uint32_t hi = (uint32_t)(make_smem_desc(0, 16) >> 32);           // same for both operand forms
+    const uint32_t lbo_mn_lo = (uint32_t)make_smem_desc(0, 64 * BK * 2);   // low word carries the LBO field
+    auto issue_pv = [&](int j) {  // C = P V of item j; P lies over the item's Q and K tiles
+      const uint32_t s = (uint32_t)(j % AT_STAGES), g = (uint32_t)j & 1;
+      const uint32_t sq = smem_u32(smem + (size_t)s * AT_STAGE_BYTES);
+      const uint32_t p_lo = (uint32_t)make_smem_desc(sq, 16);
+      const uint32_t v_lo = lbo_mn_lo | (((sq + 2 * AT_TILE_BYTES) & 0x3FFFFu) >> 4);
       uint32_t accum = 0;
 #pragma unroll
       for (int kb = 0; kb < 2; kb++)
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; k++) {
-          const uint64_t ad = ((uint64_t)hi_k << 32) | (p_desc_lo + kb * (128 * 128 / 16) + k * (UMMA_K * 2 / 16));
-          const uint64_t bd = ((uint64_t)hi_mn << 32) | (v_lo + kb * (AT_TILE_BYTES / 2 / 16) + k * (UMMA_K * 128 / 16));
-          tc_mma(tmem_base + AT_O_COL, ad, bd, p.idesc_o, accum);
+          const uint64_t ad = ((uint64_t)hi << 32) | (p_lo + kb * (AT_TILE_BYTES / 16) + k * (UMMA_K * 2 / 16));
+          const uint64_t bd = ((uint64_t)hi << 32) | (v_lo + kb * (AT_TILE_BYTES / 2 / 16) + k * (UMMA_K * 128 / 16));
+          tc_mma(tmem_base + AT_O_COL + g * 64, ad, bd, p.idesc_o, accum);
           accum = 1;
         }
-      tc_commit(smem_u32(ofull_bar));
-      tc_commit(smem_u32(&empty_bar[s]));  // Q, K, V of the item are no longer needed
+      tc_commit(smem_u32(&ofull_bar[g]));
+      tc_commit(smem_u32(&empty_bar[s]));  // the item's tiles are no longer needed
     };
     for (int i = 0; i < n_my && ok; i++) {
       const uint32_t s = (uint32_t)(i % AT_STAGES), round = (uint32_t)(i / AT_STAGES);
@@ -164,19 +167,21 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       const uint32_t q_lo = (uint32_t)make_smem_desc(sq, 16), k_lo = (uint32_t)make_smem_desc(sq + AT_TILE_BYTES, 16);
 #pragma unroll
       for (int k = 0; k < BK / UMMA_K; k++) {
-        const uint64_t ad = ((uint64_t)hi_k << 32) | (q_lo + k * (UMMA_K * 2 / 16));
-        const uint64_t bd = ((uint64_t)hi_k << 32) | (k_lo + k * (UMMA_K * 2 / 16));
+        const uint64_t ad = ((uint64_t)hi << 32) | (q_lo + k * (UMMA_K * 2 / 16));
+        const uint64_t bd = ((uint64_t)hi << 32) | (k_lo + k * (UMMA_K * 2 / 16));
         tc_mma(tmem_base + b * 128, ad, bd, p.idesc_s, k > 0 ? 1u : 0u);
       }
       tc_commit(smem_u32(&sfull_bar[b]));
-      if (i > 0) {  // the previous item's probabilities should be ready by now
-        if (!mbar_wait(smem_u32(pready_bar), (uint32_t)(i - 1) & 1, abort_flag, p.status)) { ok = false; break; }
+      if (i > 0) {  // the previous item's probabilities: its group has been at work since S(i-1)
+        const uint32_t g = (uint32_t)(i - 1) & 1, guse = (uint32_t)(i - 1) >> 1;
+        if (!mbar_wait(smem_u32(&pready_bar[g]), guse & 1, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         issue_pv(i - 1);
       }
     }
     if (ok && n_my > 0) {
-      if (mbar_wait(smem_u32(pready_bar), (uint32_t)(n_my - 1) & 1, abort_flag, p.status)) {
+      const uint32_t g = (uint32_t)(n_my - 1) & 1, guse = (uint32_t)(n_my - 1) >> 1;
+      if (mbar_wait(smem_u32(&pready_bar[g]), guse & 1, abort_flag, p.status)) {
         tc_fence_after();
         issue_pv(n_my - 1);
       } else {
@@ -190,92 +195,100 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
       while (now_cycles() - t0 < 2000000ll) {}
     }
   } else if (warp >= 2) {
-    // ------------------------------- softmax and context epilogue -------------------------------
+    // ------------------------------- softmax groups -------------------------------
     const int q = warp & 3;              // TMEM lane quarter this warp may read
-    const int hsel = (warp - 2) >> 2;    // which of the two warps of the quarter
+    const int g = (warp - 2) >> 2;       // softmax group: items g, g + 2, ...
     uint8_t* stg = staging + (size_t)(warp - 2) * AT_STAGING;
-    const int me = q * 2 + hsel, other = q * 2 + (hsel ^ 1);
-    const int r = q * 32 + lane;         // row of the item this lane owns
+    const int r = q * 32 + lane;         // query row this thread owns
     bool ok = true;
-    for (int i = 0; i < n_my && ok; i++) {
+    for (int i = g; i < n_my && ok; i += 2) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
       const int zo = w / p.heads, zi = w - zo * p.heads;
-      const uint32_t b = (uint32_t)i & 1, use = (uint32_t)i >> 1;
+      const uint32_t s = (uint32_t)(i % AT_STAGES), use = (uint32_t)i >> 1;
       int len = p.seq_lens ? p.seq_lens[zo] : p.S;
       len = min(max(len, 1), p.S);
-      if (!mbar_wait(smem_u32(&sfull_bar[b]), use & 1, abort_flag, p.status)) { ok = false; break; }
+      if (!mbar_wait(smem_u32(&sfull_bar[g]), use & 1, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      const int c0 = hsel, c1 = hsel + 2;  // this warp's two 32-column chunks
-      float2 v0[16], v1[16];
-      float mx = -INFINITY;
-      const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + b * 128;
-      tc_ld32(trow + c0 * 32, v0);
-      tc_ld32(trow + c1 * 32, v1);
+      float2 v[4][16];  // the row's 128 scores, then its probabilities
+      const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g * 128;
 #pragma unroll
-      for (int j = 0; j < 16; j++) {
-        v0[j].x = (c0 * 32 + 2 * j < len) ? v0[j].x * p.scale : -INFINITY;
-        v0[j].y = (c0 * 32 + 2 * j + 1 < len) ? v0[j].y * p.scale : -INFINITY;
-        v1[j].x = (c1 * 32 + 2 * j < len) ? v1[j].x * p.scale : -INFINITY;
-        v1[j].y = (c1 * 32 + 2 * j + 1 < len) ? v1[j].y * p.scale : -INFINITY;
-        mx = fmaxf(mx, fmaxf(fmaxf(v0[j].x, v0[j].y), fmaxf(v1[j].x, v1[j].y)));
-      }
+      for (int c = 0; c < 4; c++) tc_ld32(trow + c * 32, v[c]);
       // the scores are in registers: hand the accumulator back
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(&sempty_bar[b]));
-      const int seq = i * 2 + 1;
-      xmax[me * 32 + lane] = mx;
-      if (!pair_sync(xflag, me, other, seq, lane, abort_flag, p.status)) { ok = false; break; }
-      mx = fmaxf(mx, xmax[other * 32 + lane]);
-      float sum = 0.f;
+      if (lane == 0) mbar_arrive(smem_u32(&sempty_bar[g]));
+      // Row maximum over the valid keys: one chain per 32-column chunk keeps the dependent
+      // chains short; only a chunk that crosses the length needs element-wise masking.
+      float mc[4];
 #pragma unroll
-      for (int j = 0; j < 16; j++) {
-        v0[j].x = __expf(v0[j].x - mx);
-        v0[j].y = __expf(v0[j].y - mx);
-        v1[j].x = __expf(v1[j].x - mx);
-        v1[j].y = __expf(v1[j].y - mx);
-        sum += (v0[j].x + v0[j].y) + (v1[j].x + v1[j].y);
+      for (int c = 0; c < 4; c++) {
+        mc[c] = -INFINITY;
+        if ((c + 1) * 32 > len) {
+#pragma unroll
+          for (int j = 0; j < 16; j++) {
+            if (c * 32 + 2 * j >= len) v[c][j].x = -INFINITY;
+            if (c * 32 + 2 * j + 1 >= len) v[c][j].y = -INFINITY;
+          }
+        }
+#pragma unroll
+        for (int j = 0; j < 16; j++) mc[c] = fmaxf(mc[c], fmaxf(v[c][j].x, v[c][j].y));
       }
-      xsum[me * 32 + lane] = sum;
-      if (!pair_sync(xflag, me, other, seq + 1, lane, abort_flag, p.status)) { ok = false; break; }
-      sum += xsum[other * 32 + lane];
+      const float mx = fmaxf(fmaxf(mc[0], mc[1]), fmaxf(mc[2], mc[3]));
+      // exp(scale * (x - max)) as 2^(x * scale * log2(e) - max * scale * log2(e)): one packed
+      // multiply-add per pair and one exponential per element; masked keys give 2^(-inf) = 0
+      const float sl2 = p.scale * 1.4426950408889634f;
+      const float2 k2 = splat2(sl2), nm2 = splat2(-mx * sl2);
+      float2 sc[4];
+#pragma unroll
+      for (int c = 0; c < 4; c++) {
+        sc[c] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < 16; j++) {
+          const float2 t = __ffma2_rn(v[c][j], k2, nm2);
+          v[c][j].x = fast_exp2(t.x);
+          v[c][j].y = fast_exp2(t.y);
+          sc[c] = __fadd2_rn(sc[c], v[c][j]);
+        }
+      }
+      const float sum = ((sc[0].x + sc[0].y) + (sc[1].x + sc[1].y)) + ((sc[2].x + sc[2].y) + (sc[3].x + sc[3].y));
       const float2 inv = splat2(1.0f / sum);
-#pragma unroll
-      for (int j = 0; j < 16; j++) {
-        v0[j] = __fmul2_rn(v0[j], inv);
-        v1[j] = __fmul2_rn(v1[j], inv);
-      }
-      // P as the A operand of the second product: k block = 64 keys, row r at 128 * r, its eight
+      // P as the A operand of the second product, over the item's Q and K tiles (both products
+      // of the first kind have completed): k block = 64 keys = 16 KB, row r at 128 * r, its eight
       // 16-byte pieces permuted by r mod 8 (the 128-byte swizzle the tensor core expects)
+      uint8_t* prow = smem + (size_t)s * AT_STAGE_BYTES + r * 128;
 #pragma unroll
-      for (int half = 0; half < 2; half++) {
-        const int c = half ? c1 : c0;
-        uint8_t* blk = p_smem + (c >> 1) * (128 * 128) + r * 128;
+      for (int c = 0; c < 4; c++) {
+#pragma unroll
+        for (int j = 0; j < 16; j++) v[c][j] = __fmul2_rn(v[c][j], inv);
 #pragma unroll
         for (int j = 0; j < 4; j++) {
           uint4 pk;
           __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
 #pragma unroll
-          for (int e = 0; e < 4; e++) h[e] = __float22bfloat162_rn(half ? v1[4 * j + e] : v0[4 * j + e]);
-          *reinterpret_cast<uint4*>(blk + ((((c & 1) * 4 + j) ^ (r & 7)) << 4)) = pk;
+          for (int e = 0; e < 4; e++) h[e] = __float22bfloat162_rn(v[c][4 * j + e]);
+          *reinterpret_cast<uint4*>(prow + (c >> 1) * AT_TILE_BYTES + ((((c & 1) * 4 + j) ^ (r & 7)) << 4)) = pk;
         }
       }
       // make the generic-proxy writes visible to the tensor core, then tell the MMA thread
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(pready_bar));
+      if (lane == 0) mbar_arrive(smem_u32(&pready_bar[g]));
       if (p.P != nullptr) {
         bf16* pg = p.P + zo * p.p_bo + zi * p.p_bi;
-        if (c0 * 32 < p.S) stage_store_bf16(stg, lane, v0, pg, p.S, q * 32, c0 * 32, p.S, p.S, p.vec_ok_p);
-        if (c1 * 32 < p.S) stage_store_bf16(stg, lane, v1, pg, p.S, q * 32, c1 * 32, p.S, p.S, p.vec_ok_p);
+#pragma unroll
+        for (int c = 0; c < 4; c++)
+          if (c * 32 < p.S) stage_store_bf16(stg, lane, v[c], pg, p.S, q * 32, c * 32, p.S, p.S, p.vec_ok_p);
       }
-      // context tile: 64 columns, one 32-column chunk per warp of the quarter
-      if (!mbar_wait(smem_u32(ofull_bar), (uint32_t)i & 1, abort_flag, p.status)) { ok = false; break; }
+      // context tile: 64 columns of this group's accumulator
+      if (!mbar_wait(smem_u32(&ofull_bar[g]), use & 1, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
-      tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + AT_O_COL + hsel * 32, v0);
+      const uint32_t orow = tmem_base + ((uint32_t)(q * 32) << 16) + AT_O_COL + (uint32_t)g * 64;
+      tc_ld32(orow, v[0]);
+      tc_ld32(orow + 32, v[1]);
       tc_fence_before();
-      stage_store_bf16(stg, lane, v0, p.C + zo * p.c_bo + zi * p.c_bi, p.c_ld, q * 32, hsel * 32, p.S, 64,
-                       p.vec_ok_c);
+      bf16* cg = p.C + zo * p.c_bo + zi * p.c_bi;
+      stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, 0, p.S, 64, p.vec_ok_c);
+      stage_store_bf16(stg, lane, v[1], cg, p.c_ld, q * 32, 32, p.S, 64, p.vec_ok_c);
     }
   }
 
@@ -330,8 +343,7 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
   rc = get_map(base + 2 * H, d, S, 1, 3 * H, (long long)S * 3 * H, d, A, B, 64, &mv, err);
   if (rc) return rc;
   for (int i = 0; i < 3; i++) { p.q_perm[i] = mq.perm[i]; p.k_perm[i] = mk.perm[i]; p.v_perm[i] = mv.perm[i]; }
-  const size_t smem_bytes = (size_t)AT_STAGES * AT_STAGE_BYTES + AT_P_BYTES + NUM_EPI_WARPS * AT_STAGING + 1024 +
-                            256 + 64 + 2 * NUM_EPI_WARPS * 32 * 4;
+  const size_t smem_bytes = (size_t)AT_STAGES * AT_STAGE_BYTES + NUM_EPI_WARPS * AT_STAGING + 1024 + 256;
   if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
   static bool attr_set = false;
   if (!attr_set) {
