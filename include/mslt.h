@@ -293,6 +293,16 @@ int mslt_op_attention(const void* d_qkv, void* d_probs, void* d_ctx, const int32
                       int32_t S, int32_t heads, float scale, int32_t* d_status, void* cuda_stream,
                       int32_t sync);
 
+/* Backward of mslt_op_attention in a single kernel (reverse-mode gradient of the same definition):
+ * with P the probabilities the forward call wrote and dC = d_dctx,
+ *   dV = P^T dC,  dP = dC V^T,  dS = P o (dP - rowsum(dP o P)) * scale,  dQ = dS K,  dK = dS^T Q,
+ * written to d_dqkv in d_qkv's layout.  bf16, head width 64, S a multiple of 8 in [8, 128].
+ * d_qkv, d_probs ([B, heads, S, S]), d_dctx ([B*S, heads*64]) are inputs, d_dqkv ([B*S, 3*heads*64])
+ * is the output; all device, 16-byte aligned, caller-owned.  d_status and sync as above. */
+int mslt_op_attention_bwd(const void* d_qkv, const void* d_probs, const void* d_dctx, void* d_dqkv, int32_t B,
+                          int32_t S, int32_t heads, float scale, int32_t* d_status, void* cuda_stream,
+                          int32_t sync);
+
 /*
  * mslt_op_cross_entropy without any device allocation by anybody.  (The paper has no counterpart
  * of this call; it exists for the integration below.)

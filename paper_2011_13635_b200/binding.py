@@ -56,7 +56,7 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_op_gemm", "mslt_op_gemm_enqueue", "mslt_op_cross_entropy",
            "mslt_op_cross_entropy_scratch_bytes", "mslt_op_cross_entropy_noalloc", "mslt_op_layernorm",
            "mslt_op_layernorm_bwd", "mslt_op_softmax", "mslt_op_softmax_bwd", "mslt_op_colsum",
-           "mslt_op_attention",
+           "mslt_op_attention", "mslt_op_attention_bwd",
            "mslt_debug_starve_next_gemm", "mslt_debug_check_guards"]
 
 lib.mslt_last_error.restype = C.c_char_p
@@ -110,6 +110,7 @@ lib.mslt_op_layernorm_bwd.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, _P, C.c
 lib.mslt_op_softmax.argtypes = [C.c_int32, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
 lib.mslt_op_softmax_bwd.argtypes = [C.c_int32, _P, _P, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
 lib.mslt_op_attention.argtypes = [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, _P, C.c_int32]
+lib.mslt_op_attention_bwd.argtypes = [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, _P, C.c_int32]
 lib.mslt_op_colsum.argtypes = [C.c_int32, _P, C.c_int64, C.c_int32, C.c_int32, _P, _P, C.c_int32]
 
 
@@ -190,6 +191,13 @@ def mslt_op_attention(qkv, probs, ctx, seq_lens, B: int, S: int, heads: int, sca
     """qkv bf16 [B*S, 3*heads*64]; probs bf16 [B, heads, S, S] or None; ctx bf16 [B*S, heads*64]."""
     _check(lib.mslt_op_attention(qkv.data_ptr(), _ptr(probs), ctx.data_ptr(), _ptr(seq_lens), B, S, heads,
                                  scale, status.data_ptr(), C.c_void_p(stream), int(sync)))
+
+
+def mslt_op_attention_bwd(qkv, probs, dctx, dqkv, B: int, S: int, heads: int, scale: float, status,
+                          stream: int, sync: bool = True) -> None:
+    """qkv, dqkv bf16 [B*S, 3*heads*64]; probs bf16 [B, heads, S, S]; dctx bf16 [B*S, heads*64]."""
+    _check(lib.mslt_op_attention_bwd(qkv.data_ptr(), probs.data_ptr(), dctx.data_ptr(), dqkv.data_ptr(), B, S,
+                                     heads, scale, status.data_ptr(), C.c_void_p(stream), int(sync)))
 
 
 def mslt_op_softmax_bwd(dp, probs, scale: float, stream: int, sync: bool = True) -> None:

@@ -302,6 +302,272 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   }
 }
 
+// ---- backward ---------------------------------------------------------------------------------------
+// Per (sequence, head) item, with P the saved probabilities and dC the gradient of the context:
+//   dV = P^T dC,  dP = dC V^T,  dS = P o (dP - rowsum(dP o P)) * scale,  dQ = dS K,  dK = dS^T Q.
+// The same roles as the forward kernel.  One shared-memory stage holds the item's Q, K, V, dC and
+// P tiles, every tile as 128-byte-swizzled rows indexed by position, which serves both operand
+// forms: rows as the m/n index with k contiguous, or rows as the k index with m/n contiguous.
+// dS (bf16) overwrites P once the first two products have completed.  A softmax group's thread
+// owns row r of its item: query r of dP, dS and dQ, key r of dK and dV.  Tensor memory per group:
+// dP in 128 columns, later reused by dQ and dK, and dV in 64.
+constexpr int AB_STAGE_BYTES = 6 * AT_TILE_BYTES;  // Q, K, V, dC, P (two tiles): 96 KB
+constexpr uint32_t AB_GROUP_COLS = 192;
+
+struct AttnBwdParams {
+  int S, heads, items;
+  float scale;
+  bf16* dQKV;         // element (b, i, which, h, e) at dQKV + b * g_bo + i * g_ld + which * H + h * 64 + e
+  long long g_ld, g_bo, H;
+  int vec_ok;
+  int q_perm[3], k_perm[3], v_perm[3], c_perm[3], p_perm[3];
+  long long wait_limit;
+  int* status;
+  uint32_t idesc_dv, idesc_dp, idesc_dq, idesc_dk;
+};
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV, const __grid_constant__ CUtensorMap tmC,
+                const __grid_constant__ CUtensorMap tmP, const AttnBwdParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* staging = smem + 2 * AB_STAGE_BYTES;
+  uint64_t* bars = (uint64_t*)(staging + NUM_EPI_WARPS * AT_STAGING);
+  uint64_t* full_bar = bars;           // [2] the item's tiles have landed (stage = group = item parity)
+  uint64_t* empty_bar = bars + 2;      // [2] every product of the item has read them
+  uint64_t* dpfull_bar = bars + 4;     // [2] dV and dP complete
+  uint64_t* dsready_bar = bars + 6;    // [2] dS in shared memory, dP read by the whole group
+  uint64_t* gfull_bar = bars + 8;      // [2] dQ and dK complete
+  uint64_t* accfree_bar = bars + 10;   // [2] the group has read dQ, dK, dV of its item
+  uint32_t* tmem_slot = (uint32_t*)(bars + 12);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int a = 0; a < 2; a++) {
+      mbar_init(smem_u32(&full_bar[a]), 1);
+      mbar_init(smem_u32(&empty_bar[a]), 1);
+      mbar_init(smem_u32(&dpfull_bar[a]), 1);
+      mbar_init(smem_u32(&dsready_bar[a]), AT_GROUP_WARPS);
+      mbar_init(smem_u32(&gfull_bar[a]), 1);
+      mbar_init(smem_u32(&accfree_bar[a]), AT_GROUP_WARPS);
+    }
+    *abort_flag = 0;
+    *reinterpret_cast<volatile long long*>(abort_flag + 1) = p.wait_limit;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(AT_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int n_my = ((int)blockIdx.x < p.items) ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    bool ok = true;
+    int issued = 0;
+    for (int i = 0; i < n_my && ok; i++) {
+      const int w = (int)blockIdx.x + i * (int)gridDim.x;
+      const int zo = w / p.heads, zi = w - zo * p.heads;
+      const uint32_t s = (uint32_t)i & 1, round = (uint32_t)i >> 1;
+      if (!mbar_wait(smem_u32(&empty_bar[s]), (round & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      const uint32_t fb = smem_u32(&full_bar[s]);
+      mbar_expect_tx(fb, AB_STAGE_BYTES);
+      const uint32_t base = smem_u32(smem + (size_t)s * AB_STAGE_BYTES);
+      int c[4];
+      c[0] = 0; c[p.q_perm[0]] = 0; c[p.q_perm[1]] = zi; c[p.q_perm[2]] = zo;
+      tma_load_4d(base, &tmQ, fb, c[0], c[1], c[2], c[3]);
+      c[0] = 0; c[p.k_perm[0]] = 0; c[p.k_perm[1]] = zi; c[p.k_perm[2]] = zo;
+      tma_load_4d(base + AT_TILE_BYTES, &tmK, fb, c[0], c[1], c[2], c[3]);
+      c[0] = 0; c[p.v_perm[0]] = 0; c[p.v_perm[1]] = zi; c[p.v_perm[2]] = zo;
+      tma_load_4d(base + 2 * AT_TILE_BYTES, &tmV, fb, c[0], c[1], c[2], c[3]);
+      c[0] = 0; c[p.c_perm[0]] = 0; c[p.c_perm[1]] = zi; c[p.c_perm[2]] = zo;
+      tma_load_4d(base + 3 * AT_TILE_BYTES, &tmC, fb, c[0], c[1], c[2], c[3]);
+      // P: two tiles of 64 keys, each 128 query rows of 128 bytes
+      c[p.p_perm[0]] = 0; c[p.p_perm[1]] = zi; c[p.p_perm[2]] = zo;
+      c[0] = 0;
+      tma_load_4d(base + 4 * AT_TILE_BYTES, &tmP, fb, c[0], c[1], c[2], c[3]);
+      c[0] = 64;
+      tma_load_4d(base + 5 * AT_TILE_BYTES, &tmP, fb, c[0], c[1], c[2], c[3]);
+      issued = i + 1;
+    }
+    if (!ok || *abort_flag) {
+      const int n = issued < 2 ? issued : 2;
+      for (int k = 0; k < n; k++) {
+        const int j = issued - 1 - k;
+        const uint32_t fb = smem_u32(&full_bar[j & 1]);
+        const long long t0 = now_cycles();
+        while (!mbar_try_wait(fb, (uint32_t)(j >> 1) & 1) && now_cycles() - t0 < 200000000ll) {}
+      }
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------- MMA issuer -------------------------------
+    bool ok = true;
+    const uint32_t hi = (uint32_t)(make_smem_desc(0, 16) >> 32);
+    const uint32_t lbo_k = (uint32_t)make_smem_desc(0, 16);            // k-contiguous operand
+    const uint32_t lbo_mn1 = (uint32_t)make_smem_desc(0, 8192);        // rows = k, one 64-wide m/n block
+    const uint32_t lbo_mn2 = (uint32_t)make_smem_desc(0, AT_TILE_BYTES);  // two 64-wide blocks 16 KB apart
+    auto addr16 = [](uint32_t a) { return (a & 0x3FFFFu) >> 4; };
+    auto mma_k128 = [&](uint32_t d_tmem, uint32_t a_lo, uint32_t a_kb, uint32_t a_ks, uint32_t b_lo,
+                        uint32_t b_kb, uint32_t b_ks, uint32_t idesc) {  // contraction over 128 = 2 x 4 x 16
+      uint32_t accum = 0;
+#pragma unroll
+      for (int kb = 0; kb < 2; kb++)
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+          const uint64_t ad = ((uint64_t)hi << 32) | (a_lo + kb * a_kb + k * a_ks);
+          const uint64_t bd = ((uint64_t)hi << 32) | (b_lo + kb * b_kb + k * b_ks);
+          tc_mma(d_tmem, ad, bd, idesc, accum);
+          accum = 1;
+        }
+    };
+    constexpr uint32_t KS_K = UMMA_K * 2 / 16;      // 16 k values of a k-contiguous tile, in 16-byte units
+    constexpr uint32_t KS_MN = UMMA_K * 128 / 16;   // 16 k rows of a row-is-k tile
+    constexpr uint32_t KB_MN = 8192 / 16;           // 64 k rows
+    constexpr uint32_t KB_K = AT_TILE_BYTES / 16;   // next 64-wide k block of a two-tile operand
+    auto second_products = [&](int j) {  // dQ = dS K and dK = dS^T Q of item j
+      const uint32_t g = (uint32_t)j & 1;
+      const uint32_t base = smem_u32(smem + (size_t)g * AB_STAGE_BYTES);
+      const uint32_t ds = addr16(base + 4 * AT_TILE_BYTES);
+      const uint32_t acc = tmem_base + g * AB_GROUP_COLS;
+      mma_k128(acc, lbo_k | ds, KB_K, KS_K, lbo_mn1 | addr16(base + AT_TILE_BYTES), KB_MN, KS_MN, p.idesc_dq);
+      mma_k128(acc + 64, lbo_mn2 | ds, KB_MN, KS_MN, lbo_mn1 | addr16(base), KB_MN, KS_MN, p.idesc_dk);
+      tc_commit(smem_u32(&gfull_bar[g]));
+      tc_commit(smem_u32(&empty_bar[g]));
+    };
+    for (int i = 0; i < n_my && ok; i++) {
+      const uint32_t g = (uint32_t)i & 1, use = (uint32_t)i >> 1;
+      if (!mbar_wait(smem_u32(&full_bar[g]), use & 1, abort_flag, p.status)) { ok = false; break; }
+      if (!mbar_wait(smem_u32(&accfree_bar[g]), (use & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      const uint32_t base = smem_u32(smem + (size_t)g * AB_STAGE_BYTES);
+      const uint32_t acc = tmem_base + g * AB_GROUP_COLS;
+      const uint32_t dc = addr16(base + 3 * AT_TILE_BYTES);
+      // dV = P^T dC: both operands with rows = query index = k
+      mma_k128(acc + 128, lbo_mn2 | addr16(base + 4 * AT_TILE_BYTES), KB_MN, KS_MN, lbo_mn1 | dc, KB_MN, KS_MN,
+               p.idesc_dv);
+      // dP = dC V^T: both operands k-contiguous, contraction over the head width
+#pragma unroll
+      for (int k = 0; k < 4; k++) {
+        const uint64_t ad = ((uint64_t)hi << 32) | ((lbo_k | dc) + k * KS_K);
+        const uint64_t bd = ((uint64_t)hi << 32) | ((lbo_k | addr16(base + 2 * AT_TILE_BYTES)) + k * KS_K);
+        tc_mma(acc, ad, bd, p.idesc_dp, k > 0 ? 1u : 0u);
+      }
+      tc_commit(smem_u32(&dpfull_bar[g]));
+      if (i > 0) {
+        const uint32_t g1 = (uint32_t)(i - 1) & 1, use1 = (uint32_t)(i - 1) >> 1;
+        if (!mbar_wait(smem_u32(&dsready_bar[g1]), use1 & 1, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        second_products(i - 1);
+      }
+    }
+    if (ok && n_my > 0) {
+      const uint32_t g1 = (uint32_t)(n_my - 1) & 1, use1 = (uint32_t)(n_my - 1) >> 1;
+      if (mbar_wait(smem_u32(&dsready_bar[g1]), use1 & 1, abort_flag, p.status)) {
+        tc_fence_after();
+        second_products(n_my - 1);
+      } else {
+        ok = false;
+      }
+    }
+    if (!ok || *abort_flag) {
+      tc_commit(smem_u32(&dpfull_bar[0]));
+      const long long t0 = now_cycles();
+      while (now_cycles() - t0 < 2000000ll) {}
+    }
+  } else if (warp >= 2) {
+    // ------------------------------- softmax-backward groups -------------------------------
+    const int q = warp & 3;
+    const int g = (warp - 2) >> 2;
+    uint8_t* stg = staging + (size_t)(warp - 2) * AT_STAGING;
+    const int r = q * 32 + lane;
+    bool ok = true;
+    for (int i = g; i < n_my && ok; i += 2) {
+      const int w = (int)blockIdx.x + i * (int)gridDim.x;
+      const int zo = w / p.heads, zi = w - zo * p.heads;
+      const uint32_t use = (uint32_t)i >> 1;
+      if (!mbar_wait(smem_u32(&dpfull_bar[g]), use & 1, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      float2 v[4][16];  // row r of dP
+      const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g * AB_GROUP_COLS;
+#pragma unroll
+      for (int c = 0; c < 4; c++) tc_ld32(trow + c * 32, v[c]);
+      // row r of P (and then of dS): two 128-byte halves, 16-byte pieces permuted by r mod 8
+      uint8_t* prow = smem + (size_t)g * AB_STAGE_BYTES + 4 * AT_TILE_BYTES + r * 128;
+      float2 dl[4];
+#pragma unroll
+      for (int c = 0; c < 4; c++) {
+        dl[c] = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+          const uint4 pk = *reinterpret_cast<const uint4*>(prow + (c >> 1) * AT_TILE_BYTES +
+                                                           ((((c & 1) * 4 + j) ^ (r & 7)) << 4));
+          dl[c] = __ffma2_rn(v[c][4 * j], bf162_to_f2(pk.x), dl[c]);
+          dl[c] = __ffma2_rn(v[c][4 * j + 1], bf162_to_f2(pk.y), dl[c]);
+          dl[c] = __ffma2_rn(v[c][4 * j + 2], bf162_to_f2(pk.z), dl[c]);
+          dl[c] = __ffma2_rn(v[c][4 * j + 3], bf162_to_f2(pk.w), dl[c]);
+        }
+      }
+      const float delta = ((dl[0].x + dl[0].y) + (dl[1].x + dl[1].y)) + ((dl[2].x + dl[2].y) + (dl[3].x + dl[3].y));
+      const float2 nd = splat2(-delta), sc2 = splat2(p.scale);
+#pragma unroll
+      for (int c = 0; c < 4; c++) {
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+          uint8_t* piece = prow + (c >> 1) * AT_TILE_BYTES + ((((c & 1) * 4 + j) ^ (r & 7)) << 4);
+          const uint4 pk = *reinterpret_cast<const uint4*>(piece);
+          const uint32_t pw[4] = {pk.x, pk.y, pk.z, pk.w};
+          uint4 out;
+          __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&out);
+#pragma unroll
+          for (int e = 0; e < 4; e++) {
+            const float2 t = __fmul2_rn(__fadd2_rn(v[c][4 * j + e], nd), sc2);
+            h[e] = __float22bfloat162_rn(__fmul2_rn(t, bf162_to_f2(pw[e])));
+          }
+          *reinterpret_cast<uint4*>(piece) = out;
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&dsready_bar[g]));
+      bf16* gq = p.dQKV + zo * p.g_bo + zi * 64;
+      // dV (complete since dP was): key r, 64 columns
+      tc_ld32(trow + 128, v[0]);
+      tc_ld32(trow + 160, v[1]);
+      stage_store_bf16(stg, lane, v[0], gq + 2 * p.H, p.g_ld, q * 32, 0, p.S, 64, p.vec_ok);
+      stage_store_bf16(stg, lane, v[1], gq + 2 * p.H, p.g_ld, q * 32, 32, p.S, 64, p.vec_ok);
+      if (!mbar_wait(smem_u32(&gfull_bar[g]), use & 1, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+#pragma unroll
+      for (int c = 0; c < 4; c++) tc_ld32(trow + c * 32, v[c]);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(&accfree_bar[g]));
+      stage_store_bf16(stg, lane, v[0], gq, p.g_ld, q * 32, 0, p.S, 64, p.vec_ok);
+      stage_store_bf16(stg, lane, v[1], gq, p.g_ld, q * 32, 32, p.S, 64, p.vec_ok);
+      stage_store_bf16(stg, lane, v[2], gq + p.H, p.g_ld, q * 32, 0, p.S, 64, p.vec_ok);
+      stage_store_bf16(stg, lane, v[3], gq + p.H, p.g_ld, q * 32, 32, p.S, 64, p.vec_ok);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(AT_TMEM_COLS)
+                 : "memory");
+  }
+}
+
 }  // namespace
 
 static std::atomic<long long> g_attn_launches{0};
@@ -353,6 +619,66 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
   }
   const int grid = p.items < num_sms ? p.items : num_sms;
   attn_fwd_kernel<<<grid, NUM_THREADS, smem_bytes, st>>>(mq.map, mk.map, mv.map, p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { snprintf(err, 256, "attention: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+  g_attn_launches++;
+  return 0;
+}
+
+int attn_bwd_launch(const void* qkv, const void* probs, const void* dctx, void* dqkv, int B, int S, int A, int d,
+                    float scale, int* status, cudaStream_t st, char* err) {
+  static int num_sms = 0, smem_optin = 0;
+  if (num_sms == 0) {
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (num_sms <= 0) { snprintf(err, 256, "attention: no CUDA device"); return MSLT_ERR_CUDA; }
+  }
+  if (d != 64 || S < 8 || S > 128 || S % 8 || B < 1 || A < 1 || !status || !qkv || !probs || !dctx || !dqkv) {
+    snprintf(err, 256, "attention backward: the fused kernel needs head width 64 and S a multiple of 8 in [8, 128]");
+    return MSLT_ERR_ARG;
+  }
+  const long long H = (long long)A * d;
+  AttnBwdParams p;
+  memset(&p, 0, sizeof(p));
+  p.S = S; p.heads = A; p.items = B * A; p.scale = scale;
+  p.dQKV = (bf16*)dqkv; p.g_ld = 3 * H; p.g_bo = (long long)S * 3 * H; p.H = H;
+  p.vec_ok = ((uintptr_t)dqkv & 15) == 0 ? 1 : 0;
+  p.wait_limit = WAIT_LIMIT_CYCLES;
+  p.status = status;
+  // fp32 accumulate, bf16 x bf16, M = 128; bit 15 / 16: A / B operand with rows = k index
+  const uint32_t common = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
+  p.idesc_dv = common | (1u << 15) | (1u << 16) | ((uint32_t)(64 >> 3) << 17);
+  p.idesc_dp = common | ((uint32_t)(128 >> 3) << 17);
+  p.idesc_dq = common | (1u << 16) | ((uint32_t)(64 >> 3) << 17);
+  p.idesc_dk = common | (1u << 15) | (1u << 16) | ((uint32_t)(64 >> 3) << 17);
+  const bf16* base = (const bf16*)qkv;
+  MapVal mq, mk, mv, mc, mp;
+  int rc = get_map(base, S, d, 3 * H, 1, (long long)S * 3 * H, d, A, B, BM, &mq, err);
+  if (rc) return rc;
+  rc = get_map(base + H, S, d, 3 * H, 1, (long long)S * 3 * H, d, A, B, BM, &mk, err);
+  if (rc) return rc;
+  rc = get_map(base + 2 * H, S, d, 3 * H, 1, (long long)S * 3 * H, d, A, B, BM, &mv, err);
+  if (rc) return rc;
+  rc = get_map(dctx, S, d, H, 1, (long long)S * H, d, A, B, BM, &mc, err);
+  if (rc) return rc;
+  rc = get_map(probs, S, S, S, 1, (long long)A * S * S, (long long)S * S, A, B, BM, &mp, err);
+  if (rc) return rc;
+  for (int i = 0; i < 3; i++) {
+    p.q_perm[i] = mq.perm[i]; p.k_perm[i] = mk.perm[i]; p.v_perm[i] = mv.perm[i];
+    p.c_perm[i] = mc.perm[i]; p.p_perm[i] = mp.perm[i];
+  }
+  const size_t smem_bytes = (size_t)2 * AB_STAGE_BYTES + NUM_EPI_WARPS * AT_STAGING + 1024 + 256;
+  if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+    if (e != cudaSuccess) { snprintf(err, 256, "attention: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+    attr_set = true;
+  }
+  const int grid = p.items < num_sms ? p.items : num_sms;
+  attn_bwd_kernel<<<grid, NUM_THREADS, smem_bytes, st>>>(mq.map, mk.map, mv.map, mc.map, mp.map, p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { snprintf(err, 256, "attention: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
   g_attn_launches++;

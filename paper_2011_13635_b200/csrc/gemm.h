@@ -27,6 +27,11 @@ void gemm_tc_starve_next(int on);
 // gemm_launch.  Returns 0 or a negative mslt_status with a message in `err`.
 int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens, int B, int S, int A, int d,
                     float scale, int* status, cudaStream_t st, char* err);
+// Its backward: dqkv ([B*S, 3*A*d], queries | keys | values like qkv) from the saved probabilities
+// and the gradient of the context dctx ([B*S, A*d]); S a multiple of 8.
+//   dV = P^T dC,  dP = dC V^T,  dS = P o (dP - rowsum(dP o P)) * scale,  dQ = dS K,  dK = dS^T Q
+int attn_bwd_launch(const void* qkv, const void* probs, const void* dctx, void* dqkv, int B, int S, int A, int d,
+                    float scale, int* status, cudaStream_t st, char* err);
 long long attn_launches();
 
 // Kernels launched by the GEMM front end since the library was loaded (for launch accounting).

@@ -328,6 +328,21 @@ int run_attention(mslt_ctx* c, const void* qkv, void* probs, void* ctx, const in
   return 0;
 }
 
+int run_attention_bwd(mslt_ctx* c, const void* qkv, const void* probs, const void* dctx, void* dqkv, int B,
+                      int S, int A, int d, float scale) {
+  char err[256] = "";
+  const bool prof = c->profile && c->prec.size() * 2 + 2 <= c->pev.size();
+  if (prof) cudaEventRecord(c->pev[2 * c->prec.size()], c->st);
+  int rc = attn_bwd_launch(qkv, probs, dctx, dqkv, B, S, A, d, scale, c->ws.scalars, c->st, err);
+  if (prof) {
+    cudaEventRecord(c->pev[2 * c->prec.size() + 1], c->st);
+    c->prec.push_back({1, 8.0 * B * A * (double)S * S * d});
+  }
+  if (rc) return fail(rc, "%s", err);
+  c->launches++;
+  return 0;
+}
+
 int run_gemm(mslt_ctx* c, const mslt_gemm_desc& d) {
   if (d.M <= 0 || d.N <= 0 || d.K <= 0 || d.batch <= 0) return 0;
   char err[256] = "";
@@ -478,38 +493,43 @@ int layer_backward(mslt_ctx* c, int l, const void* x_in, LayerBuf& b, const void
   KL(PC_COLSUM, 1.0 * T * H * c->esz, launch_colsum(c->bf, w.dz1, H, T, H, G(c, toff(c, l, "out.bias")), c->st));
   TRY(linear_dgrad(c, w.dz1, T, H, H, toff(c, l, "out.weight"), H, w.dc, 0, nullptr, nullptr));
   const int64_t qs = (int64_t)S * 3 * H, ps = (int64_t)A * S * S, cs = (int64_t)S * H;
-  {  // dV[j,:] = sum_i p[i,j] dC[i,:]
-    Lin g(c, S, d, S);
-    g.d.batch = B * A; g.d.hdiv = A;
-    g.d.A = b.p; g.d.a_rs = 1; g.d.a_ks = S; g.d.a_bo = ps; g.d.a_bi = (int64_t)S * S;
-    g.d.B = w.dc; g.d.b_rs = 1; g.d.b_ks = H; g.d.b_bo = cs; g.d.b_bi = d;
-    g.d.D = w.dqkv + (int64_t)2 * H * E; g.d.ldd = 3 * H; g.d.d_bo = qs; g.d.d_bi = d;
-    TRY(run_gemm(c, g.d));
-  }
-  {  // dP[i,j] = dC[i,:] . v_j
-    Lin g(c, S, S, d);
-    g.d.batch = B * A; g.d.hdiv = A;
-    g.d.A = w.dc; g.d.a_rs = H; g.d.a_ks = 1; g.d.a_bo = cs; g.d.a_bi = d;
-    g.d.B = b.qkv + (int64_t)2 * H * E; g.d.b_rs = 3 * H; g.d.b_ks = 1; g.d.b_bo = qs; g.d.b_bi = d;
-    g.d.D = w.dp; g.d.ldd = S; g.d.d_bo = ps; g.d.d_bi = (int64_t)S * S;
-    TRY(run_gemm(c, g.d));
-  }
-  KL(PC_SOFTMAX_BWD, 3.0 * B * A * S * S * c->esz, launch_softmax_bwd(c->bf, w.dp, b.p, B * A * S, S, scale, c->st));
-  {  // dQ[i,:] = sum_j dS[i,j] k_j
-    Lin g(c, S, d, S);
-    g.d.batch = B * A; g.d.hdiv = A;
-    g.d.A = w.dp; g.d.a_rs = S; g.d.a_ks = 1; g.d.a_bo = ps; g.d.a_bi = (int64_t)S * S;
-    g.d.B = b.qkv + (int64_t)H * E; g.d.b_rs = 1; g.d.b_ks = 3 * H; g.d.b_bo = qs; g.d.b_bi = d;
-    g.d.D = w.dqkv; g.d.ldd = 3 * H; g.d.d_bo = qs; g.d.d_bi = d;
-    TRY(run_gemm(c, g.d));
-  }
-  {  // dK[j,:] = sum_i dS[i,j] q_i
-    Lin g(c, S, d, S);
-    g.d.batch = B * A; g.d.hdiv = A;
-    g.d.A = w.dp; g.d.a_rs = 1; g.d.a_ks = S; g.d.a_bo = ps; g.d.a_bi = (int64_t)S * S;
-    g.d.B = b.qkv; g.d.b_rs = 1; g.d.b_ks = 3 * H; g.d.b_bo = qs; g.d.b_bi = d;
-    g.d.D = w.dqkv + (int64_t)H * E; g.d.ldd = 3 * H; g.d.d_bo = qs; g.d.d_bi = d;
-    TRY(run_gemm(c, g.d));
+  if (c->bf && S <= 128 && S % 8 == 0 && d == 64 && !getenv_cuda_cores() && !getenv_unfused_attention()) {
+    // dV, dP, softmax backward, dQ and dK of the layer in one kernel
+    TRY(run_attention_bwd(c, b.qkv, b.p, w.dc, w.dqkv, B, S, A, d, scale));
+  } else {
+    {  // dV[j,:] = sum_i p[i,j] dC[i,:]
+      Lin g(c, S, d, S);
+      g.d.batch = B * A; g.d.hdiv = A;
+      g.d.A = b.p; g.d.a_rs = 1; g.d.a_ks = S; g.d.a_bo = ps; g.d.a_bi = (int64_t)S * S;
+      g.d.B = w.dc; g.d.b_rs = 1; g.d.b_ks = H; g.d.b_bo = cs; g.d.b_bi = d;
+      g.d.D = w.dqkv + (int64_t)2 * H * E; g.d.ldd = 3 * H; g.d.d_bo = qs; g.d.d_bi = d;
+      TRY(run_gemm(c, g.d));
+    }
+    {  // dP[i,j] = dC[i,:] . v_j
+      Lin g(c, S, S, d);
+      g.d.batch = B * A; g.d.hdiv = A;
+      g.d.A = w.dc; g.d.a_rs = H; g.d.a_ks = 1; g.d.a_bo = cs; g.d.a_bi = d;
+      g.d.B = b.qkv + (int64_t)2 * H * E; g.d.b_rs = 3 * H; g.d.b_ks = 1; g.d.b_bo = qs; g.d.b_bi = d;
+      g.d.D = w.dp; g.d.ldd = S; g.d.d_bo = ps; g.d.d_bi = (int64_t)S * S;
+      TRY(run_gemm(c, g.d));
+    }
+    KL(PC_SOFTMAX_BWD, 3.0 * B * A * S * S * c->esz, launch_softmax_bwd(c->bf, w.dp, b.p, B * A * S, S, scale, c->st));
+    {  // dQ[i,:] = sum_j dS[i,j] k_j
+      Lin g(c, S, d, S);
+      g.d.batch = B * A; g.d.hdiv = A;
+      g.d.A = w.dp; g.d.a_rs = S; g.d.a_ks = 1; g.d.a_bo = ps; g.d.a_bi = (int64_t)S * S;
+      g.d.B = b.qkv + (int64_t)H * E; g.d.b_rs = 1; g.d.b_ks = 3 * H; g.d.b_bo = qs; g.d.b_bi = d;
+      g.d.D = w.dqkv; g.d.ldd = 3 * H; g.d.d_bo = qs; g.d.d_bi = d;
+      TRY(run_gemm(c, g.d));
+    }
+    {  // dK[j,:] = sum_i dS[i,j] q_i
+      Lin g(c, S, d, S);
+      g.d.batch = B * A; g.d.hdiv = A;
+      g.d.A = w.dp; g.d.a_rs = 1; g.d.a_ks = S; g.d.a_bo = ps; g.d.a_bi = (int64_t)S * S;
+      g.d.B = b.qkv; g.d.b_rs = 1; g.d.b_ks = 3 * H; g.d.b_bo = qs; g.d.b_bi = d;
+      g.d.D = w.dqkv + (int64_t)H * E; g.d.ldd = 3 * H; g.d.d_bo = qs; g.d.d_bi = d;
+      TRY(run_gemm(c, g.d));
+    }
   }
   TRY(linear_wgrad(c, w.dqkv, T, 3 * H, 3 * H, x_in, H, toff(c, l, "qkv.weight")));
   KL(PC_COLSUM, 3.0 * T * H * c->esz, launch_colsum(c->bf, w.dqkv, 3 * H, T, 3 * H, G(c, toff(c, l, "qkv.bias")), c->st));

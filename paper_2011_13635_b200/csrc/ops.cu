@@ -218,6 +218,32 @@ int mslt_op_attention(const void* d_qkv, void* d_probs, void* d_ctx, const int32
   return finish_op("attention", st, 0);
 }
 
+int mslt_op_attention_bwd(const void* d_qkv, const void* d_probs, const void* d_dctx, void* d_dqkv, int32_t B,
+                          int32_t S, int32_t heads, float scale, int32_t* d_status, void* cuda_stream,
+                          int32_t sync) {
+  if (!d_qkv || !d_probs || !d_dctx || !d_dqkv || !d_status)
+    return op_fail(MSLT_ERR_ARG, "attention_bwd: null pointer");
+  if (((uintptr_t)d_qkv | (uintptr_t)d_probs | (uintptr_t)d_dctx | (uintptr_t)d_dqkv) & 15)
+    return op_fail(MSLT_ERR_ARG, "attention_bwd: buffers must be 16-byte aligned");
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1)
+    return op_fail(MSLT_ERR_CUDA, "no CUDA device: this library has no CPU path");
+  cudaStream_t st = (cudaStream_t)cuda_stream;
+  char err[256] = "";
+  int rc = attn_bwd_launch(d_qkv, d_probs, d_dctx, d_dqkv, B, S, heads, 64, scale, d_status, st, err);
+  if (rc) return op_fail(rc, "%s", err);
+  if (sync) {
+    rc = finish_op("attention_bwd", st, 1);
+    if (rc) return rc;
+    int h = 0;
+    if (cudaMemcpy(&h, d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess)
+      return op_fail(MSLT_ERR_CUDA, "attention_bwd: reading the status word failed");
+    if (h & 1) return op_fail(MSLT_ERR_DEVICE, "attention_bwd: a bounded wait ran out on the device");
+    return 0;
+  }
+  return finish_op("attention_bwd", st, 0);
+}
+
 int mslt_op_softmax(int32_t dtype, const void* d_scores, void* d_probs, const int32_t* d_seq_lens,
                     int32_t rows, int32_t S, int32_t rows_per_seq, float scale, void* cuda_stream,
                     int32_t sync) {

@@ -1,7 +1,7 @@
 """Bandwidth of the fused memory-bound kernels, one at a time, through the mslt_op_* entry points.
 
     python -m paper_2011_13635_b200.op_bench [--rows 16384] [--hidden 768] [--ffn 3072] [--heads 12]
-        [--seq 128] [--batch 128] [--dtype bf16|fp32]
+        [--seq 128] [--batch 128] [--dtype bf16|fp32] [--only NAME[,NAME...]]
 
 Each kernel is launched back to back on a rotation of buffers whose total size exceeds the 126 MB L2,
 so that every launch reads its input from HBM; times are CUDA events on the launching stream.
@@ -25,7 +25,10 @@ def main():
     ap.add_argument("--batch", type=int, default=128)
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--iters", type=int, default=40)
+    ap.add_argument("--only", default="", help="comma-separated kernel groups: ln, colsum, softmax, attention, ce")
     a = ap.parse_args()
+    only = set(x for x in a.only.split(",") if x)
+    want = lambda group: not only or group in only
     tdt = torch.bfloat16 if a.dtype == "bf16" else torch.float32
     E = 2 if a.dtype == "bf16" else 4
     st = torch.cuda.current_stream().cuda_stream
@@ -52,6 +55,22 @@ def main():
         print(json.dumps(dict(kernel=name, dtype=a.dtype, bytes=nbytes, us=round(us, 2),
                               gbs=round(nbytes / us / 1e3, 1))))
 
+    if want("attention") and a.dtype == "bf16" and a.seq <= 128:
+        # fused attention of one layer: reads Q, K, V once, writes the context (and the probabilities)
+        B, S, A = a.batch, a.seq, a.heads
+        qs = rotation((B * S, 3 * A * 64), tdt)
+        ctx = torch.empty((B * S, A * 64), device="cuda", dtype=tdt)
+        probs = torch.empty((B, A, S, S), device="cuda", dtype=tdt)
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+        run("attention_fused", 4 * B * S * A * 64 * E,
+            lambda i: Bd.mslt_op_attention(qs[i], None, ctx, None, B, S, A, 0.125, status, st, sync=False), len(qs))
+        run("attention_fused_with_probs", 4 * B * S * A * 64 * E + B * A * S * S * E,
+            lambda i: Bd.mslt_op_attention(qs[i], probs, ctx, None, B, S, A, 0.125, status, st, sync=False), len(qs))
+        if int(status.item()) != 0:
+            raise RuntimeError("the attention kernel reported a wait that ran out")
+        del qs, ctx, probs
+    if not (want("ln") or want("colsum") or want("softmax") or want("ce")):
+        return
     gamma = torch.ones(H, device="cuda"); beta = torch.zeros(H, device="cuda")
     zs = rotation((T, H), tdt)
     y = torch.empty((T, H), device="cuda", dtype=tdt)

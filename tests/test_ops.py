@@ -207,3 +207,40 @@ def test_fused_attention_rejects_other_shapes():
         Bd.mslt_op_attention(qkv, None, ctx, None, 1, 256, 1, 0.125, status, _stream())
     with pytest.raises(Bd.MsltError):
         Bd.mslt_op_attention(qkv, None, ctx, None, 0, 128, 1, 0.125, status, _stream())
+
+
+@pytest.mark.parametrize("B,S,A,masked", [(2, 128, 2, False), (3, 128, 12, True), (2, 104, 3, True),
+                                          (5, 64, 2, True), (1, 24, 1, False), (37, 128, 12, True)])
+def test_fused_attention_backward_matches_oracle(B, S, A, masked):
+    """dQ, dK, dV of one kernel against the reverse-mode formulas written with the oracle's
+    softmax_backward, on the same bf16-rounded inputs (probabilities from the oracle's softmax)."""
+    import math
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    d, H = 64, A * 64
+    rng = np.random.default_rng(B * 977 + S + A)
+    bf = lambda a: torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda().bfloat16()
+    qkv = bf(rng.standard_normal((B * S, 3 * H)) * 1.5)
+    dctx = bf(rng.standard_normal((B * S, H)))
+    lens = rng.integers(1, S + 1, size=B).astype(np.int32) if masked else np.full(B, S, np.int32)
+    scale = 1.0 / math.sqrt(d)
+    x = qkv.float().cpu().numpy().astype(np.float64).reshape(B, S, 3, A, d)
+    q, k, v = (x[:, :, i].transpose(0, 2, 1, 3) for i in range(3))            # [B, A, S, d]
+    probs = bf(O.masked_softmax(np.einsum("bhid,bhjd->bhij", q, k) * scale, lens))
+    p = probs.float().cpu().numpy().astype(np.float64)
+    dc = dctx.float().cpu().numpy().astype(np.float64).reshape(B, S, A, d).transpose(0, 2, 1, 3)
+    dv = np.einsum("bhij,bhid->bhjd", p, dc)
+    ds = O.softmax_backward(np.einsum("bhid,bhjd->bhij", dc, v), p) * scale
+    dq = np.einsum("bhij,bhjd->bhid", ds, k)
+    dk = np.einsum("bhij,bhid->bhjd", ds, q)
+    want = np.stack([dq, dk, dv], axis=0).transpose(1, 3, 0, 2, 4).reshape(B * S, 3 * H)   # [B,S,3,A,d]
+    dqkv = torch.full((B * S, 3 * H), 7.0, device="cuda", dtype=torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for _ in range(2):
+        Bd.mslt_op_attention_bwd(qkv, probs, dctx, dqkv, B, S, A, scale, status, _stream())
+    assert int(status.item()) == 0
+    got = dqkv.float().cpu().numpy().reshape(B, S, 3, H)
+    want = want.reshape(B, S, 3, H)
+    for which, name in enumerate(("dq", "dk", "dv")):
+        err = np.abs(got[:, :, which] - want[:, :, which]).max() / np.abs(want[:, :, which]).max()
+        assert err < 1.5e-2, (name, err)
