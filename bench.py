@@ -314,7 +314,8 @@ def run_ours(args, cfg):
         else:
             line["roofline"] = dict(bound="alu", kernel="gemm_simt_kernel", achieved=lin_tflops, peak=None,
                                     unit="TFLOP/s", frac=None, traffic=None)
-        line["attention_gemms"] = dict(
+        # attention: fused kernels (HBM-bound) where the sequence fits one tile, batched products otherwise
+        line["attention"] = dict(
             tflops=att["work"] / (att["ms"] * 1e-3) / 1e12 if att["ms"] > 0 else 0.0,
             ms_per_step=att["ms"] / n_prof, launches_per_step=att["launches"] / n_prof)
         line["phases_ms"] = phases

@@ -66,9 +66,15 @@ def main():
             lambda i: Bd.mslt_op_attention(qs[i], None, ctx, None, B, S, A, 0.125, status, st, sync=False), len(qs))
         run("attention_fused_with_probs", 4 * B * S * A * 64 * E + B * A * S * S * E,
             lambda i: Bd.mslt_op_attention(qs[i], probs, ctx, None, B, S, A, 0.125, status, st, sync=False), len(qs))
+        # its backward: reads Q, K, V, the probabilities and the context gradient, writes dQ, dK, dV
+        probs.copy_(torch.softmax(torch.randn((B, A, S, S), device="cuda"), -1))
+        dqkv = torch.empty((B * S, 3 * A * 64), device="cuda", dtype=tdt)
+        run("attention_fused_backward", 7 * B * S * A * 64 * E + B * A * S * S * E,
+            lambda i: Bd.mslt_op_attention_bwd(qs[i], probs, ctx, dqkv, B, S, A, 0.125, status, st, sync=False),
+            len(qs))
         if int(status.item()) != 0:
             raise RuntimeError("the attention kernel reported a wait that ran out")
-        del qs, ctx, probs
+        del qs, ctx, probs, dqkv
     if not (want("ln") or want("colsum") or want("softmax") or want("ce")):
         return
     gamma = torch.ones(H, device="cuda"); beta = torch.zeros(H, device="cuda")
