@@ -259,13 +259,15 @@ int mslt_op_cross_entropy(int32_t dtype, const float* d_logits, int64_t ldl, con
  * LayerNorm of the encoder (post-LN BERT, Section 4.1): y = gamma * (z - mean) / sqrt(var + eps) +
  * beta over rows of H <= 1024 elements, biased variance; d_stats (may be NULL) receives
  * {mean, 1/sqrt(var + eps)} per row.  The backward call takes those statistics and returns dz and
- * ADDS the column sums dgamma += sum dy * xhat, dbeta += sum dy (the caller zeroes them).
+ * ADDS the column sums dgamma += sum dy * xhat, dbeta += sum dy (the caller zeroes them); with
+ * d_dbias != NULL it also ADDS dbias += sum dz, the bias gradient of the linear layer whose output
+ * (plus residual) was normalised, which saves a separate pass over dz.
  */
 int mslt_op_layernorm(int32_t dtype, const void* d_z, const float* d_gamma, const float* d_beta, void* d_y,
                       float* d_stats, int32_t rows, int32_t H, float eps, void* cuda_stream, int32_t sync);
 int mslt_op_layernorm_bwd(int32_t dtype, const void* d_dy, const void* d_z, const float* d_stats,
-                          const float* d_gamma, void* d_dz, float* d_dgamma, float* d_dbeta, int32_t rows,
-                          int32_t H, void* cuda_stream, int32_t sync);
+                          const float* d_gamma, void* d_dz, float* d_dgamma, float* d_dbeta, float* d_dbias,
+                          int32_t rows, int32_t H, void* cuda_stream, int32_t sync);
 /* Scaled masked softmax of attention over rows of S <= 512 scores: row r belongs to sequence
  * r / rows_per_seq; key j is valid iff j < d_seq_lens[sequence] (NULL: all valid); masked
  * probabilities are exactly 0.  May run in place.  The backward call overwrites dp with

@@ -106,7 +106,7 @@ _P = C.c_void_p
 lib.mslt_debug_starve_next_gemm.argtypes = [C.c_int32]
 lib.mslt_debug_check_guards.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
 lib.mslt_op_layernorm.argtypes = [C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
-lib.mslt_op_layernorm_bwd.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, _P, C.c_int32]
+lib.mslt_op_layernorm_bwd.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, _P, C.c_int32]
 lib.mslt_op_softmax.argtypes = [C.c_int32, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
 lib.mslt_op_softmax_bwd.argtypes = [C.c_int32, _P, _P, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
 lib.mslt_op_attention.argtypes = [_P, _P, _P, _P, C.c_int32, C.c_int32, C.c_int32, C.c_float, _P, _P, C.c_int32]
@@ -172,9 +172,11 @@ def mslt_op_layernorm(z, gamma, beta, y, stats, eps: float, stream: int, sync: b
                                  _ptr(stats), z.shape[0], z.shape[1], eps, C.c_void_p(stream), int(sync)))
 
 
-def mslt_op_layernorm_bwd(dy, z, stats, gamma, dz, dgamma, dbeta, stream: int, sync: bool = True) -> None:
+def mslt_op_layernorm_bwd(dy, z, stats, gamma, dz, dgamma, dbeta, stream: int, sync: bool = True,
+                          dbias=None) -> None:
+    """dbias (fp32 [H] or None) receives += the column sums of dz."""
     _check(lib.mslt_op_layernorm_bwd(_dt(z), dy.data_ptr(), z.data_ptr(), stats.data_ptr(), gamma.data_ptr(),
-                                     dz.data_ptr(), dgamma.data_ptr(), dbeta.data_ptr(), z.shape[0],
+                                     dz.data_ptr(), dgamma.data_ptr(), dbeta.data_ptr(), _ptr(dbias), z.shape[0],
                                      z.shape[1], C.c_void_p(stream), int(sync)))
 
 

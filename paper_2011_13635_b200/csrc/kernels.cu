@@ -210,101 +210,146 @@ embed_ln_kernel(const int* __restrict__ tokens, const T* __restrict__ word,
 
 // ---------------------------------------------------------------------------------------
 // LayerNorm backward: dz = rstd * (dxhat - mean(dxhat) - xhat * mean(dxhat * xhat)),
-// dgamma += sum_rows dy * xhat, dbeta += sum_rows dy (fp32 atomics, one per column per block).
+// dgamma += sum_rows dy * xhat, dbeta += sum_rows dy and, when asked for, dbias += sum_rows dz
+// (the bias gradient of the linear layer whose output was normalised) - fp32 atomics, one per
+// column per block.
+// A row is split over NSLICE warps, each owning one 16-byte vector per lane, so that the column
+// accumulators cost a lane 3 x 8 registers instead of 3 x 24 and twice as many loads are in
+// flight per SM; a warp works on LN_BWD_ROWS rows at once and the NSLICE partial row sums meet in shared
+// memory (double-buffered: one block barrier per LR rows).
 // ---------------------------------------------------------------------------------------
-template <typename T, int MAXE>
-__global__ void __launch_bounds__(128)
+template <typename T, int NSLICE, int RG, int LN_BWD_ROWS>
+__global__ void __launch_bounds__(NSLICE * RG * 32, 1)
 ln_bwd_kernel(const T* __restrict__ dy, const T* __restrict__ z, const float* __restrict__ stats,
               const float* __restrict__ gamma, T* __restrict__ dz, float* __restrict__ dgamma,
-              float* __restrict__ dbeta, int rows, int H) {
+              float* __restrict__ dbeta, float* __restrict__ dbias, int rows, int H) {
   constexpr int VN = VecT<T>::N;
-  constexpr int NV = MAXE / VN;
-  constexpr int NW = 4;  // warps per block
-  __shared__ float red[NW][MAXE * 32];
+  constexpr int LR = LN_BWD_ROWS;  // rows a warp has in flight
+  typedef typename VecT<T>::Raw Raw;
+  __shared__ float part[2][RG][LR][NSLICE][2];
+  __shared__ float red[RG][NSLICE * 32 * VN];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int gw = blockIdx.x * NW + warp, nw = gridDim.x * NW;
-  float ag[MAXE], ab[MAXE], g[MAXE];
+  const int slice = warp % NSLICE, rg = warp / NSLICE;
+  const int c = (slice * 32 + lane) * VN;
+  const bool col_ok = c < H;
+  float g[VN], ag[VN], ab[VN], az[VN];
 #pragma unroll
-  for (int i = 0; i < MAXE; i++) { ag[i] = 0.f; ab[i] = 0.f; g[i] = 0.f; }
+  for (int e = 0; e < VN; e++) { g[e] = 0.f; ag[e] = 0.f; ab[e] = 0.f; az[e] = 0.f; }
+  if (col_ok) {
 #pragma unroll
-  for (int i = 0; i < NV; i++) {
-    const int c = (lane + 32 * i) * VN;
-    if (c < H) {
-#pragma unroll
-      for (int e = 0; e < VN; e += 4) {
-        const float4 g4 = *reinterpret_cast<const float4*>(gamma + c + e);
-        g[i * VN + e] = g4.x; g[i * VN + e + 1] = g4.y; g[i * VN + e + 2] = g4.z; g[i * VN + e + 3] = g4.w;
-      }
+    for (int e = 0; e < VN; e += 4) {
+      const float4 g4 = *reinterpret_cast<const float4*>(gamma + c + e);
+      g[e] = g4.x; g[e + 1] = g4.y; g[e + 2] = g4.z; g[e + 3] = g4.w;
     }
   }
   const float invH = 1.0f / (float)H;
-  for (int row = gw; row < rows; row += nw) {
-    const float mean = stats[2 * (int64_t)row], rstd = stats[2 * (int64_t)row + 1];
-    // the row stays packed in registers between the two passes (fewer registers, more warps)
-    typename VecT<T>::Raw ra[NV], rb[NV];
-    float s1 = 0.f, s2 = 0.f;
+  int buf = 0;
+  for (int base = blockIdx.x * (RG * LR); base < rows; base += gridDim.x * (RG * LR), buf ^= 1) {
+    const int row0 = base + rg * LR;
+    Raw ra[LR], rb[LR];
+    float mean[LR], rstd[LR];
 #pragma unroll
-    for (int i = 0; i < NV; i++) {
-      const int c = (lane + 32 * i) * VN;
-      if (c < H) {
-        ra[i] = VecT<T>::load_raw(dy + (int64_t)row * H + c);
-        rb[i] = VecT<T>::load_raw(z + (int64_t)row * H + c);
+    for (int k = 0; k < LR; k++) {
+      const bool ok = col_ok && row0 + k < rows;
+      if (ok) {
+        ra[k] = VecT<T>::load_raw(dy + (int64_t)(row0 + k) * H + c);
+        rb[k] = VecT<T>::load_raw(z + (int64_t)(row0 + k) * H + c);
       }
+      const int rr = min(row0 + k, rows - 1);
+      mean[k] = stats[2 * (int64_t)rr];
+      rstd[k] = stats[2 * (int64_t)rr + 1];
     }
+    // Packed two-wide fp32 arithmetic and row constants folded once per row keep this at a few
+    // instructions per element (the plain form was bound by instruction issue, not by memory):
+    //   q = sum dy*gamma*z gives sum dy*gamma*xhat = rstd * (q - mean * s1);
+    //   xhat = z * rstd + nmr;  dz = dy * (gamma * rstd) + z * c2 + c3.
+    float s1[LR], s2[LR];
 #pragma unroll
-    for (int i = 0; i < NV; i++) {
-      const int c = (lane + 32 * i) * VN;
-      if (c < H) {
+    for (int k = 0; k < LR; k++) {
+      float2 t1 = make_float2(0.f, 0.f), tq = make_float2(0.f, 0.f);
+      if (col_ok && row0 + k < rows) {
         float a[VN], b[VN];
-        VecT<T>::unpack(ra[i], a);
-        VecT<T>::unpack(rb[i], b);
+        VecT<T>::unpack(ra[k], a);
+        VecT<T>::unpack(rb[k], b);
+        const float2 r2 = make_float2(rstd[k], rstd[k]), n2 = make_float2(-mean[k] * rstd[k], -mean[k] * rstd[k]);
 #pragma unroll
-        for (int e = 0; e < VN; e++) {
-          const float xhat = (b[e] - mean) * rstd;
-          const float dxh = a[e] * g[i * VN + e];
-          s1 += dxh;
-          s2 += dxh * xhat;
-          ag[i * VN + e] += a[e] * xhat;
-          ab[i * VN + e] += a[e];
+        for (int e = 0; e < VN; e += 2) {
+          const float2 a2 = make_float2(a[e], a[e + 1]), b2 = make_float2(b[e], b[e + 1]);
+          const float2 dxh = __fmul2_rn(a2, make_float2(g[e], g[e + 1]));
+          t1 = __fadd2_rn(t1, dxh);
+          tq = __ffma2_rn(dxh, b2, tq);
+          const float2 xhat = __ffma2_rn(b2, r2, n2);
+          const float2 ga = __ffma2_rn(a2, xhat, make_float2(ag[e], ag[e + 1]));
+          const float2 ba = __fadd2_rn(a2, make_float2(ab[e], ab[e + 1]));
+          ag[e] = ga.x; ag[e + 1] = ga.y;
+          ab[e] = ba.x; ab[e + 1] = ba.y;
         }
       }
+      s1[k] = t1.x + t1.y;
+      s2[k] = tq.x + tq.y;
     }
-    s1 = warp_sum(s1) * invH;
-    s2 = warp_sum(s2) * invH;
 #pragma unroll
-    for (int i = 0; i < NV; i++) {
-      const int c = (lane + 32 * i) * VN;
-      if (c < H) {
+    for (int o = 16; o > 0; o >>= 1)
+#pragma unroll
+      for (int k = 0; k < LR; k++) {
+        s1[k] += __shfl_xor_sync(0xffffffffu, s1[k], o);
+        s2[k] += __shfl_xor_sync(0xffffffffu, s2[k], o);
+      }
+    if (NSLICE > 1) {
+      if (lane < LR) {
+        float v1 = s1[0], v2 = s2[0];
+#pragma unroll
+        for (int k = 1; k < LR; k++)
+          if (lane == k) { v1 = s1[k]; v2 = s2[k]; }
+        part[buf][rg][lane][slice][0] = v1;
+        part[buf][rg][lane][slice][1] = v2;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int k = 0; k < LR; k++) {
+        float t1 = 0.f, t2 = 0.f;
+#pragma unroll
+        for (int w = 0; w < NSLICE; w++) { t1 += part[buf][rg][k][w][0]; t2 += part[buf][rg][k][w][1]; }
+        s1[k] = t1; s2[k] = t2;
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < LR; k++) {
+      if (col_ok && row0 + k < rows) {
         float a[VN], b[VN], o[VN];
-        VecT<T>::unpack(ra[i], a);
-        VecT<T>::unpack(rb[i], b);
+        VecT<T>::unpack(ra[k], a);
+        VecT<T>::unpack(rb[k], b);
+        const float m1 = s1[k] * invH, m2 = rstd[k] * (s2[k] - mean[k] * s1[k]) * invH;
+        const float c2 = -rstd[k] * rstd[k] * m2, c3 = -rstd[k] * m1 - c2 * mean[k];
+        const float2 r2 = make_float2(rstd[k], rstd[k]), c22 = make_float2(c2, c2), c32 = make_float2(c3, c3);
 #pragma unroll
-        for (int e = 0; e < VN; e++) {
-          const float xhat = (b[e] - mean) * rstd;
-          o[e] = rstd * (a[e] * g[i * VN + e] - s1 - xhat * s2);
+        for (int e = 0; e < VN; e += 2) {
+          const float2 gr = __fmul2_rn(make_float2(g[e], g[e + 1]), r2);
+          const float2 o2 = __ffma2_rn(make_float2(a[e], a[e + 1]), gr,
+                                       __ffma2_rn(make_float2(b[e], b[e + 1]), c22, c32));
+          const float2 za = __fadd2_rn(o2, make_float2(az[e], az[e + 1]));
+          o[e] = o2.x; o[e + 1] = o2.y;
+          az[e] = za.x; az[e + 1] = za.y;
         }
-        VecT<T>::store(dz + (int64_t)row * H + c, o);
+        VecT<T>::store(dz + (int64_t)(row0 + k) * H + c, o);
       }
     }
   }
-  // block reduction of the column sums, then one atomic per column
+  // block reduction of the column sums over the row groups, then one atomic per column
 #pragma unroll
-  for (int pass = 0; pass < 2; pass++) {
+  for (int pass = 0; pass < 3; pass++) {
+    float* dst = pass == 0 ? dgamma : (pass == 1 ? dbeta : dbias);
+    if (dst == nullptr) continue;  // uniform over the block
     __syncthreads();
 #pragma unroll
-    for (int i = 0; i < NV; i++) {
-      const int c = (lane + 32 * i) * VN;
-#pragma unroll
-      for (int e = 0; e < VN; e++)
-        red[warp][c + e] = pass == 0 ? ag[i * VN + e] : ab[i * VN + e];
-    }
+    for (int e = 0; e < VN; e++)
+      red[rg][(slice * 32 + lane) * VN + e] = pass == 0 ? ag[e] : (pass == 1 ? ab[e] : az[e]);
     __syncthreads();
-    float* dst = pass == 0 ? dgamma : dbeta;
-    for (int c = threadIdx.x; c < H; c += 128) {
-      float s = 0.f;
+    for (int cc = threadIdx.x; cc < H; cc += NSLICE * RG * 32) {
+      float t = 0.f;
 #pragma unroll
-      for (int w = 0; w < NW; w++) s += red[w][c];
-      atomicAdd(dst + c, s);
+      for (int w = 0; w < RG; w++) t += red[w][cc];
+      atomicAdd(dst + cc, t);
     }
   }
 }
@@ -892,19 +937,24 @@ void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* p
 }
 
 void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, const float* gamma,
-                   void* dz, float* dgamma, float* dbeta, int rows, int H, cudaStream_t st) {
+                   void* dz, float* dgamma, float* dbeta, float* dbias, int rows, int H, cudaStream_t st) {
   if (rows <= 0) return;
-  // elements a lane holds: the smallest of 8 / 16 / 24 / 32 that covers the row keeps registers low
+  // warps per row: one 16-byte vector per lane; row groups fill the block up to 12-16 warps
   const int vn = bf ? 8 : 4;
-  const int need = (H + 32 * vn - 1) / (32 * vn) * vn;
-  const int blocks = std::min(div_up(rows, 4 * 2), 148 * 8);
-#define LN_BWD(E)                                                                                      \
-  DISPATCH_T(bf, (ln_bwd_kernel<T, E><<<blocks, 128, 0, st>>>((const T*)dy, (const T*)z, stats, gamma, \
-                                                              (T*)dz, dgamma, dbeta, rows, H)))
-  if (need <= 8) LN_BWD(8);
-  else if (need <= 16) LN_BWD(16);
-  else if (need <= 24) LN_BWD(24);
-  else LN_BWD(32);
+  const int nslice = (H + 32 * vn - 1) / (32 * vn);
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  // one block per SM walks the rows: the column sums end in one atomic per column and block
+#define LN_BWD(NS, RG)                                                                                   \
+  DISPATCH_T(bf, (ln_bwd_kernel<T, NS, RG, 4><<<std::min(div_up(rows, RG * 4), sms), NS * RG * 32, 0, st>>>( \
+                     (const T*)dy, (const T*)z, stats, gamma, (T*)dz, dgamma, dbeta, dbias, rows, H)))
+  if (nslice <= 1) LN_BWD(1, 8);
+  else if (nslice <= 2) LN_BWD(2, 6);
+  else if (nslice <= 3) LN_BWD(3, 4);
+  else if (nslice <= 4) LN_BWD(4, 3);
+  else if (nslice <= 6) LN_BWD(6, 2);
+  else LN_BWD(8, 2);
 #undef LN_BWD
 }
 

@@ -24,7 +24,7 @@ void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* p
                      const float* gamma, const float* beta, void* y, void* zstash, float* stats,
                      int rows, int S, int H, int V, float eps, int* status, cudaStream_t st);
 void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, const float* gamma,
-                   void* dz, float* dgamma, float* dbeta, int rows, int H, cudaStream_t st);
+                   void* dz, float* dgamma, float* dbeta, float* dbias, int rows, int H, cudaStream_t st);
 void launch_softmax_fwd(bool bf, const void* sc, void* p, const int* seq_lens, int rows, int S,
                         int rows_per_seq, float scale, cudaStream_t st);
 void launch_softmax_bwd(bool bf, void* dp, const void* p, int rows, int S, float scale,

@@ -480,17 +480,15 @@ int layer_backward(mslt_ctx* c, int l, const void* x_in, LayerBuf& b, const void
   Workspace& w = c->ws;
   const float scale = 1.0f / sqrtf((float)d);
   KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, dx, b.z2, b.st2, Wv(c, toff(c, l, "ln2.gamma")), w.dz2,
-                   G(c, toff(c, l, "ln2.gamma")), G(c, toff(c, l, "ln2.beta")), T, H, c->st));
+                   G(c, toff(c, l, "ln2.gamma")), G(c, toff(c, l, "ln2.beta")), G(c, toff(c, l, "ffn2.bias")), T, H, c->st));
   TRY(linear_wgrad(c, w.dz2, T, H, H, b.g, F, toff(c, l, "ffn2.weight")));
-  KL(PC_COLSUM, 1.0 * T * H * c->esz, launch_colsum(c->bf, w.dz2, H, T, H, G(c, toff(c, l, "ffn2.bias")), c->st));
   TRY(linear_dgrad(c, w.dz2, T, H, H, toff(c, l, "ffn2.weight"), F, w.dg, 2, b.u, nullptr));
   TRY(linear_wgrad(c, w.dg, T, F, F, b.y, H, toff(c, l, "ffn1.weight")));
   KL(PC_COLSUM, 1.0 * T * F * c->esz, launch_colsum(c->bf, w.dg, F, T, F, G(c, toff(c, l, "ffn1.bias")), c->st));
   TRY(linear_dgrad(c, w.dg, T, F, F, toff(c, l, "ffn1.weight"), H, w.dy, 0, nullptr, w.dz2));
   KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, w.dy, b.z1, b.st1, Wv(c, toff(c, l, "ln1.gamma")), w.dz1,
-                   G(c, toff(c, l, "ln1.gamma")), G(c, toff(c, l, "ln1.beta")), T, H, c->st));
+                   G(c, toff(c, l, "ln1.gamma")), G(c, toff(c, l, "ln1.beta")), G(c, toff(c, l, "out.bias")), T, H, c->st));
   TRY(linear_wgrad(c, w.dz1, T, H, H, b.c, H, toff(c, l, "out.weight")));
-  KL(PC_COLSUM, 1.0 * T * H * c->esz, launch_colsum(c->bf, w.dz1, H, T, H, G(c, toff(c, l, "out.bias")), c->st));
   TRY(linear_dgrad(c, w.dz1, T, H, H, toff(c, l, "out.weight"), H, w.dc, 0, nullptr, nullptr));
   const int64_t qs = (int64_t)S * 3 * H, ps = (int64_t)A * S * S, cs = (int64_t)S * H;
   if (c->bf && S <= 128 && S % 8 == 0 && d == 64 && !getenv_cuda_cores() && !getenv_unfused_attention()) {
@@ -580,7 +578,7 @@ int head_backward(mslt_ctx* c, int B, int S, int P, bool full) {
     TRY(run_gemm(c, g.d));
   }
   KL(PC_LN_BWD, 3.0 * R * H * c->esz, launch_ln_bwd(c->bf, w.dtm, w.gt, w.hst, Wv(c, toff(c, -1, "head.ln.gamma")), w.dgt,
-                   G(c, toff(c, -1, "head.ln.gamma")), G(c, toff(c, -1, "head.ln.beta")), R, H, c->st));
+                   G(c, toff(c, -1, "head.ln.gamma")), G(c, toff(c, -1, "head.ln.beta")), nullptr, R, H, c->st));
   KL(PC_OTHER, 3.0 * R * H * c->esz, launch_dgelu(c->bf, w.dgt, w.ut, (int64_t)R * H, c->st));
   TRY(linear_wgrad(c, w.dgt, R, H, H, w.hm, H, toff(c, -1, "head.transform.weight")));
   KL(PC_COLSUM, 1.0 * R * H * c->esz, launch_colsum(c->bf, w.dgt, H, R, H, G(c, toff(c, -1, "head.transform.bias")), c->st));
@@ -799,7 +797,7 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   }
   if (full) {
     KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, dx, w.z0, w.st0, Wv(c, toff(c, -1, "emb.ln.gamma")), w.dz2,
-                     G(c, toff(c, -1, "emb.ln.gamma")), G(c, toff(c, -1, "emb.ln.beta")), T, H, c->st));
+                     G(c, toff(c, -1, "emb.ln.gamma")), G(c, toff(c, -1, "emb.ln.beta")), nullptr, T, H, c->st));
     KL(PC_OTHER, 1.0 * T * H * c->esz, launch_embed_scatter(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
                             G(c, toff(c, -1, "emb.pos")), T, S, H, V, c->st));
   }

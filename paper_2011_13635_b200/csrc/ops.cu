@@ -182,14 +182,14 @@ int mslt_op_layernorm(int32_t dtype, const void* d_z, const float* d_gamma, cons
 }
 
 int mslt_op_layernorm_bwd(int32_t dtype, const void* d_dy, const void* d_z, const float* d_stats,
-                          const float* d_gamma, void* d_dz, float* d_dgamma, float* d_dbeta, int32_t rows,
-                          int32_t H, void* cuda_stream, int32_t sync) {
+                          const float* d_gamma, void* d_dz, float* d_dgamma, float* d_dbeta, float* d_dbias,
+                          int32_t rows, int32_t H, void* cuda_stream, int32_t sync) {
   if (!d_dy || !d_z || !d_stats || !d_gamma || !d_dz || !d_dgamma || !d_dbeta)
     return op_fail(MSLT_ERR_ARG, "layernorm_bwd: null pointer");
   int rc = check_rows("layernorm_bwd", dtype, rows, H, 8, 1024);
   if (rc) return rc;
   cudaStream_t st = (cudaStream_t)cuda_stream;
-  launch_ln_bwd(dtype == 1, d_dy, d_z, d_stats, d_gamma, d_dz, d_dgamma, d_dbeta, rows, H, st);
+  launch_ln_bwd(dtype == 1, d_dy, d_z, d_stats, d_gamma, d_dz, d_dgamma, d_dbeta, d_dbias, rows, H, st);
   return finish_op("layernorm_bwd", st, sync);
 }
 

@@ -87,9 +87,13 @@ def test_layernorm_forward_and_backward_match_oracle(dtype, rows, H):
     # backward
     dz = torch.empty_like(z)
     dgam = torch.zeros(H, device="cuda"); dbet = torch.zeros(H, device="cuda")
-    Bd.mslt_op_layernorm_bwd(dy, z, stats, d_g, dz, dgam, dbet, _stream())
+    dbias = torch.zeros(H, device="cuda")
+    Bd.mslt_op_layernorm_bwd(dy, z, stats, d_g, dz, dgam, dbet, _stream(), dbias=dbias)
     dz_ref, dg_ref, db_ref = O.layer_norm_backward(dy64, xhat, rstd, gamma.astype(np.float64))
     assert np.abs(dz.double().cpu().numpy() - dz_ref).max() / np.abs(dz_ref).max() < tol
+    # the fused bias gradient: column sums of dz (they nearly cancel within a row, so compare
+    # against the size of dz rather than of the sums)
+    assert np.abs(dbias.cpu().numpy() - dz_ref.sum(axis=0)).max() < (1e-4 if dtype == 0 else 2e-2) * np.abs(dz_ref).max() * np.sqrt(dz_ref.shape[0])
     assert np.abs(dgam.cpu().numpy() - dg_ref).max() / np.abs(dg_ref).max() < 1e-4
     assert np.abs(dbet.cpu().numpy() - db_ref).max() / np.abs(db_ref).max() < 1e-4
     # the column sums are accumulated: a second call doubles them
