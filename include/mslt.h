@@ -284,7 +284,7 @@ int mslt_op_colsum(int32_t dtype, const void* d_x, int64_t ld, int32_t rows, int
 
 /* Attention of one encoder layer in a single kernel (the paper defers the encoder to BERT,
  * Section 4.1: scaled dot-product attention with a key-padding mask), bf16 only, head width 64,
- * 1 <= S <= 128:  probs[b,h,i,:] = softmax over the valid keys j < d_seq_lens[b] (NULL: all S) of
+ * 1 <= S <= 512 (rows of more than 128 keys run a two-pass form of the kernel):  probs[b,h,i,:] = softmax over the valid keys j < d_seq_lens[b] (NULL: all S) of
  * scale * q_i . k_j, masked probabilities exactly 0;  ctx[b,i,h,:] = sum_j probs[b,h,i,j] v_j with
  * probs rounded to bf16 first.  d_qkv: device, [B*S, 3*heads*64] row-major, columns = queries |
  * keys | values, head h in columns h*64.. of each; d_probs: device, [B, heads, S, S] or NULL (not

@@ -302,6 +302,320 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   }
 }
 
+// ---- forward for rows of 129..512 keys -----------------------------------------------------------
+// A work item is (sequence, head, tile of 128 queries); the keys come in blocks of 128.  The scores
+// of a row do not fit tensor memory next to the context, so the item runs two passes over the key
+// blocks: pass 1 forms the row maximum and the sum of exponentials (S = Q K_j^T only), pass 2
+// forms the scores again, writes P_j = exp(.)/sum as bf16 and accumulates C += P_j V_j.  The
+// second score product costs the tensor pipe little; what it buys is an exact softmax with no
+// rescaling of the context, and probabilities that can be stored as they are.
+// The two softmax groups take alternate score accumulators of the same item (a thread owns one
+// query row in its group's blocks) and exchange their partial (max, sum) between the passes.
+constexpr int AL_KV_STAGES = 4;
+constexpr int AL_KV_BYTES = 2 * AT_TILE_BYTES;   // K block and V block: 32 KB
+constexpr int AL_P_BYTES = 2 * AT_TILE_BYTES;    // P_j as an MMA operand: 32 KB
+
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                     const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  uint8_t* q_smem = smem;                                   // two Q tiles, by item parity
+  uint8_t* kv_smem = q_smem + 2 * AT_TILE_BYTES;            // ring of K/V blocks
+  uint8_t* p_smem = kv_smem + AL_KV_STAGES * AL_KV_BYTES;   // one P block
+  uint8_t* staging = p_smem + AL_P_BYTES;
+  float2* xstat = (float2*)(staging + NUM_EPI_WARPS * AT_STAGING);  // [2 items][2 groups][128 rows] (max, sum)
+  uint64_t* bars = (uint64_t*)(xstat + 2 * 2 * 128);
+  uint64_t* qfull_bar = bars;                       // [2]
+  uint64_t* qempty_bar = bars + 2;                  // [2]
+  uint64_t* kvfull_bar = bars + 4;                  // [AL_KV_STAGES]
+  uint64_t* kvempty_bar = bars + 4 + AL_KV_STAGES;  // [AL_KV_STAGES]
+  uint64_t* sfull_bar = bars + 4 + 2 * AL_KV_STAGES;       // [2] scores of the group's next block complete
+  uint64_t* sempty_bar = sfull_bar + 2;                    // [2] read by the group
+  uint64_t* pready_bar = sfull_bar + 4;                    // P block in shared memory
+  uint64_t* pfree_bar = sfull_bar + 5;                     // second product has read it
+  uint64_t* ofull_bar = sfull_bar + 6;                     // context of the item complete
+  uint64_t* oempty_bar = sfull_bar + 7;                    // read by both groups
+  uint64_t* x_bar = sfull_bar + 8;                         // partial row statistics of both groups written
+  uint32_t* tmem_slot = (uint32_t*)(sfull_bar + 9);
+  volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (threadIdx.x == 0) {
+    for (int a = 0; a < 2; a++) {
+      mbar_init(smem_u32(&qfull_bar[a]), 1);
+      mbar_init(smem_u32(&qempty_bar[a]), 1);
+      mbar_init(smem_u32(&sfull_bar[a]), 1);
+      mbar_init(smem_u32(&sempty_bar[a]), AT_GROUP_WARPS);
+    }
+    for (int a = 0; a < AL_KV_STAGES; a++) {
+      mbar_init(smem_u32(&kvfull_bar[a]), 1);
+      mbar_init(smem_u32(&kvempty_bar[a]), 1);
+    }
+    mbar_init(smem_u32(pready_bar), AT_GROUP_WARPS);
+    mbar_init(smem_u32(pfree_bar), 1);
+    mbar_init(smem_u32(ofull_bar), 1);
+    mbar_init(smem_u32(oempty_bar), NUM_EPI_WARPS);
+    mbar_init(smem_u32(x_bar), NUM_EPI_WARPS);
+    *abort_flag = 0;
+    *reinterpret_cast<volatile long long*>(abort_flag + 1) = p.wait_limit;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                 "r"(AT_TMEM_COLS)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+  const int nkb = (p.S + 127) >> 7;   // key blocks
+  const int nqt = nkb;                // query tiles per (sequence, head)
+  const int n_my = ((int)blockIdx.x < p.items) ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+  // Per item there are 2 * nkb score products, numbered t = 0, 1, ... over the CTA's whole run; the
+  // accumulator and the softmax group of product t are t & 1, its K/V stage t % AL_KV_STAGES.
+
+  if (warp == 0 && lane == 0) {
+    // ------------------------------- TMA producer -------------------------------
+    bool ok = true;
+    uint32_t t = 0;
+    for (int i = 0; i < n_my && ok; i++) {
+      const int w = (int)blockIdx.x + i * (int)gridDim.x;
+      const int zh = w / nqt, qt = w - zh * nqt;
+      const int zo = zh / p.heads, zi = zh - zo * p.heads;
+      const uint32_t qb = (uint32_t)i & 1, quse = (uint32_t)i >> 1;
+      if (!mbar_wait(smem_u32(&qempty_bar[qb]), (quse & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      int c[4];
+      c[0] = 0; c[p.q_perm[0]] = qt * 128; c[p.q_perm[1]] = zi; c[p.q_perm[2]] = zo;
+      mbar_expect_tx(smem_u32(&qfull_bar[qb]), AT_TILE_BYTES);
+      tma_load_4d(smem_u32(q_smem + qb * AT_TILE_BYTES), &tmQ, smem_u32(&qfull_bar[qb]), c[0], c[1], c[2], c[3]);
+      for (int pass = 0; pass < 2 && ok; pass++)
+        for (int j = 0; j < nkb; j++, t++) {
+          const uint32_t s = t % AL_KV_STAGES, round = t / AL_KV_STAGES;
+          if (!mbar_wait(smem_u32(&kvempty_bar[s]), (round & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t fb = smem_u32(&kvfull_bar[s]);
+          const uint32_t dst = smem_u32(kv_smem + (size_t)s * AL_KV_BYTES);
+          mbar_expect_tx(fb, pass == 0 ? AT_TILE_BYTES : 2 * AT_TILE_BYTES);
+          c[0] = 0; c[p.k_perm[0]] = j * 128; c[p.k_perm[1]] = zi; c[p.k_perm[2]] = zo;
+          tma_load_4d(dst, &tmK, fb, c[0], c[1], c[2], c[3]);
+          if (pass == 1) {
+            c[0] = 0; c[p.v_perm[0]] = j * 128; c[p.v_perm[1]] = zi; c[p.v_perm[2]] = zo;
+            tma_load_4d(dst + AT_TILE_BYTES, &tmV, fb, c[0], c[1], c[2], c[3]);
+          }
+        }
+    }
+    if (!ok || *abort_flag) {  // give the copies in flight time to land before the CTA leaves
+      const long long t0 = now_cycles();
+      while (now_cycles() - t0 < 4000000ll) {}
+    }
+  } else if (warp == 1 && lane == 0) {
+    // ------------------------------- MMA issuer -------------------------------
+    bool ok = true;
+    const uint32_t hi = (uint32_t)(make_smem_desc(0, 16) >> 32);
+    const uint32_t lbo_mn_lo = (uint32_t)make_smem_desc(0, 64 * BK * 2);
+    const uint32_t p_lo = (uint32_t)make_smem_desc(smem_u32(p_smem), 16);
+    uint32_t t = 0, u = 0;  // score products and second products issued so far
+    for (int i = 0; i < n_my && ok; i++) {
+      const uint32_t qb = (uint32_t)i & 1, quse = (uint32_t)i >> 1;
+      if (!mbar_wait(smem_u32(&qfull_bar[qb]), quse & 1, abort_flag, p.status)) { ok = false; break; }
+      const uint32_t q_lo = (uint32_t)make_smem_desc(smem_u32(q_smem + qb * AT_TILE_BYTES), 16);
+      auto issue_scores = [&](uint32_t tt) -> bool {
+        const uint32_t s = tt % AL_KV_STAGES, round = tt / AL_KV_STAGES, b = tt & 1, use = tt >> 1;
+        if (!mbar_wait(smem_u32(&kvfull_bar[s]), round & 1, abort_flag, p.status)) return false;
+        if (!mbar_wait(smem_u32(&sempty_bar[b]), (use & 1) ^ 1, abort_flag, p.status)) return false;
+        tc_fence_after();
+        const uint32_t k_lo = (uint32_t)make_smem_desc(smem_u32(kv_smem + (size_t)s * AL_KV_BYTES), 16);
+#pragma unroll
+        for (int k = 0; k < BK / UMMA_K; k++) {
+          const uint64_t ad = ((uint64_t)hi << 32) | (q_lo + k * (UMMA_K * 2 / 16));
+          const uint64_t bd = ((uint64_t)hi << 32) | (k_lo + k * (UMMA_K * 2 / 16));
+          tc_mma(tmem_base + b * 128, ad, bd, p.idesc_s, k > 0 ? 1u : 0u);
+        }
+        tc_commit(smem_u32(&sfull_bar[b]));
+        return true;
+      };
+      auto issue_pv = [&](uint32_t tt, int j) -> bool {  // C (+)= P_j V_j; V_j sits in the stage of product tt
+        if (!mbar_wait(smem_u32(pready_bar), u & 1, abort_flag, p.status)) return false;
+        if (j == 0 && !mbar_wait(smem_u32(oempty_bar), ((uint32_t)i & 1) ^ 1, abort_flag, p.status)) return false;
+        tc_fence_after();
+        const uint32_t s = tt % AL_KV_STAGES;
+        const uint32_t sv = smem_u32(kv_smem + (size_t)s * AL_KV_BYTES + AT_TILE_BYTES);
+        const uint32_t v_lo = lbo_mn_lo | ((sv & 0x3FFFFu) >> 4);
+#pragma unroll
+        for (int kb = 0; kb < 2; kb++)
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; k++) {
+            const uint64_t ad = ((uint64_t)hi << 32) | (p_lo + kb * (AT_TILE_BYTES / 16) + k * (UMMA_K * 2 / 16));
+            const uint64_t bd = ((uint64_t)hi << 32) | (v_lo + kb * (AT_TILE_BYTES / 2 / 16) + k * (UMMA_K * 128 / 16));
+            tc_mma(tmem_base + AT_O_COL, ad, bd, p.idesc_o, (j > 0 || kb > 0 || k > 0) ? 1u : 0u);
+          }
+        tc_commit(smem_u32(pfree_bar));
+        tc_commit(smem_u32(&kvempty_bar[s]));
+        u++;
+        return true;
+      };
+      // pass 1: scores only; the K block is free as soon as its product has completed
+      for (int j = 0; j < nkb && ok; j++, t++) {
+        ok = issue_scores(t);
+        if (ok) tc_commit(smem_u32(&kvempty_bar[t % AL_KV_STAGES]));
+      }
+      // pass 2: the second product of block j - 1 is issued after the scores of block j
+      for (int j = 0; j < nkb && ok; j++, t++) {
+        ok = issue_scores(t);
+        if (ok && j > 0) ok = issue_pv(t - 1, j - 1);
+      }
+      if (ok) ok = issue_pv(t - 1, nkb - 1);
+      if (ok) {
+        tc_commit(smem_u32(ofull_bar));
+        tc_commit(smem_u32(&qempty_bar[qb]));
+      }
+    }
+    if (!ok || *abort_flag) {
+      tc_commit(smem_u32(&sfull_bar[0]));
+      const long long t0 = now_cycles();
+      while (now_cycles() - t0 < 2000000ll) {}
+    }
+  } else if (warp >= 2) {
+    // ------------------------------- softmax groups -------------------------------
+    const int q = warp & 3;
+    const int g = (warp - 2) >> 2;
+    uint8_t* stg = staging + (size_t)(warp - 2) * AT_STAGING;
+    const int r = q * 32 + lane;
+    const float sl2 = p.scale * 1.4426950408889634f;
+    const float2 k2 = splat2(sl2);
+    bool ok = true;
+    uint32_t t = 0, u = 0;
+    const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g * 128;
+    for (int i = 0; i < n_my && ok; i++) {
+      const int w = (int)blockIdx.x + i * (int)gridDim.x;
+      const int zh = w / nqt, qt = w - zh * nqt;
+      const int zo = zh / p.heads, zi = zh - zo * p.heads;
+      int len = p.seq_lens ? p.seq_lens[zo] : p.S;
+      len = min(max(len, 1), p.S);
+      float2 v[4][16];
+      // reads this group's next score block into v, masks it; returns its row maximum
+      auto load_block = [&](uint32_t tt, int j, float& bm) -> bool {
+        if (!mbar_wait(smem_u32(&sfull_bar[g]), (tt >> 1) & 1, abort_flag, p.status)) return false;
+        tc_fence_after();
+#pragma unroll
+        for (int c = 0; c < 4; c++) tc_ld32(trow + c * 32, v[c]);
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&sempty_bar[g]));
+        float mc[4];
+#pragma unroll
+        for (int c = 0; c < 4; c++) {
+          mc[c] = -INFINITY;
+          const int k0 = j * 128 + c * 32;
+          if (k0 + 32 > len) {
+#pragma unroll
+            for (int e = 0; e < 16; e++) {
+              if (k0 + 2 * e >= len) v[c][e].x = -INFINITY;
+              if (k0 + 2 * e + 1 >= len) v[c][e].y = -INFINITY;
+            }
+          }
+#pragma unroll
+          for (int e = 0; e < 16; e++) mc[c] = fmaxf(mc[c], fmaxf(v[c][e].x, v[c][e].y));
+        }
+        bm = fmaxf(fmaxf(mc[0], mc[1]), fmaxf(mc[2], mc[3]));
+        return true;
+      };
+      // pass 1: running maximum (raw scores) and sum of 2^((s - max) * scale * log2 e)
+      float mr = -INFINITY, l = 0.f;
+      for (int j = 0; j < nkb && ok; j++, t++) {
+        if ((t & 1) != (uint32_t)g) continue;
+        float bm;
+        if (!load_block(t, j, bm)) { ok = false; break; }
+        const float mn = fmaxf(mr, bm);
+        if (mn == -INFINITY) continue;  // nothing valid so far
+        const float2 nm2 = splat2(-mn * sl2);
+        float2 sc[4];
+#pragma unroll
+        for (int c = 0; c < 4; c++) {
+          sc[c] = make_float2(0.f, 0.f);
+#pragma unroll
+          for (int e = 0; e < 16; e++) {
+            const float2 a = __ffma2_rn(v[c][e], k2, nm2);
+            sc[c] = __fadd2_rn(sc[c], make_float2(fast_exp2(a.x), fast_exp2(a.y)));
+          }
+        }
+        const float bs = ((sc[0].x + sc[0].y) + (sc[1].x + sc[1].y)) + ((sc[2].x + sc[2].y) + (sc[3].x + sc[3].y));
+        l = l * fast_exp2((mr - mn) * sl2) + bs;  // 2^(-inf) = 0 on the first valid block
+        mr = mn;
+      }
+      if (!ok) break;
+      // exchange with the other group
+      float2* xs = xstat + ((i & 1) * 2) * 128;
+      xs[g * 128 + r] = make_float2(mr, l);
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(x_bar));
+      if (!mbar_wait(smem_u32(x_bar), (uint32_t)i & 1, abort_flag, p.status)) { ok = false; break; }
+      const float2 other = xs[(g ^ 1) * 128 + r];
+      const float M = fmaxf(mr, other.x);  // finite: at least one key of the row is valid
+      const float L = l * fast_exp2((mr - M) * sl2) + other.y * fast_exp2((other.x - M) * sl2);
+      const float2 inv = splat2(1.0f / L), nM2 = splat2(-M * sl2);
+      // pass 2
+      for (int j = 0; j < nkb && ok; j++, t++) {
+        if ((t & 1) != (uint32_t)g) { u++; continue; }
+        float bm;
+        if (!load_block(t, j, bm)) { ok = false; break; }
+#pragma unroll
+        for (int c = 0; c < 4; c++)
+#pragma unroll
+          for (int e = 0; e < 16; e++) {
+            const float2 a = __ffma2_rn(v[c][e], k2, nM2);
+            v[c][e] = __fmul2_rn(make_float2(fast_exp2(a.x), fast_exp2(a.y)), inv);
+          }
+        // the single P block is free once the previous second product has read it
+        if (!mbar_wait(smem_u32(pfree_bar), (u & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+        uint8_t* prow = p_smem + r * 128;
+#pragma unroll
+        for (int c = 0; c < 4; c++)
+#pragma unroll
+          for (int e4 = 0; e4 < 4; e4++) {
+            uint4 pk;
+            __nv_bfloat162* h = reinterpret_cast<__nv_bfloat162*>(&pk);
+#pragma unroll
+            for (int e = 0; e < 4; e++) h[e] = __float22bfloat162_rn(v[c][4 * e4 + e]);
+            *reinterpret_cast<uint4*>(prow + (c >> 1) * AT_TILE_BYTES + ((((c & 1) * 4 + e4) ^ (r & 7)) << 4)) = pk;
+          }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(pready_bar));
+        u++;
+        if (p.P != nullptr) {
+          bf16* pg = p.P + zo * p.p_bo + zi * p.p_bi + (long long)qt * 128 * p.S;
+#pragma unroll
+          for (int c = 0; c < 4; c++)
+            if (j * 128 + c * 32 < p.S)
+              stage_store_bf16(stg, lane, v[c], pg, p.S, q * 32, j * 128 + c * 32, p.S - qt * 128, p.S, p.vec_ok_p);
+        }
+      }
+      if (!ok) break;
+      // context tile: this group stores 32 of its 64 columns
+      if (!mbar_wait(smem_u32(ofull_bar), (uint32_t)i & 1, abort_flag, p.status)) { ok = false; break; }
+      tc_fence_after();
+      tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + AT_O_COL + (uint32_t)g * 32, v[0]);
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_u32(oempty_bar));
+      bf16* cg = p.C + zo * p.c_bo + zi * p.c_bi + (long long)qt * 128 * p.c_ld;
+      stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, g * 32, p.S - qt * 128, 64, p.vec_ok_c);
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(AT_TMEM_COLS)
+                 : "memory");
+  }
+}
+
 // ---- backward ---------------------------------------------------------------------------------------
 // Per (sequence, head) item, with P the saved probabilities and dC the gradient of the context:
 //   dV = P^T dC,  dP = dC V^T,  dS = P o (dP - rowsum(dP o P)) * scale,  dQ = dS K,  dK = dS^T Q.
@@ -583,14 +897,15 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
     cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     if (num_sms <= 0) { snprintf(err, 256, "attention: no CUDA device"); return MSLT_ERR_CUDA; }
   }
-  if (d != 64 || S < 1 || S > 128 || B < 1 || A < 1 || !status) {
-    snprintf(err, 256, "attention: the fused kernel needs head width 64 and 1 <= S <= 128");
+  if (d != 64 || S < 1 || S > 512 || B < 1 || A < 1 || !status) {
+    snprintf(err, 256, "attention: the fused kernel needs head width 64 and 1 <= S <= 512");
     return MSLT_ERR_ARG;
   }
+  const bool long_rows = S > 128;  // several key blocks per row: the two-pass kernel
   const long long H = (long long)A * d;
   AttnParams p;
   memset(&p, 0, sizeof(p));
-  p.S = S; p.heads = A; p.items = B * A; p.scale = scale; p.seq_lens = seq_lens;
+  p.S = S; p.heads = A; p.items = B * A * (long_rows ? (S + 127) / 128 : 1); p.scale = scale; p.seq_lens = seq_lens;
   p.P = (bf16*)probs; p.p_bo = (long long)A * S * S; p.p_bi = (long long)S * S;
   p.C = (bf16*)ctx; p.c_ld = H; p.c_bo = (long long)S * H; p.c_bi = d;
   p.vec_ok_p = (S % 8 == 0 && ((uintptr_t)probs & 15) == 0) ? 1 : 0;
@@ -606,9 +921,29 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
   if (rc) return rc;
   rc = get_map(base + H, S, d, 3 * H, 1, (long long)S * 3 * H, d, A, B, BM, &mk, err);
   if (rc) return rc;
-  rc = get_map(base + 2 * H, d, S, 1, 3 * H, (long long)S * 3 * H, d, A, B, 64, &mv, err);
+  // V: the short kernel reads it as two boxes of 64 keys with the head width contiguous; the long
+  // one as one box of 128 key rows, which are the same bytes in shared memory
+  if (long_rows) rc = get_map(base + 2 * H, S, d, 3 * H, 1, (long long)S * 3 * H, d, A, B, BM, &mv, err);
+  else rc = get_map(base + 2 * H, d, S, 1, 3 * H, (long long)S * 3 * H, d, A, B, 64, &mv, err);
   if (rc) return rc;
   for (int i = 0; i < 3; i++) { p.q_perm[i] = mq.perm[i]; p.k_perm[i] = mk.perm[i]; p.v_perm[i] = mv.perm[i]; }
+  if (long_rows) {
+    const size_t smem_long = 2 * (size_t)AT_TILE_BYTES + (size_t)AL_KV_STAGES * AL_KV_BYTES + AL_P_BYTES +
+                             NUM_EPI_WARPS * AT_STAGING + 2 * 2 * 128 * sizeof(float2) + 1024 + 256;
+    if ((int)smem_long > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
+    static bool attr_long = false;
+    if (!attr_long) {
+      cudaError_t e = cudaFuncSetAttribute(attn_fwd_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+      if (e != cudaSuccess) { snprintf(err, 256, "attention: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+      attr_long = true;
+    }
+    const int grid_long = p.items < num_sms ? p.items : num_sms;
+    attn_fwd_long_kernel<<<grid_long, NUM_THREADS, smem_long, st>>>(mq.map, mk.map, mv.map, p);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) { snprintf(err, 256, "attention: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+    g_attn_launches++;
+    return 0;
+  }
   const size_t smem_bytes = (size_t)AT_STAGES * AT_STAGE_BYTES + NUM_EPI_WARPS * AT_STAGING + 1024 + 256;
   if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
   static bool attr_set = false;

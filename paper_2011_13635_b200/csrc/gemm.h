@@ -20,7 +20,7 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
 // about 20 ms, so that its first wait runs out and the give-up path is exercised.
 void gemm_tc_starve_next(int on);
 
-// Fused attention forward (attn_tc.cu) for bf16, head width 64 and at most 128 keys per row:
+// Fused attention forward (attn_tc.cu) for bf16, head width 64 and at most 512 keys per row:
 //   probs[b,h,i,:] = softmax over valid keys j < seq_lens[b] of scale * q_i . k_j,  ctx = probs * v.
 // qkv is the fused projection [B*S, 3*A*d] (queries, keys, values; head h in columns h*d..);
 // probs ([B, A, S, S], may be null: not written) and ctx ([B*S, A*d]) are outputs.  `status` as for

@@ -99,22 +99,24 @@ ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ gamma, const fl
     float first[VN];
     VecT<T>::unpack(raw[r][0], first);
     const float x0 = __shfl_sync(0xffffffffu, first[0], 0);
-    float s1 = 0.f, s2 = 0.f;
+    // packed two-wide fp32 arithmetic: the kernel is bound by instruction issue, not by memory
+    float2 s1 = make_float2(0.f, 0.f), s2 = make_float2(0.f, 0.f);
+    const float2 nx0 = make_float2(-x0, -x0);
 #pragma unroll
     for (int i = 0; i < NV; i++) {
       if ((lane + 32 * i) * VN < H && row0 + r < rows) {
         float t[VN];
         VecT<T>::unpack(raw[r][i], t);
 #pragma unroll
-        for (int e = 0; e < VN; e++) {
-          const float d = t[e] - x0;
-          s1 += d;
-          s2 = fmaf(d, d, s2);
+        for (int e = 0; e < VN; e += 2) {
+          const float2 d = __fadd2_rn(make_float2(t[e], t[e + 1]), nx0);
+          s1 = __fadd2_rn(s1, d);
+          s2 = __ffma2_rn(d, d, s2);
         }
       }
     }
-    mean[r] = s1;
-    rstd[r] = s2;
+    mean[r] = s1.x + s1.y;
+    rstd[r] = s2.x + s2.y;
   }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) {
@@ -157,10 +159,17 @@ ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ gamma, const fl
 #pragma unroll
       for (int r = 0; r < ROWS; r++) {
         if (row0 + r < rows) {
+          // y = x * (gamma * rstd) + (beta - mean * rstd * gamma)
           float t[VN], o[VN];
           VecT<T>::unpack(raw[r][i], t);
+          const float2 r2 = make_float2(rstd[r], rstd[r]), nm2 = make_float2(-mean[r] * rstd[r], -mean[r] * rstd[r]);
 #pragma unroll
-          for (int e = 0; e < VN; e++) o[e] = g[e] * ((t[e] - mean[r]) * rstd[r]) + b[e];
+          for (int e = 0; e < VN; e += 2) {
+            const float2 g2 = make_float2(g[e], g[e + 1]);
+            const float2 o2 = __ffma2_rn(make_float2(t[e], t[e + 1]), __fmul2_rn(g2, r2),
+                                         __ffma2_rn(nm2, g2, make_float2(b[e], b[e + 1])));
+            o[e] = o2.x; o[e + 1] = o2.y;
+          }
           VecT<T>::store(y + (int64_t)(row0 + r) * H + c, o);
         }
       }

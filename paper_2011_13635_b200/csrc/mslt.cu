@@ -432,7 +432,7 @@ int layer_forward(mslt_ctx* c, int l, const void* x, LayerBuf& b, void* out, boo
   const float scale = 1.0f / sqrtf((float)d);
   TRY(linear_fwd(c, x, T, H, toff(c, l, "qkv.weight"), toff(c, l, "qkv.bias"), 3 * H, b.qkv, 0,
                  nullptr, nullptr));
-  if (c->bf && S <= 128 && d == 64 && !getenv_cuda_cores() && !getenv_unfused_attention()) {
+  if (c->bf && S <= 512 && d == 64 && !getenv_cuda_cores() && !getenv_unfused_attention()) {
     // the probabilities go to memory only where the backward pass will read them
     TRY(run_attention(c, b.qkv, save ? b.p : nullptr, b.c, seq_lens, B, S, A, d, scale));
   } else {

@@ -161,7 +161,9 @@ def test_op_argument_checks():
 
 
 @pytest.mark.parametrize("B,S,A,masked", [(2, 128, 2, False), (3, 128, 12, True), (2, 100, 3, True),
-                                          (5, 64, 2, True), (1, 24, 1, False), (37, 128, 12, True)])
+                                          (5, 64, 2, True), (1, 24, 1, False), (37, 128, 12, True),
+                                          (2, 256, 2, False), (3, 512, 4, True), (2, 384, 3, True),
+                                          (3, 200, 2, True), (40, 512, 16, True), (1, 136, 1, False)])
 @pytest.mark.parametrize("want_probs", [True, False], ids=["probs", "noprobs"])
 def test_fused_attention_matches_oracle(B, S, A, masked, want_probs):
     """Scores, masked softmax and context in one kernel against the oracle's definition
@@ -208,7 +210,7 @@ def test_fused_attention_rejects_other_shapes():
     ctx = torch.zeros((256, 64), device="cuda", dtype=torch.bfloat16)
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     with pytest.raises(Bd.MsltError):
-        Bd.mslt_op_attention(qkv, None, ctx, None, 1, 256, 1, 0.125, status, _stream())
+        Bd.mslt_op_attention(qkv, None, ctx, None, 1, 1024, 1, 0.125, status, _stream())
     with pytest.raises(Bd.MsltError):
         Bd.mslt_op_attention(qkv, None, ctx, None, 0, 128, 1, 0.125, status, _stream())
 
