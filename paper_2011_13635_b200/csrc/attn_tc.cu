@@ -49,6 +49,26 @@ struct AttnParams {
   uint32_t idesc_s, idesc_o;
 };
 
+// Four 32-column reads of a row in flight together, one wait for all.
+__device__ __forceinline__ void tc_ld128(uint32_t taddr, float2 (&v)[4][16]) {
+  uint32_t r0[32], r1[32], r2[32], r3[32];
+  tc_ld32_issue(taddr, r0);
+  tc_ld32_issue(taddr + 32, r1);
+  tc_ld32_issue(taddr + 64, r2);
+  tc_ld32_issue(taddr + 96, r3);
+  tc_ld32_wait(r0);
+  tc_ld32_wait(r1);
+  tc_ld32_wait(r2);
+  tc_ld32_wait(r3);
+#pragma unroll
+  for (int i = 0; i < 16; i++) {
+    v[0][i] = make_float2(__uint_as_float(r0[2 * i]), __uint_as_float(r0[2 * i + 1]));
+    v[1][i] = make_float2(__uint_as_float(r1[2 * i]), __uint_as_float(r1[2 * i + 1]));
+    v[2][i] = make_float2(__uint_as_float(r2[2 * i]), __uint_as_float(r2[2 * i + 1]));
+    v[3][i] = make_float2(__uint_as_float(r3[2 * i]), __uint_as_float(r3[2 * i + 1]));
+  }
+}
+
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -371,8 +391,15 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const int nkb = (p.S + 127) >> 7;   // key blocks
-  const int nqt = nkb;                // query tiles per (sequence, head)
+  const int nqt = (p.S + 127) >> 7;   // query tiles per (sequence, head); key blocks likewise
+  // Keys at or beyond the sequence's length have probability 0: an item covers only the
+  // ceil(len / 128) key blocks that hold valid keys, and a query tile that lies wholly in the
+  // padding is not computed at all (its context rows, which nothing may depend on, are zeroed).
+  // Every role derives the same counts from seq_lens; `ip` counts the items actually computed.
+  auto item_len = [&](int zo) {
+    int len = p.seq_lens ? p.seq_lens[zo] : p.S;
+    return min(max(len, 1), p.S);
+  };
   const int n_my = ((int)blockIdx.x < p.items) ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
   // Per item there are 2 * nkb score products, numbered t = 0, 1, ... over the CTA's whole run; the
   // accumulator and the softmax group of product t are t & 1, its K/V stage t % AL_KV_STAGES.
@@ -380,12 +407,16 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   if (warp == 0 && lane == 0) {
     // ------------------------------- TMA producer -------------------------------
     bool ok = true;
-    uint32_t t = 0;
+    uint32_t t = 0, ip = 0;
     for (int i = 0; i < n_my && ok; i++) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
       const int zh = w / nqt, qt = w - zh * nqt;
       const int zo = zh / p.heads, zi = zh - zo * p.heads;
-      const uint32_t qb = (uint32_t)i & 1, quse = (uint32_t)i >> 1;
+      const int len = item_len(zo);
+      if (qt * 128 >= len) continue;
+      const int nkb = (len + 127) >> 7;
+      const uint32_t qb = ip & 1, quse = ip >> 1;
+      ip++;
       if (!mbar_wait(smem_u32(&qempty_bar[qb]), (quse & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
       int c[4];
       c[0] = 0; c[p.q_perm[0]] = qt * 128; c[p.q_perm[1]] = zi; c[p.q_perm[2]] = zo;
@@ -416,9 +447,15 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t hi = (uint32_t)(make_smem_desc(0, 16) >> 32);
     const uint32_t lbo_mn_lo = (uint32_t)make_smem_desc(0, 64 * BK * 2);
     const uint32_t p_lo = (uint32_t)make_smem_desc(smem_u32(p_smem), 16);
-    uint32_t t = 0, u = 0;  // score products and second products issued so far
+    uint32_t t = 0, u = 0, ip = 0;  // score products, second products and items so far
     for (int i = 0; i < n_my && ok; i++) {
-      const uint32_t qb = (uint32_t)i & 1, quse = (uint32_t)i >> 1;
+      const int w = (int)blockIdx.x + i * (int)gridDim.x;
+      const int zh = w / nqt, qt = w - zh * nqt;
+      const int len = item_len(zh / p.heads);
+      if (qt * 128 >= len) continue;
+      const int nkb = (len + 127) >> 7;
+      const uint32_t qb = ip & 1, quse = ip >> 1, ipar = ip & 1;
+      ip++;
       if (!mbar_wait(smem_u32(&qfull_bar[qb]), quse & 1, abort_flag, p.status)) { ok = false; break; }
       const uint32_t q_lo = (uint32_t)make_smem_desc(smem_u32(q_smem + qb * AT_TILE_BYTES), 16);
       auto issue_scores = [&](uint32_t tt) -> bool {
@@ -438,7 +475,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       };
       auto issue_pv = [&](uint32_t tt, int j) -> bool {  // C (+)= P_j V_j; V_j sits in the stage of product tt
         if (!mbar_wait(smem_u32(pready_bar), u & 1, abort_flag, p.status)) return false;
-        if (j == 0 && !mbar_wait(smem_u32(oempty_bar), ((uint32_t)i & 1) ^ 1, abort_flag, p.status)) return false;
+        if (j == 0 && !mbar_wait(smem_u32(oempty_bar), ipar ^ 1, abort_flag, p.status)) return false;
         tc_fence_after();
         const uint32_t s = tt % AL_KV_STAGES;
         const uint32_t sv = smem_u32(kv_smem + (size_t)s * AL_KV_BYTES + AT_TILE_BYTES);
@@ -486,21 +523,34 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const float sl2 = p.scale * 1.4426950408889634f;
     const float2 k2 = splat2(sl2);
     bool ok = true;
-    uint32_t t = 0, u = 0;
+    uint32_t t = 0, u = 0, ip = 0;
     const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g * 128;
     for (int i = 0; i < n_my && ok; i++) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
       const int zh = w / nqt, qt = w - zh * nqt;
       const int zo = zh / p.heads, zi = zh - zo * p.heads;
-      int len = p.seq_lens ? p.seq_lens[zo] : p.S;
-      len = min(max(len, 1), p.S);
+      const int len = item_len(zo);
       float2 v[4][16];
+      bf16* cg = p.C + zo * p.c_bo + zi * p.c_bi + (long long)qt * 128 * p.c_ld;
+      bf16* pg = p.P ? p.P + zo * p.p_bo + zi * p.p_bi + (long long)qt * 128 * p.S : nullptr;
+      if (qt * 128 >= len) {
+        // a query tile in the padding: zero context rows (finite, so that masked reads stay harmless)
+#pragma unroll
+        for (int e = 0; e < 16; e++) v[0][e] = make_float2(0.f, 0.f);
+        stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, g * 32, p.S - qt * 128, 64, p.vec_ok_c);
+        if (pg != nullptr)
+          for (int n0 = g * 32; n0 < p.S; n0 += 64)
+            stage_store_bf16(stg, lane, v[0], pg, p.S, q * 32, n0, p.S - qt * 128, p.S, p.vec_ok_p);
+        continue;
+      }
+      const int nkb = (len + 127) >> 7;
+      const uint32_t ipar = ip & 1;
+      ip++;
       // reads this group's next score block into v, masks it; returns its row maximum
       auto load_block = [&](uint32_t tt, int j, float& bm) -> bool {
         if (!mbar_wait(smem_u32(&sfull_bar[g]), (tt >> 1) & 1, abort_flag, p.status)) return false;
         tc_fence_after();
-#pragma unroll
-        for (int c = 0; c < 4; c++) tc_ld32(trow + c * 32, v[c]);
+        tc_ld128(trow, v);
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&sempty_bar[g]));
@@ -547,11 +597,11 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
       if (!ok) break;
       // exchange with the other group
-      float2* xs = xstat + ((i & 1) * 2) * 128;
+      float2* xs = xstat + (ipar * 2) * 128;
       xs[g * 128 + r] = make_float2(mr, l);
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(x_bar));
-      if (!mbar_wait(smem_u32(x_bar), (uint32_t)i & 1, abort_flag, p.status)) { ok = false; break; }
+      if (!mbar_wait(smem_u32(x_bar), ipar, abort_flag, p.status)) { ok = false; break; }
       const float2 other = xs[(g ^ 1) * 128 + r];
       const float M = fmaxf(mr, other.x);  // finite: at least one key of the row is valid
       const float L = l * fast_exp2((mr - M) * sl2) + other.y * fast_exp2((other.x - M) * sl2);
@@ -585,8 +635,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(pready_bar));
         u++;
-        if (p.P != nullptr) {
-          bf16* pg = p.P + zo * p.p_bo + zi * p.p_bi + (long long)qt * 128 * p.S;
+        if (pg != nullptr) {
 #pragma unroll
           for (int c = 0; c < 4; c++)
             if (j * 128 + c * 32 < p.S)
@@ -595,13 +644,20 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
       }
       if (!ok) break;
       // context tile: this group stores 32 of its 64 columns
-      if (!mbar_wait(smem_u32(ofull_bar), (uint32_t)i & 1, abort_flag, p.status)) { ok = false; break; }
+      // key blocks past the length: their probabilities are 0 (this group zeroes its half of the columns)
+      if (pg != nullptr && nkb * 128 < p.S) {
+        float2 zr[16];
+#pragma unroll
+        for (int e = 0; e < 16; e++) zr[e] = make_float2(0.f, 0.f);
+        for (int n0 = nkb * 128 + g * 32; n0 < p.S; n0 += 64)
+          stage_store_bf16(stg, lane, zr, pg, p.S, q * 32, n0, p.S - qt * 128, p.S, p.vec_ok_p);
+      }
+      if (!mbar_wait(smem_u32(ofull_bar), ipar, abort_flag, p.status)) { ok = false; break; }
       tc_fence_after();
       tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + AT_O_COL + (uint32_t)g * 32, v[0]);
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(smem_u32(oempty_bar));
-      bf16* cg = p.C + zo * p.c_bo + zi * p.c_bi + (long long)qt * 128 * p.c_ld;
       stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, g * 32, p.S - qt * 128, 64, p.vec_ok_c);
     }
   }

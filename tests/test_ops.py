@@ -192,11 +192,14 @@ def test_fused_attention_matches_oracle(B, S, A, masked, want_probs):
     c_ref = np.einsum("bhij,bhjd->bhid", p_ref, v).transpose(0, 2, 1, 3).reshape(B * S, H)
     if want_probs:
         got = probs.float().cpu().numpy()
-        assert np.abs(got - p_ref).max() < 6e-3                              # bf16 resolution at p <= 1
         for b in range(B):
+            # rows at padded query positions are unspecified (a long-row kernel skips tiles of them)
+            assert np.abs(got[b, :, :lens[b]] - p_ref[b, :, :lens[b]]).max() < 6e-3   # bf16 resolution at p <= 1
             assert not got[b, :, :, lens[b]:].any()                          # masked keys exactly 0
+            assert np.isfinite(got[b]).all()
     # rows at padded query positions are unspecified: compare valid rows only
     got = ctx.float().cpu().numpy().reshape(B, S, H)
+    assert np.isfinite(got).all()                                            # padded rows too: later layers read them
     ref = c_ref.reshape(B, S, H)
     for b in range(B):
         err = np.abs(got[b, :lens[b]] - ref[b, :lens[b]]).max()
