@@ -392,6 +392,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
   const int nqt = (p.S + 127) >> 7;   // query tiles per (sequence, head); key blocks likewise
+  const int nzh = p.items / nqt;      // (sequence, head) pairs
   // Keys at or beyond the sequence's length have probability 0: an item covers only the
   // ceil(len / 128) key blocks that hold valid keys, and a query tile that lies wholly in the
   // padding is not computed at all (its context rows, which nothing may depend on, are zeroed).
@@ -410,7 +411,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint32_t t = 0, ip = 0;
     for (int i = 0; i < n_my && ok; i++) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
-      const int zh = w / nqt, qt = w - zh * nqt;
+      const int qt = w / nzh, zh = w - qt * nzh;  // query tile slowest: tiles that may be padding come last
       const int zo = zh / p.heads, zi = zh - zo * p.heads;
       const int len = item_len(zo);
       if (qt * 128 >= len) continue;
@@ -450,7 +451,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     uint32_t t = 0, u = 0, ip = 0;  // score products, second products and items so far
     for (int i = 0; i < n_my && ok; i++) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
-      const int zh = w / nqt, qt = w - zh * nqt;
+      const int qt = w / nzh, zh = w - qt * nzh;  // query tile slowest: tiles that may be padding come last
       const int len = item_len(zh / p.heads);
       if (qt * 128 >= len) continue;
       const int nkb = (len + 127) >> 7;
@@ -527,7 +528,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
     const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g * 128;
     for (int i = 0; i < n_my && ok; i++) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
-      const int zh = w / nqt, qt = w - zh * nqt;
+      const int qt = w / nzh, zh = w - qt * nzh;  // query tile slowest: tiles that may be padding come last
       const int zo = zh / p.heads, zi = zh - zo * p.heads;
       const int len = item_len(zo);
       float2 v[4][16];
