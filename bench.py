@@ -338,6 +338,17 @@ def run_ours(args, cfg):
                 note="step time of 9 frozen + 3 trainable layers over all 12 trainable, same shapes, "
                      "data and seed, one GPU, no communication")
             mf.close()
+        if world == 1 and cfg.dtype == "bf16" and cfg.seq <= 512 and args.isolated:
+            # the same kernels one at a time, back to back on rotating buffers larger than L2: no
+            # event pair per launch, so short kernels are not understated as in hbm_kernels
+            from paper_2011_13635_b200 import op_bench
+            recs = op_bench.main(["--rows", str(cfg.batch * cfg.seq), "--hidden", str(cfg.hidden), "--ffn", str(cfg.ffn),
+                                  "--heads", str(cfg.heads), "--seq", str(cfg.seq), "--batch", str(cfg.batch),
+                                  "--iters", "20", "--only", "attention,ln,colsum"], emit=None)
+            line["hbm_kernels_alone"] = {
+                r["kernel"]: dict(us=r["us"], gbs=r["gbs"], frac_of_measured_copy=r["gbs"] / peaks["hbm_gbs"])
+                for r in recs}
+            torch.cuda.empty_cache()
         if world == 1:
             n_seq = args.cpu_seqs
             line["cpu_baseline"], _ = cpu_baseline(cfg, n_seq)
@@ -356,6 +367,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seqs", type=int, default=8, help="sequences in the oracle's timed sample")
     ap.add_argument("--no-ratio", dest="ratio", action="store_false")
+    ap.add_argument("--no-isolated", dest="isolated", action="store_false",
+                    help="skip the one-kernel-at-a-time bandwidth figures")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
                     help="launch every timed step eagerly instead of replaying one captured step")
     args = ap.parse_args()

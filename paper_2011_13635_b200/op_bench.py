@@ -13,9 +13,11 @@ import argparse
 import json
 
 
-def main():
+def main(argv=None, emit=print):
+    """Runs the kernels and emits one JSON line per kernel; returns the list of records."""
     import torch
     from . import binding as Bd
+    records = []
     ap = argparse.ArgumentParser()
     ap.add_argument("--rows", type=int, default=16384)
     ap.add_argument("--hidden", type=int, default=768)
@@ -26,7 +28,7 @@ def main():
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp32"])
     ap.add_argument("--iters", type=int, default=40)
     ap.add_argument("--only", default="", help="comma-separated kernel groups: ln, colsum, softmax, attention, ce")
-    a = ap.parse_args()
+    a = ap.parse_args(argv)
     only = set(x for x in a.only.split(",") if x)
     want = lambda group: not only or group in only
     tdt = torch.bfloat16 if a.dtype == "bf16" else torch.float32
@@ -52,8 +54,10 @@ def main():
         e1.record()
         torch.cuda.synchronize()
         us = e0.elapsed_time(e1) / a.iters * 1e3
-        print(json.dumps(dict(kernel=name, dtype=a.dtype, bytes=nbytes, us=round(us, 2),
-                              gbs=round(nbytes / us / 1e3, 1))))
+        rec = dict(kernel=name, dtype=a.dtype, bytes=nbytes, us=round(us, 2), gbs=round(nbytes / us / 1e3, 1))
+        records.append(rec)
+        if emit is not None:
+            emit(json.dumps(rec))
 
     if want("attention") and a.dtype == "bf16" and a.seq <= 512:
         # fused attention of one layer: reads Q, K, V once, writes the context (and the probabilities)
@@ -78,7 +82,7 @@ def main():
             raise RuntimeError("the attention kernel reported a wait that ran out")
         del qs, ctx, probs
     if not (want("ln") or want("colsum") or want("softmax") or want("ce")):
-        return
+        return records
     gamma = torch.ones(H, device="cuda"); beta = torch.zeros(H, device="cuda")
     zs = rotation((T, H), tdt)
     y = torch.empty((T, H), device="cuda", dtype=tdt)
@@ -99,6 +103,8 @@ def main():
     gs = rotation((T, F), tdt)
     run("colsum_ffn", T * F * E, lambda i: Bd.mslt_op_colsum(gs[i], F, out, st, sync=False), len(gs))
     del gs, zs
+    if not (want("softmax") or want("ce")):
+        return records
     R, S = a.batch * a.heads * a.seq, a.seq
     ps = rotation((R, S), tdt)
     pout = torch.empty((R, S), device="cuda", dtype=tdt)
@@ -118,6 +124,7 @@ def main():
     run("cross_entropy(sync)", Rm * Vp * (4 + E),
         lambda i: Bd.mslt_op_cross_entropy(1 if a.dtype == "bf16" else 0, logits[i], labels, V, dl, loss,
                                            scratch, st), 2)
+    return records
 
 
 if __name__ == "__main__":
