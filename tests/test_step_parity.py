@@ -110,3 +110,35 @@ def test_forward_matches_oracle(cfg):
     assert abs(loss - nll.mean()) / nll.mean() < 1e-5
     assert m.mslt_debug_check_guards() == 0
     m.close()
+
+
+def test_bf16_step_with_unfused_attention_in_a_child_process():
+    """The batched-product attention path (what longer rows and odd lengths fall back to) is selected
+    by an environment switch the library reads once, so it runs in a child process: same parity
+    check as above on BERT-Base widths with a padding mask."""
+    import os
+    import subprocess
+    import sys
+    code = (
+        "import math\n"
+        "from paper_2011_13635_b200 import inputs as I\n"
+        "from tests import parity as PT\n"
+        "cfg = I.scaled(I.CONFIGS['base_stage'], layers=2, trainable=1, batch=3)\n"
+        "cfg = I.StageConfig('unfused', hidden=cfg.hidden, heads=cfg.heads, ffn=cfg.ffn, vocab=cfg.vocab,\n"
+        "                    max_pos=cfg.max_pos, layers=2, trainable=1, batch=3, seq=128, pred=cfg.pred,\n"
+        "                    dtype='bf16', varlen=(40, 128), seed_index=23)\n"
+        "m, oracle = PT.build_pair(cfg, lr=1e-4)\n"
+        "before = m.launch_count\n"
+        "PT.compare_step(m, oracle, cfg, I.make_batch(cfg), PT.TOL[cfg.dtype])\n"
+        "print('launches', m.launch_count - before)\n"
+        "m.close()\n")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    counts = {}
+    for unfused in ("0", "1"):
+        env = dict(os.environ, MSLT_UNFUSED_ATTENTION=unfused, PYTHONPATH=root)
+        r = subprocess.run([sys.executable, "-c", code], cwd=root, env=env, capture_output=True, text=True,
+                           timeout=600)
+        assert r.returncode == 0, r.stdout + r.stderr
+        counts[unfused] = int(r.stdout.strip().split()[-1])
+    # two launches per layer forward become three, one per trainable layer backward becomes five
+    assert counts["1"] > counts["0"]
