@@ -228,6 +228,9 @@ int mslt_op_gemm_enqueue(const mslt_gemm_desc* desc, void* cuda_stream, int32_t*
  * garbage.  The context and the device stay usable.
  */
 int mslt_debug_starve_next_gemm(int32_t on);
+/* The same hook for the fused attention kernels: the NEXT mslt_op_attention / mslt_op_attention_bwd
+ * call (or attention launch inside a step) runs with an idle producer and a 20 ms wait limit. */
+int mslt_debug_starve_next_attention(int32_t on);
 
 /*
  * Memory-safety check for tests: every buffer the library carves out of the workspace is followed

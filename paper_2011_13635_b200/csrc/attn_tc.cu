@@ -46,6 +46,7 @@ struct AttnParams {
   int fast_p, fast_c;  // rows may be stored directly with 32-byte stores
   int q_perm[3], k_perm[3], v_perm[3];
   long long wait_limit;
+  int starve;         // test hook: the producer issues no copies, so the first wait runs out
   int* status;
   uint32_t idesc_s, idesc_o;
 };
@@ -141,7 +142,7 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tmem_base = *tmem_slot;
   const int n_my = ((int)blockIdx.x < p.items) ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && !p.starve) {
     // ------------------------------- TMA producer -------------------------------
     bool ok = true;
     int issued = 0;
@@ -442,7 +443,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   // Per item there are 2 * nkb score products, numbered t = 0, 1, ... over the CTA's whole run; the
   // accumulator and the softmax group of product t are t & 1, its K/V stage t % AL_KV_STAGES.
 
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && !p.starve) {
     // ------------------------------- TMA producer -------------------------------
     bool ok = true;
     uint32_t t = 0, ip = 0;
@@ -742,6 +743,7 @@ struct AttnBwdParams {
   int vec_ok, fast;
   int q_perm[3], k_perm[3], v_perm[3], c_perm[3], p_perm[3];
   long long wait_limit;
+  int starve;         // test hook, as in the forward kernels
   int* status;
   uint32_t idesc_dv, idesc_dp, idesc_dq, idesc_dk;
 };
@@ -789,7 +791,7 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
   const uint32_t tmem_base = *tmem_slot;
   const int n_my = ((int)blockIdx.x < p.items) ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
 
-  if (warp == 0 && lane == 0) {
+  if (warp == 0 && lane == 0 && !p.starve) {
     // ------------------------------- TMA producer -------------------------------
     bool ok = true;
     int issued = 0;
@@ -1008,6 +1010,8 @@ attn_bwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 }  // namespace
 
 static std::atomic<long long> g_attn_launches{0};
+static std::atomic<int> g_attn_starve{0};
+void attn_starve_next(int on) { g_attn_starve.store(on ? 1 : 0); }
 long long attn_launches() { return g_attn_launches.load(); }
 
 int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens, int B, int S, int A, int d,
@@ -1037,6 +1041,10 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
   p.fast_p = (probs != nullptr && S % 32 == 0) ? row_fast(probs, S) : 0;
   p.wait_limit = WAIT_LIMIT_CYCLES;
   p.status = status;
+  if (g_attn_starve.exchange(0)) {  // armed by mslt_debug_starve_next_attention
+    p.starve = 1;
+    p.wait_limit = 40000000ll;  // about 20 ms
+  }
   // fp32 accumulate, bf16 x bf16; scores: both operands k-contiguous, N = 128; context: V row-contiguous, N = 64
   p.idesc_s = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(128 >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
   p.idesc_o = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 16) | ((uint32_t)(64 >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -1108,6 +1116,10 @@ int attn_bwd_launch(const void* qkv, const void* probs, const void* dctx, void* 
   p.fast = 0;  // direct 32-byte row stores measured slower here (58 vs 54 us): three 128-byte pieces per row
   p.wait_limit = WAIT_LIMIT_CYCLES;
   p.status = status;
+  if (g_attn_starve.exchange(0)) {  // armed by mslt_debug_starve_next_attention
+    p.starve = 1;
+    p.wait_limit = 40000000ll;  // about 20 ms
+  }
   // fp32 accumulate, bf16 x bf16, M = 128; bit 15 / 16: A / B operand with rows = k index
   const uint32_t common = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
   p.idesc_dv = common | (1u << 15) | (1u << 16) | ((uint32_t)(64 >> 3) << 17);

@@ -33,6 +33,8 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
 int attn_bwd_launch(const void* qkv, const void* probs, const void* dctx, void* dqkv, int B, int S, int A, int d,
                     float scale, int* status, cudaStream_t st, char* err);
 long long attn_launches();
+// Test hook like gemm_tc_starve_next, for the next attention launch (forward or backward).
+void attn_starve_next(int on);
 
 // Kernels launched by the GEMM front end since the library was loaded (for launch accounting).
 int64_t gemm_launches();

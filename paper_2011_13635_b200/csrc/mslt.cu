@@ -1009,6 +1009,11 @@ int mslt_debug_check_guards(mslt_ctx* c, int32_t* bad_out) {
   return 0;
 }
 
+int mslt_debug_starve_next_attention(int32_t on) {
+  attn_starve_next(on);
+  return 0;
+}
+
 int mslt_debug_starve_next_gemm(int32_t on) {
   gemm_tc_starve_next(on);
   return 0;

@@ -253,3 +253,46 @@ def test_fused_attention_backward_matches_oracle(B, S, A, masked):
     for which, name in enumerate(("dq", "dk", "dv")):
         err = np.abs(got[:, :, which] - want[:, :, which]).max() / np.abs(want[:, :, which]).max()
         assert err < 1.5e-2, (name, err)
+
+
+@pytest.mark.parametrize("which", ["forward", "forward_long_rows", "backward"])
+def test_attention_wait_that_runs_out_is_reported_and_leaves_the_device_usable(which):
+    """Every wait in the attention kernels is bounded.  With the test hook armed the next launch has
+    an idle producer and a 20 ms limit: the kernel must come back with the status bit set (no
+    fault, no hang), and the very next call must work and be correct again."""
+    import math
+    import torch
+    from paper_2011_13635_b200 import binding as Bd
+    B, A = 2, 2
+    S = 256 if which == "forward_long_rows" else 128
+    H = A * 64
+    rng = np.random.default_rng(5)
+    qkv = torch.from_numpy(rng.standard_normal((B * S, 3 * H)).astype(np.float32)).cuda().bfloat16()
+    ctx = torch.zeros((B * S, H), device="cuda", dtype=torch.bfloat16)
+    probs = torch.zeros((B, A, S, S), device="cuda", dtype=torch.bfloat16)
+    dqkv = torch.zeros((B * S, 3 * H), device="cuda", dtype=torch.bfloat16)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    scale = 1.0 / math.sqrt(64)
+
+    def call():
+        if which == "backward":
+            Bd.mslt_op_attention_bwd(qkv, probs, ctx, dqkv, B, S, A, scale, status, _stream())
+        else:
+            Bd.mslt_op_attention(qkv, probs, ctx, None, B, S, A, scale, status, _stream())
+
+    Bd.lib.mslt_debug_starve_next_attention(1)
+    with pytest.raises(Bd.MsltError) as ei:
+        call()
+    assert ei.value.code == -5
+    assert int(status.item()) & 1
+    status.zero_()
+    Bd.mslt_op_attention(qkv, probs, ctx, None, B, S, A, scale, status, _stream())   # disarmed: works again
+    assert int(status.item()) == 0
+    x = qkv.float().cpu().numpy().astype(np.float64).reshape(B, S, 3, A, 64)
+    q, k, v = (x[:, :, i].transpose(0, 2, 1, 3) for i in range(3))
+    p_ref = O.masked_softmax(np.einsum("bhid,bhjd->bhij", q, k) * scale, np.full(B, S))
+    c_ref = np.einsum("bhij,bhjd->bhid", p_ref, v).transpose(0, 2, 1, 3).reshape(B * S, H)
+    assert np.abs(ctx.float().cpu().numpy() - c_ref).max() / np.abs(c_ref).max() < 1.5e-2
+    if which == "backward":
+        call()
+        assert int(status.item()) == 0
