@@ -233,6 +233,14 @@ int mslt_debug_starve_next_gemm(int32_t on);
 int mslt_debug_starve_next_attention(int32_t on);
 
 /*
+ * Measurement hook: how the dtype-1 contraction kernel tiles its output from now on, process
+ * wide.  0 (the default): the library chooses; 1: one CTA per 128 x BN tile; 2: a pair of CTAs per
+ * 256 x 256 tile wherever the shape allows it.  Results are identical up to summation order; only
+ * the speed differs.  Used by the micro-benchmarks to compare the two forms on one shape.
+ */
+int mslt_debug_set_gemm_variant(int32_t variant);
+
+/*
  * Memory-safety check for tests: every buffer the library carves out of the workspace is followed
  * by a 256-byte guard band that no kernel may write and that is zero from mslt_create on.  Counts
  * the guard bands that are no longer zero (*bad_out, host; 0 = no stray write).  Synchronises. */

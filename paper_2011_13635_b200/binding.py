@@ -57,7 +57,8 @@ EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers",
            "mslt_op_cross_entropy_scratch_bytes", "mslt_op_cross_entropy_noalloc", "mslt_op_layernorm",
            "mslt_op_layernorm_bwd", "mslt_op_softmax", "mslt_op_softmax_bwd", "mslt_op_colsum",
            "mslt_op_attention", "mslt_op_attention_bwd",
-           "mslt_debug_starve_next_gemm", "mslt_debug_starve_next_attention", "mslt_debug_check_guards"]
+           "mslt_debug_starve_next_gemm", "mslt_debug_starve_next_attention", "mslt_debug_check_guards",
+           "mslt_debug_set_gemm_variant"]
 
 lib.mslt_last_error.restype = C.c_char_p
 lib.mslt_last_error.argtypes = [C.c_void_p]
@@ -105,6 +106,7 @@ lib.mslt_op_cross_entropy_noalloc.argtypes = [C.c_int32, C.c_void_p, C.c_int64, 
 _P = C.c_void_p
 lib.mslt_debug_starve_next_gemm.argtypes = [C.c_int32]
 lib.mslt_debug_starve_next_attention.argtypes = [C.c_int32]
+lib.mslt_debug_set_gemm_variant.argtypes = [C.c_int32]
 lib.mslt_debug_check_guards.argtypes = [C.c_void_p, C.POINTER(C.c_int32)]
 lib.mslt_op_layernorm.argtypes = [C.c_int32, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, C.c_float, _P, C.c_int32]
 lib.mslt_op_layernorm_bwd.argtypes = [C.c_int32, _P, _P, _P, _P, _P, _P, _P, _P, C.c_int32, C.c_int32, _P, C.c_int32]

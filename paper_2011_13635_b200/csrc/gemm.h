@@ -19,6 +19,8 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
 // Test hook: the next tensor-core launch gets a producer that issues no copies and a wait limit of
 // about 20 ms, so that its first wait runs out and the give-up path is exercised.
 void gemm_tc_starve_next(int on);
+// Measurement hook: 0 = automatic tiling, 1 = one CTA per tile, 2 = CTA pairs wherever possible.
+void gemm_tc_set_variant(int variant);
 
 // Fused attention forward (attn_tc.cu) for bf16, head width 64 and at most 512 keys per row:
 //   probs[b,h,i,:] = softmax over valid keys j < seq_lens[b] of scale * q_i . k_j,  ctx = probs * v.

@@ -2,12 +2,16 @@
 //   D[z][m][n] = epilogue(alpha * sum_k A[z](m,k) * B[z](n,k)),  fp32 accumulation in TMEM.
 //
 // One persistent CTA per SM walks a list of (split, batch, m-tile, n-tile) work items.
-//   warp 0   : TMA producer.  128-byte-swizzled operand tiles go global -> shared through a ring
-//              of stages, each guarded by a full/empty mbarrier pair.
+//   warps 0, 2, 3: TMA producers (one thread each).  128-byte-swizzled operand tiles go global ->
+//              shared through a ring of stages, each guarded by a full/empty mbarrier pair.  The
+//              k blocks are dealt out round robin: measured on B200, one thread needs about 560
+//              cycles for {wait, expect_tx, two tile copies} however small the tiles are, more than
+//              the 512 cycles the tensor core takes for a 128 x 256 x 64 block, while several
+//              threads in different warps issue side by side at the same per-thread cost.
 //   warp 1   : allocates tensor memory and issues tcgen05.mma (one thread) for 128 x BN x 16
-//              steps; tcgen05.commit hands shared-memory stages back to the producer and
+//              steps; tcgen05.commit hands shared-memory stages back to the producers and
 //              accumulators over to the epilogue.
-//   warps 2-9: epilogue.  Two warps per 32-lane quarter of TMEM read the accumulator with
+//   warps 4-11: epilogue.  Two warps per 32-lane quarter of TMEM read the accumulator with
 //              tcgen05.ld, apply scale, bias, GELU / GELU', residual, and store bf16 or fp32
 //              (plain, or as vector reductions for split-k) through a swizzled staging buffer so
 //              that global stores are whole row segments.  Two accumulators of up to 256 columns
@@ -32,6 +36,10 @@
 namespace mslt {
 
 namespace {
+
+constexpr int NUM_PRODUCERS = 3;                              // warps 0, 2, 3
+constexpr int FIRST_EPI_WARP = 4;                             // warps 4..11 (warp & 3 = TMEM lane quarter)
+constexpr int GEMM_THREADS = 32 * (FIRST_EPI_WARP + NUM_EPI_WARPS);
 
 struct TcParams {
   int M, N, K, batch, hdiv;
@@ -163,9 +171,9 @@ __device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------
-// 10 warps are allocated registers as 12, which caps a thread at 168 registers
+// 12 warps: a thread may use up to 168 registers
 template <int kMode, bool kPair>
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const TcParams p) {
   constexpr bool kSoftmax = kMode == EPI_SOFTMAX;
@@ -182,8 +190,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int mt_rows = kPair ? 2 * BM : BM;      // rows of a work item's output tile
   const int w_first = kPair ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int w_step = kPair ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  // A ring stage holds KSUB 64-deep k blocks of both operands ("a round").  The issuing thread
+  // spends a fixed ~250-350 cycles per round on its barrier hand-shakes whatever the round holds;
+  // with four MMAs (512 cycles of tensor-core work) per round that kept the tensor core waiting,
+  // with eight it does not.  The pair form has the shared memory for three such stages.
+  constexpr int KSUB = kPair ? 2 : 1;
   const int b_stage_bytes = bn_cta * BK * 2;
-  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes;
+  const int sub_bytes = A_STAGE_BYTES + b_stage_bytes;
+  const int stage_bytes = KSUB * sub_bytes;
   uint8_t* staging = smem + (size_t)p.stages * stage_bytes;
   uint64_t* bars = (uint64_t*)(staging + NUM_EPI_WARPS * STAGING_BYTES);
   uint64_t* full_bar = bars;
@@ -236,16 +250,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
   const int tiles_per_z = p.m_tiles * p.n_tiles;
   const int per_split = tiles_per_z * p.batch;
 
-  if (warp == 0 && lane == 0 && !p.starve) {
-    // ------------------------------- TMA producer -------------------------------
-    // Ring position kept as (stage, phase) counters and tile coordinates kept in scalars: the loop
-    // body is a wait, a handful of adds and the copies, so one thread keeps the ring full.
-    uint32_t it = 0, s = 0, ph = 0;
+  if ((warp == 0 || warp == 2 || warp == 3) && lane == 0 && !p.starve) {
+    // ------------------------------- TMA producers -------------------------------
+    // Producer j takes the k blocks whose running index is j modulo NUM_PRODUCERS.  Every producer
+    // walks the whole work list (ring position as (stage, phase) counters, tile coordinates in
+    // scalars) and issues only its own blocks.
+    const uint32_t me = warp == 0 ? 0u : (uint32_t)warp - 1u;
+    uint32_t it = 0, s = 0, ph = 0, turn = 0;
+    uint32_t last_it = 0, mine = 0;
     bool ok = true;
     // which coordinate slot carries k: slot 0 for a k-contiguous operand, else the permuted one
     const int ak = p.a_mn ? p.a_perm[0] : 0, bk = p.b_mn ? p.b_perm[0] : 0;
-    const int da0 = ak == 0 ? BK : 0, da1 = ak == 1 ? BK : 0, da2 = ak == 2 ? BK : 0, da3 = ak == 3 ? BK : 0;
-    const int db0 = bk == 0 ? BK : 0, db1 = bk == 1 ? BK : 0, db2 = bk == 2 ? BK : 0, db3 = bk == 3 ? BK : 0;
+    constexpr int RK = KSUB * BK;  // k extent of a round
+    const int da0 = ak == 0 ? RK : 0, da1 = ak == 1 ? RK : 0, da2 = ak == 2 ? RK : 0, da3 = ak == 3 ? RK : 0;
+    const int db0 = bk == 0 ? RK : 0, db1 = bk == 1 ? RK : 0, db2 = bk == 2 ? RK : 0, db3 = bk == 3 ? RK : 0;
     const uint32_t smem0 = smem_u32(smem);
     const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
     const uint32_t tx_bytes = kPair ? 2 * stage_bytes : stage_bytes;
@@ -262,48 +280,62 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const int row0 = mt * mt_rows + (int)cta_rank * BM;
       const int col0 = nt * p.bn + (int)cta_rank * bn_cta;
       int ca[4], cb[4];
-      if (!p.a_mn) { ca[0] = kb0 * BK; ca[p.a_perm[0]] = row0; }
-      else         { ca[0] = row0; ca[p.a_perm[0]] = kb0 * BK; }
+      if (!p.a_mn) { ca[0] = kb0 * RK; ca[p.a_perm[0]] = row0; }
+      else         { ca[0] = row0; ca[p.a_perm[0]] = kb0 * RK; }
       ca[p.a_perm[1]] = zi; ca[p.a_perm[2]] = zo;
-      if (!p.b_mn) { cb[0] = kb0 * BK; cb[p.b_perm[0]] = col0; }
-      else         { cb[0] = col0; cb[p.b_perm[0]] = kb0 * BK; }
+      if (!p.b_mn) { cb[0] = kb0 * RK; cb[p.b_perm[0]] = col0; }
+      else         { cb[0] = col0; cb[p.b_perm[0]] = kb0 * RK; }
       cb[p.b_perm[1]] = zi; cb[p.b_perm[2]] = zo;
       int a0 = ca[0], a1 = ca[1], a2 = ca[2], a3 = ca[3];
       int b0 = cb[0], b1 = cb[1], b2 = cb[2], b3 = cb[3];
       for (int kb = kb0; kb < kb1; kb++, it++) {
-        if (!mbar_wait(empty0 + s * 8, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
-        const uint32_t fb_own = full0 + s * 8;
-        // pair mode: both CTAs' copies are counted on the leader's barrier
-        const uint32_t fb = kPair ? mapa_u32(fb_own, 0) : fb_own;
-        if (leader) mbar_expect_tx(fb_own, tx_bytes);
-        const uint32_t sa = smem0 + s * (uint32_t)stage_bytes;
-        const uint32_t sb = sa + A_STAGE_BYTES;
-        // k-contiguous operand: one box {64 k, rows}; row-contiguous: boxes {64 rows, 64 k}
-        for (int h = 0; h < a_boxes; h++) {
-          if (kPair) tma_load_4d_pair(sa + h * (64 * BK * 2), &tmA, fb, a0 + h * 64, a1, a2, a3);
-          else tma_load_4d(sa + h * (64 * BK * 2), &tmA, fb, a0 + h * 64, a1, a2, a3);
-        }
-        for (int h = 0; h < b_boxes; h++) {
-          if (kPair) tma_load_4d_pair(sb + h * (64 * BK * 2), &tmB, fb, b0 + h * 64, b1, b2, b3);
-          else tma_load_4d(sb + h * (64 * BK * 2), &tmB, fb, b0 + h * 64, b1, b2, b3);
+        if (turn == me) {
+          if (!mbar_wait(empty0 + s * 8, ph ^ 1, abort_flag, p.status)) { ok = false; break; }
+          const uint32_t fb_own = full0 + s * 8;
+          // pair mode: both CTAs' copies are counted on the leader's barrier
+          const uint32_t fb = kPair ? mapa_u32(fb_own, 0) : fb_own;
+          if (leader) mbar_expect_tx(fb_own, tx_bytes);
+          // k-contiguous operand: one box {64 k, rows} per k block; row-contiguous: boxes {64 rows,
+          // 64 k}.  A k block that starts at or beyond K is filled with zeros by the copy engine.
+#pragma unroll
+          for (int sub = 0; sub < KSUB; sub++) {
+            const uint32_t sa = smem0 + s * (uint32_t)stage_bytes + sub * (uint32_t)sub_bytes;
+            const uint32_t sb = sa + A_STAGE_BYTES;
+            const int ko = sub * BK;
+            const int x0 = a0 + (ak == 0 ? ko : 0), x1 = a1 + (ak == 1 ? ko : 0), x2 = a2 + (ak == 2 ? ko : 0),
+                      x3 = a3 + (ak == 3 ? ko : 0);
+            const int y0 = b0 + (bk == 0 ? ko : 0), y1 = b1 + (bk == 1 ? ko : 0), y2 = b2 + (bk == 2 ? ko : 0),
+                      y3 = b3 + (bk == 3 ? ko : 0);
+            for (int h = 0; h < a_boxes; h++) {
+              if (kPair) tma_load_4d_pair(sa + h * (64 * BK * 2), &tmA, fb, x0 + (p.a_mn ? h * 64 : 0), x1, x2, x3);
+              else tma_load_4d(sa + h * (64 * BK * 2), &tmA, fb, x0 + (p.a_mn ? h * 64 : 0), x1, x2, x3);
+            }
+            for (int h = 0; h < b_boxes; h++) {
+              if (kPair) tma_load_4d_pair(sb + h * (64 * BK * 2), &tmB, fb, y0 + (p.b_mn ? h * 64 : 0), y1, y2, y3);
+              else tma_load_4d(sb + h * (64 * BK * 2), &tmB, fb, y0 + (p.b_mn ? h * 64 : 0), y1, y2, y3);
+            }
+          }
+          last_it = it;
+          mine++;
         }
         a0 += da0; a1 += da1; a2 += da2; a3 += da3;
         b0 += db0; b1 += db1; b2 += db2; b3 += db3;
         if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
+        if (++turn == (uint32_t)NUM_PRODUCERS) turn = 0;
       }
     }
     if (!ok || *abort_flag) {
-      // give up: let the copies already in flight land before the CTA leaves
-      const uint32_t n = !leader ? 0u : (it < (uint32_t)p.stages ? it : (uint32_t)p.stages);
+      // give up: let this thread's copies that may still be in flight land before the CTA leaves
       if (!leader) {  // its copies are counted on the leader's barriers: give them time to land
         const long long t0 = now_cycles();
         while (now_cycles() - t0 < 2000000ll) {}
-      }
-      for (uint32_t i = 0; i < n; i++) {
-        const uint32_t j = it - 1 - i;
-        const uint32_t fb = smem_u32(&full_bar[j % p.stages]);
-        const long long t0 = now_cycles();
-        while (!mbar_try_wait(fb, (j / p.stages) & 1) && now_cycles() - t0 < 200000000ll) {}
+      } else {
+        for (uint32_t back = 0; back < mine && back * NUM_PRODUCERS < (uint32_t)p.stages; back++) {
+          const uint32_t j = last_it - back * NUM_PRODUCERS;
+          const uint32_t fb = smem_u32(&full_bar[j % p.stages]);
+          const long long t0 = now_cycles();
+          while (!mbar_try_wait(fb, (j / p.stages) & 1) && now_cycles() - t0 < 200000000ll) {}
+        }
       }
     }
   } else if (warp == 1 && lane == 0 && leader) {
@@ -320,32 +352,50 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const uint64_t b_desc0 = make_smem_desc(smem_u32(smem) + A_STAGE_BYTES, b_lbo);
     const uint32_t a_hi = (uint32_t)(a_desc0 >> 32), b_hi = (uint32_t)(b_desc0 >> 32);
     const uint32_t a_lo0 = (uint32_t)a_desc0, b_lo0 = (uint32_t)b_desc0;
-    const uint32_t stage_units = (uint32_t)stage_bytes >> 4;
+    const uint32_t stage_units = (uint32_t)stage_bytes >> 4, sub_units = (uint32_t)sub_bytes >> 4;
     const uint32_t full0 = smem_u32(&full_bar[0]), empty0 = smem_u32(&empty_bar[0]);
+    // A wait on a barrier that another thread completed costs this thread about 250 cycles even
+    // when the phase is long over, which alone would keep it from issuing a k block's four MMAs
+    // within the 512 cycles they run.  So every wait is issued one step early, before the MMAs
+    // of the current block, and its answer is only read afterwards: `ready` for the next ring
+    // slot, `acc_free` for the next work item's accumulator.
+    uint32_t ready = 0, acc_free = 0;
     for (int w = w_first; w < p.total_work && ok; w += w_step, tile++) {
       const int split = w / per_split;
       const int kb0 = split * p.kb_per_split;
       const int kb1 = min(p.kb_total, kb0 + p.kb_per_split);
       const uint32_t acc = tile & 1, use = tile >> 1;
-      if (!mbar_wait(smem_u32(&tempty_bar[acc]), (use & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      if (!acc_free && !mbar_wait(smem_u32(&tempty_bar[acc]), (use & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      acc_free = 0;
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + acc * 256;
       uint32_t accum = 0;
       for (int kb = kb0; kb < kb1; kb++) {
-        if (!mbar_wait(full0 + s * 8, ph, abort_flag, p.status)) { ok = false; break; }
+        if (!ready && !mbar_wait(full0 + s * 8, ph, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
-        const uint32_t a_lo = a_lo0 + s * stage_units, b_lo = b_lo0 + s * stage_units;
+        uint32_t s1 = s + 1, ph1 = ph;
+        if (s1 == (uint32_t)p.stages) { s1 = 0; ph1 ^= 1; }
+        ready = mbar_try_wait(full0 + s1 * 8, ph1) ? 1u : 0u;
+        if (kb == kb1 - 1 && w + w_step < p.total_work) {
+          const uint32_t nt = tile + 1;
+          acc_free = mbar_try_wait(smem_u32(&tempty_bar[nt & 1]), ((nt >> 1) & 1) ^ 1) ? 1u : 0u;
+        }
 #pragma unroll
-        for (int k = 0; k < BK / UMMA_K; k++) {
-          const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo + k * a_kstep);
-          const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo + k * b_kstep);
-          if (kPair) tc_mma_pair(d_tmem, ad, bd, p.idesc, accum);
-          else tc_mma(d_tmem, ad, bd, p.idesc, accum);
-          accum = 1;
+        for (int sub = 0; sub < KSUB; sub++) {
+          const uint32_t a_lo = a_lo0 + s * stage_units + sub * sub_units;
+          const uint32_t b_lo = b_lo0 + s * stage_units + sub * sub_units;
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; k++) {
+            const uint64_t ad = ((uint64_t)a_hi << 32) | (a_lo + k * a_kstep);
+            const uint64_t bd = ((uint64_t)b_hi << 32) | (b_lo + k * b_kstep);
+            if (kPair) tc_mma_pair(d_tmem, ad, bd, p.idesc, accum);
+            else tc_mma(d_tmem, ad, bd, p.idesc, accum);
+            accum = 1;
+          }
         }
         // the stage is free (in both CTAs) once these MMAs have read it
         if (kPair) tc_commit_pair(empty0 + s * 8); else tc_commit(empty0 + s * 8);
-        if (++s == (uint32_t)p.stages) { s = 0; ph ^= 1; }
+        s = s1; ph = ph1;
       }
       if (ok) {  // accumulator complete
         if (kPair) tc_commit_pair(smem_u32(&tfull_bar[acc])); else tc_commit(smem_u32(&tfull_bar[acc]));
@@ -357,14 +407,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       const long long t0 = now_cycles();
       while (now_cycles() - t0 < 2000000ll) {}
     }
-  } else if (warp >= 2) {
+  } else if (warp >= FIRST_EPI_WARP) {
     // ------------------------------- epilogue -------------------------------
     // Two warps share each TMEM lane quarter and take alternate 32-column chunks.  A warp reads
     // its 32 x 32 chunk (one row per lane), applies the epilogue, then turns the chunk through a
     // swizzled staging buffer so that global stores cover whole row segments.
     const int q = warp & 3;              // TMEM lane quarter this warp may read
-    const int hsel = (warp - 2) >> 2;    // which of the two warps of the quarter
-    uint8_t* stg = staging + (size_t)(warp - 2) * STAGING_BYTES;
+    const int hsel = (warp - FIRST_EPI_WARP) >> 2;    // which of the two warps of the quarter
+    uint8_t* stg = staging + (size_t)(warp - FIRST_EPI_WARP) * STAGING_BYTES;
     float* bias_s = reinterpret_cast<float*>(stg + 2048);  // bias of this warp's columns, chunk by chunk
     uint32_t tile = 0;
     bool ok = true;
@@ -618,16 +668,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 static std::atomic<int> g_starve_next{0};
 void gemm_tc_starve_next(int on) { g_starve_next.store(on ? 1 : 0); }
 
+// Measurement hook (mslt_debug_set_gemm_variant): 0 = automatic choice, 1 = one CTA per tile,
+// 2 = a CTA pair per 256 x 256 tile wherever the shape allows it.
+static std::atomic<int> g_tile_variant{0};
+void gemm_tc_set_variant(int v) { g_tile_variant.store(v); }
+
+namespace {
+// Per-device facts and one-time set-up, indexed by device ordinal (a process may drive several GPUs).
+struct DeviceInfo {
+  int num_sms = 0, smem_optin = 0;
+  bool attr_set = false;
+};
+constexpr int kMaxDevices = 64;
+DeviceInfo g_dev[kMaxDevices];
+std::mutex g_dev_mu;
+}  // namespace
+
 int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* err) {
-  static int num_sms = 0;
-  static int smem_optin = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (num_sms <= 0) { snprintf(err, 256, "gemm: no CUDA device"); return MSLT_ERR_CUDA; }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    snprintf(err, 256, "gemm: no CUDA device");
+    return MSLT_ERR_CUDA;
   }
+  DeviceInfo& di = g_dev[dev];
+  {
+    std::lock_guard<std::mutex> lock(g_dev_mu);
+    if (di.num_sms == 0) {
+      cudaDeviceGetAttribute(&di.num_sms, cudaDevAttrMultiProcessorCount, dev);
+      cudaDeviceGetAttribute(&di.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+      if (di.num_sms <= 0) { snprintf(err, 256, "gemm: no CUDA device"); return MSLT_ERR_CUDA; }
+    }
+  }
+  const int num_sms = di.num_sms, smem_optin = di.smem_optin;
   if (!status) { snprintf(err, 256, "gemm: the tensor-core kernel needs a device status word"); return MSLT_ERR_ARG; }
   TcParams p;
   memset(&p, 0, sizeof(p));
@@ -636,14 +708,10 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   p.b_mn = (d.b_rs == 1 && d.b_ks != 1) ? 1 : 0;
   p.bn = d.N <= 64 ? 64 : (d.N <= 128 ? 128 : 256);
   // Two CTAs per 256 x 256 tile: each SM then streams 64 instead of 96 bytes of operands per clock
-  // from L2 and has six instead of four stages in flight.  MSLT_GEMM_SINGLE_CTA=1 keeps one CTA per
-  // tile (for A/B measurements).
-  static const bool single_cta = getenv("MSLT_GEMM_SINGLE_CTA") && atoi(getenv("MSLT_GEMM_SINGLE_CTA")) == 1;
-  // Measured: the pair wins for row-contiguous (MN-major) operands and for deep contractions, and is
-  // on par or slightly behind for shallow k-contiguous products, which are bound by their epilogue.
-  static const bool force_pair = getenv("MSLT_GEMM_SINGLE_CTA") && atoi(getenv("MSLT_GEMM_SINGLE_CTA")) == 2;
-  bool pair = !single_cta && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0 &&
-              (force_pair || p.a_mn || p.b_mn || d.K >= 2048);
+  // from L2 (about 117 is what an SM was measured to take) and has six instead of four stages in
+  // flight.
+  const int variant = g_tile_variant.load();
+  bool pair = variant != 1 && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0;
   // share of the SMs that the last wave of tiles keeps busy
   auto wave_eff = [](long long work, int units_) {
     const long long waves = (work + units_ - 1) / units_;
@@ -663,15 +731,16 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   const int tile_m = pair ? 2 * BM : BM;
   p.m_tiles = (d.M + tile_m - 1) / tile_m;
   p.n_tiles = (d.N + p.bn - 1) / p.bn;
-  p.kb_total = (d.K + BK - 1) / BK;
+  const int round_k = pair ? 2 * BK : BK;  // k extent of a ring stage (see KSUB in the kernel)
+  p.kb_total = (d.K + round_k - 1) / round_k;
   const long long tiles = (long long)p.m_tiles * p.n_tiles * d.batch;
   const int units = pair ? num_sms / 2 : num_sms;  // CTAs or CTA pairs that run concurrently
   int splits = 1;
   if (d.split_k > 1) {
     splits = d.split_k;
-  } else if (d.split_k == 0 && can_split && tiles < 2 * units && p.kb_total >= 8) {
-    // the split count that fills the last wave best, with at least four k blocks per split
-    const int max_by_k = p.kb_total / 4;
+  } else if (d.split_k == 0 && can_split && tiles < 2 * units && p.kb_total * round_k >= 8 * BK) {
+    // the split count that fills the last wave best, with at least 256 k per split
+    const int max_by_k = p.kb_total * round_k / (4 * BK);
     double best = wave_eff(tiles, units);
     for (int sp = 2; sp <= 16 && sp <= max_by_k; sp++) {
       const double e = wave_eff(tiles * sp, units);
@@ -692,12 +761,10 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
     snprintf(err, 256, "gemm: the softmax epilogue needs bf16 output rows of at most 128 columns");
     return MSLT_ERR_ARG;
   }
-  const int stage_bytes = A_STAGE_BYTES + (pair ? p.bn / 2 : p.bn) * BK * 2;  // per CTA
+  const int stage_bytes = (pair ? 2 : 1) * (A_STAGE_BYTES + (pair ? p.bn / 2 : p.bn) * BK * 2);  // per CTA
   const int book_bytes = 256 + (d.act == 3 ? 64 + 2 * NUM_EPI_WARPS * 32 * 4 : 0);
   int stages = (smem_optin - NUM_EPI_WARPS * STAGING_BYTES - 1024 - book_bytes) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
-  static const int stage_cap = getenv("MSLT_GEMM_STAGES") ? atoi(getenv("MSLT_GEMM_STAGES")) : 0;
-  if (stage_cap >= 2 && stages > stage_cap) stages = stage_cap;
   if (stages < 2) { snprintf(err, 256, "gemm: not enough shared memory"); return MSLT_ERR_CUDA; }
   p.stages = stages;
   const size_t smem_bytes = (size_t)stages * stage_bytes + NUM_EPI_WARPS * STAGING_BYTES + 1024 + book_bytes;
@@ -739,8 +806,6 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   else if (d.act == 0 && d.residual && x_ok) mode = EPI_RESIDUAL;
   else if (d.act == 1 && !d.residual) mode = d.aux ? EPI_GELU_AUX : EPI_GELU;
   else if (d.act == 2 && d.aux && !d.residual && x_ok) mode = EPI_DGELU;
-  static const bool generic_only = getenv("MSLT_GEMM_GENERIC_EPILOGUE") && atoi(getenv("MSLT_GEMM_GENERIC_EPILOGUE")) == 1;
-  if (generic_only && mode != EPI_SOFTMAX) mode = EPI_GENERIC;
 
   typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const TcParams);
   static const KernelFn kernels[EPI_COUNT][2] = {
@@ -752,20 +817,21 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
       {gemm_tc_kernel<EPI_F32, false>, gemm_tc_kernel<EPI_F32, true>},
       {gemm_tc_kernel<EPI_GENERIC, false>, gemm_tc_kernel<EPI_GENERIC, true>},
       {gemm_tc_kernel<EPI_SOFTMAX, false>, nullptr}};
-  static bool attr_set = false;
-  if (!attr_set) {
+  std::unique_lock<std::mutex> dev_lock(g_dev_mu);
+  if (!di.attr_set) {
     for (int mo = 0; mo < EPI_COUNT; mo++)
       for (int pr = 0; pr < 2; pr++) {
         if (!kernels[mo][pr]) continue;
         cudaError_t e = cudaFuncSetAttribute((const void*)kernels[mo][pr], cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
         if (e != cudaSuccess) { snprintf(err, 256, "gemm: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
       }
-    attr_set = true;
+    di.attr_set = true;
   }
+  dev_lock.unlock();
   const KernelFn fn = kernels[mode][pair ? 1 : 0];
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
-  cfg.blockDim = dim3(NUM_THREADS);
+  cfg.blockDim = dim3(GEMM_THREADS);
   cfg.dynamicSmemBytes = smem_bytes;
   cfg.stream = st;
   cudaLaunchAttribute attr[1];

@@ -1019,6 +1019,12 @@ int mslt_debug_starve_next_gemm(int32_t on) {
   return 0;
 }
 
+int mslt_debug_set_gemm_variant(int32_t variant) {
+  if (variant < 0 || variant > 2) return fail(MSLT_ERR_ARG, "variant must be 0, 1 or 2");
+  gemm_tc_set_variant(variant);
+  return 0;
+}
+
 static int check_gemm_desc(const mslt_gemm_desc* d) {
   if (!d || !d->A || !d->B || !d->D) return fail(MSLT_ERR_ARG, "null pointer");
   if (d->M < 1 || d->N < 1 || d->K < 1 || d->batch < 1 || d->hdiv < 1)

@@ -11,8 +11,20 @@ from paper_2011_13635_b200 import inputs as I
 #   fp32 path: every contraction accumulates in fp32 in k order, statistics in fp32.
 #   bf16 path: activations, saved activations and activation gradients are rounded to bf16
 #   (relative 2^-9 per rounding); weight gradients accumulate in fp32.
-TOL = {"fp32": dict(loss=2e-3, grad=1e-4, weight=1e-4, hidden=1e-4, update_l1=2e-3),
-       "bf16": dict(loss=2e-3, grad=3e-2, weight=3e-2, hidden=3e-2, update_l1=0.15)}
+#   update: the change dw = w_after - w_before of one step, in two forms.  update_l1 is
+#   mean|dw - dw_ref| / mean|dw_ref| over the whole tensor.  update_max is the max-abs form
+#   max|dw - dw_ref| / max|dw_ref|; Adam's first step is -lr * g / (|g| + eps), i.e. sign-like, so
+#   an element whose gradient lies within the gradient tolerance of zero may legitimately take the
+#   opposite sign (an error of 2 in that form).  The max-abs form is therefore asserted on the
+#   elements whose reference gradient is clear of zero by twice the gradient tolerance
+#   (|g_ref| > 2 * tol_grad * G with G = max|g_ref|, where both sides must agree on the sign) and
+#   reported (not asserted) over all elements.  Its tolerance follows from the gradient tolerance:
+#   h(g) = g / (|g| + eps) has slope eps / (|g| + eps)^2, a gradient error of at most tol_grad * G
+#   is at most half of such an element, so its first-step update is off by at most
+#   lr * eps * tol_grad * G / (|g_ref| / 2 + eps)^2 (never more than lr / 4), plus update_max for
+#   the rounding of the arithmetic itself.
+TOL = {"fp32": dict(loss=2e-3, grad=1e-4, weight=1e-4, hidden=1e-4, update_l1=2e-3, update_max=1e-4),
+       "bf16": dict(loss=2e-3, grad=3e-2, weight=3e-2, hidden=3e-2, update_l1=0.15, update_max=1e-3)}
 
 
 def max_rel(a: np.ndarray, r: np.ndarray) -> float:
@@ -77,7 +89,8 @@ def compare_step(m, oracle, cfg, batch, tol, report=None):
     rel_loss = abs(loss_g - loss_o) / abs(loss_o)
     assert rel_loss < tol["loss"], (loss_g, loss_o)
 
-    worst = dict(grad=("", 0.0), weight=("", 0.0), update=("", 0.0))
+    worst = dict(grad=("", 0.0), weight=("", 0.0), update=("", 0.0), update_max_clear=("", 0.0),
+                 update_max_all=("", 0.0))
     o = oracle.opt
     t = oracle.t
     for n in names:
@@ -98,6 +111,22 @@ def compare_step(m, oracle, cfg, batch, tol, report=None):
         if e > worst["update"][1]:
             worst["update"] = (n, e)
         assert e < tol["update_l1"], ("update", n, e)
+        # max-abs form of the update: over all elements (a number for the report) and, asserted,
+        # over the elements whose reference gradient is clear of zero
+        den = max(np.abs(dwo).max(), 1e-30)
+        e_all = float(np.abs(dw - dwo).max() / den)
+        if e_all > worst["update_max_all"][1]:
+            worst["update_max_all"] = (n, e_all)
+        g_ref = oracle.grads[n]
+        clear = np.abs(g_ref) > 2.0 * tol["grad"] * np.abs(g_ref).max()
+        if t == 1 and clear.any() and o["bias_correction"]:
+            e = float(np.abs(dw - dwo)[clear].max() / den)
+            if e > worst["update_max_clear"][1]:
+                worst["update_max_clear"] = (n, e)
+            gc = np.abs(g_ref[clear])
+            allow = o["lr"] * (o["eps"] * tol["grad"] * np.abs(g_ref).max() / (gc / 2 + o["eps"]) ** 2).max() / den
+            assert e < allow + tol["update_max"], ("update, max-abs form on clear gradients", n, e, allow)
+            assert np.abs(dw[clear]).min() > 0.0, ("an element with a clear gradient did not move", n)
         # the Adam kernel alone: the oracle's update formula applied to the library's own inputs
         wd = o["weight_decay"] if w_before[n].ndim == 2 else 0.0
         w_ref, m_ref, v_ref = O.adam_update(w_before[n].astype(np.float64), g.astype(np.float64),

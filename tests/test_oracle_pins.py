@@ -287,6 +287,75 @@ def test_step_applies_decay_to_matrices_only():
         np.testing.assert_allclose(m2.p[n], want, atol=1e-14)
 
 
+def _first_step_form(m, g, w0, lr, eps):
+    """With bias correction and no decay the first Adam step moves every weight by
+    -lr * g / (|g| + eps): m_hat = g and v_hat = g^2 whatever the betas are.  It holds only while
+    the counter that enters the bias correction reads 1, so it pins the counter itself."""
+    for n in m.trainable_names():
+        np.testing.assert_allclose(m.p[n] - w0[n], -lr * g[n] / (np.abs(g[n]) + eps), atol=1e-13, err_msg=n)
+
+
+def test_step_counter_starts_at_one_and_restarts_with_every_stage_change():
+    lr, eps = 1e-2, 1e-6
+    cfg = I.scaled(TINY, layers=2)
+    w = I.make_weights(cfg, seed=5, variant="parity", std=0.3)
+    m = O.MsltOracle(w, cfg.heads, max_layers=4)
+    m.set_optimizer(lr=lr, eps=eps, weight_decay=0.0, beta1=0.9, beta2=0.999, bias_correction=1)
+    tok, lens, pos, lab = tiny_batch()
+
+    def one_step():
+        w0 = {k: v.copy() for k, v in m.p.items()}
+        _, g = m.loss_and_grads(tok, lens, pos, lab)
+        g = {k: v.copy() for k, v in g.items()}
+        m.step(tok, lens, pos, lab)
+        return w0, g
+
+    m.set_trainable(1)
+    w0, g = one_step()
+    _first_step_form(m, g, w0, lr, eps)             # a counter that started at 0 or 2 fails here
+    # the second step is not of that form (m and v now carry history) ...
+    w0, g = one_step()
+    moved = np.concatenate([(m.p[n] - w0[n]).ravel() for n in m.trainable_names()])
+    first = np.concatenate([(-lr * g[n] / (np.abs(g[n]) + eps)).ravel() for n in m.trainable_names()])
+    assert np.abs(moved - first).max() > 1e-4
+    assert m.t == 2
+    # changing the trainable slice clears the moments and the counter: first-step form again,
+    # also for tensors that were trainable (and had history) before
+    m.set_trainable(2)
+    assert m.t == 0
+    w0, g = one_step()
+    _first_step_form(m, g, w0, lr, eps)
+    # so does stacking (the new layers and the head both restart)
+    one_step()
+    m.add_layers(2)
+    assert m.t == 0 and m.top_k == 2
+    w0, g = one_step()
+    _first_step_form(m, g, w0, lr, eps)
+    # without the restart the same call would not have the first-step form: plant the mistake
+    m.t = 3
+    w0, g = one_step()
+    with pytest.raises(AssertionError):
+        _first_step_form(m, g, w0, lr, eps)
+
+
+def test_second_step_bias_correction_closed_form():
+    # constant gradient through step(): with g fixed, m_hat = g and v_hat = g^2 at every t, so each of
+    # the first steps moves head.decoder.bias by the same -lr * g / (|g| + eps) only if t counts 1, 2, ...
+    lr, eps = 1e-3, 1e-6
+    m = tiny_model(top_k=0)
+    m.set_optimizer(lr=lr, eps=eps, weight_decay=0.0, bias_correction=1)
+    g = np.linspace(-1.0, 1.0, m.p["head.decoder.bias"].size)
+    g[np.abs(g) < 1e-3] = 0.5
+    m.loss_and_grads = lambda *a: (0.0, {n: (g.copy() if n == "head.decoder.bias" else np.zeros_like(m.p[n]))
+                                         for n in m.trainable_names()})
+    tok, lens, pos, lab = tiny_batch()
+    for t in (1, 2, 3):
+        w0 = m.p["head.decoder.bias"].copy()
+        m.step(tok, lens, pos, lab)
+        assert m.t == t
+        np.testing.assert_allclose(m.p["head.decoder.bias"] - w0, -lr * g / (np.abs(g) + eps), atol=1e-15)
+
+
 # -- staging ------------------------------------------------------------------------------------------------
 
 def test_truncated_gradients_equal_full_gradients_on_the_trainable_slice():
