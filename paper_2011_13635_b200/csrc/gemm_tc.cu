@@ -49,6 +49,7 @@ struct TcParams {
   char* D;
   long long ldd, d_bo, d_bi;
   int d_fp32, accumulate, vec_ok;
+  int direct;           // rows of D (and aux) may be stored straight from registers, 32 bytes at a time
   float alpha;
   const float* bias;
   int act;
@@ -121,13 +122,50 @@ enum : int {
   EPI_COUNT
 };
 
+// A lane that owns a row stores 32 of its columns without a trip through shared memory: two
+// 32-byte stores for bf16 (every store fills a whole sector), four for fp32, or eight 16-byte
+// vector reductions when partial sums are added.  dst must be 32-byte aligned.
+__device__ __forceinline__ void row32_store_bf16(bf16* dst, const float2 (&w)[16]) {
+  uint32_t h[16];
+#pragma unroll
+  for (int e = 0; e < 16; e++) {
+    const __nv_bfloat162 t = __float22bfloat162_rn(w[e]);
+    h[e] = *reinterpret_cast<const uint32_t*>(&t);
+  }
+#pragma unroll
+  for (int c = 0; c < 2; c++)
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 16 * c), "r"(h[8 * c]),
+                 "r"(h[8 * c + 1]), "r"(h[8 * c + 2]), "r"(h[8 * c + 3]), "r"(h[8 * c + 4]), "r"(h[8 * c + 5]),
+                 "r"(h[8 * c + 6]), "r"(h[8 * c + 7])
+                 : "memory");
+}
+__device__ __forceinline__ void row32_store_f32(float* dst, const float2 (&w)[16], int accumulate) {
+  if (accumulate) {
+#pragma unroll
+    for (int c = 0; c < 8; c++)
+      asm volatile("red.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(dst + 4 * c), "f"(w[2 * c].x), "f"(w[2 * c].y),
+                   "f"(w[2 * c + 1].x), "f"(w[2 * c + 1].y)
+                   : "memory");
+  } else {
+#pragma unroll
+    for (int c = 0; c < 4; c++)
+      asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(dst + 8 * c), "f"(w[4 * c].x),
+                   "f"(w[4 * c].y), "f"(w[4 * c + 1].x), "f"(w[4 * c + 1].y), "f"(w[4 * c + 2].x), "f"(w[4 * c + 2].y),
+                   "f"(w[4 * c + 3].x), "f"(w[4 * c + 3].y)
+                   : "memory");
+  }
+}
+
 // One 32 x 32 chunk of a specialised flavour: a = this lane's 32 accumulator columns, bias_c = the
 // chunk's bias values in shared memory (zeros without a bias), x = this lane's 32 bf16 values of
 // the row-shaped extra operand (EPI_RESIDUAL, EPI_DGELU).
+// `direct`: this lane's row exists and the whole chunk lies inside the output, so the lane stores
+// its 32 columns itself; otherwise the chunk goes through the staging buffer, which handles ragged
+// edges element by element (every lane of the warp takes the same branch).
 template <int kMode>
 __device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)[32], const uint4 (&x)[4],
                                           const float* bias_c, uint8_t* stg, int lane, long long zoff,
-                                          int m_warp, int n0) {
+                                          int m_warp, int n0, bool direct) {
   float2 v[16];
   const float2 al = splat2(p.alpha);
   const float4* b4 = reinterpret_cast<const float4*>(bias_c);
@@ -139,8 +177,12 @@ __device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)
     v[2 * j + 1] = __ffma2_rn(make_float2(__uint_as_float(a[4 * j + 2]), __uint_as_float(a[4 * j + 3])), al,
                               make_float2(t.z, t.w));
   }
-  if constexpr (kMode == EPI_GELU_AUX)
-    stage_store_bf16(stg, lane, v, p.aux + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
+  const bool row_ok = m_warp + lane < p.M;
+  const long long off = zoff + (long long)(m_warp + lane) * p.ldd + n0;
+  if constexpr (kMode == EPI_GELU_AUX) {
+    if (direct) { if (row_ok) row32_store_bf16(p.aux + off, v); }
+    else stage_store_bf16(stg, lane, v, p.aux + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
+  }
   if constexpr (kMode == EPI_GELU || kMode == EPI_GELU_AUX) {
 #pragma unroll
     for (int j = 0; j < 16; j++) v[j] = gelu_fast2(v[j]);
@@ -163,11 +205,14 @@ __device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)
       v[4 * j + 3] = __fadd2_rn(v[4 * j + 3], bf162_to_f2(x[j].w));
     }
   }
-  if constexpr (kMode == EPI_F32)
-    stage_store_f32(stg, lane, v, reinterpret_cast<float*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok,
-                    p.accumulate);
-  else
-    stage_store_bf16(stg, lane, v, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
+  if constexpr (kMode == EPI_F32) {
+    if (direct) { if (row_ok) row32_store_f32(reinterpret_cast<float*>(p.D) + off, v, p.accumulate); }
+    else stage_store_f32(stg, lane, v, reinterpret_cast<float*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok,
+                         p.accumulate);
+  } else {
+    if (direct) { if (row_ok) row32_store_bf16(reinterpret_cast<bf16*>(p.D) + off, v); }
+    else stage_store_bf16(stg, lane, v, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
+  }
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------
@@ -418,6 +463,141 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     float* bias_s = reinterpret_cast<float*>(stg + 2048);  // bias of this warp's columns, chunk by chunk
     uint32_t tile = 0;
     bool ok = true;
+    if constexpr (kMode != EPI_GENERIC && !kSoftmax) {
+      // The specialised flavours.  What keeps a tile's epilogue short enough to hide behind the
+      // next tile's main loop: the work-item coordinates advance by mixed-radix addition (no
+      // division per tile); the bias of the NEXT tile is fetched while this tile is worked on; the
+      // TMEM read of the next chunk is in flight while the current chunk is converted and stored;
+      // and a lane stores its row segment straight from registers.
+      const int nch = p.bn >> 6;
+      constexpr bool kHasXf = kMode == EPI_RESIDUAL || kMode == EPI_DGELU;
+      const bf16* xsrc = kMode == EPI_DGELU ? p.aux : kMode == EPI_RESIDUAL ? p.residual : nullptr;
+      // digits of the work index (n tile fastest, then m tile, batch, split) and of the step
+      int nt, mt, z, sp, d_nt, d_mt, d_z, d_sp;
+      {
+        int r = w_first;
+        sp = r / per_split; r -= sp * per_split;
+        z = r / tiles_per_z; r -= z * tiles_per_z;
+        mt = r / p.n_tiles; nt = r - mt * p.n_tiles;
+        r = w_step;
+        d_sp = r / per_split; r -= d_sp * per_split;
+        d_z = r / tiles_per_z; r -= d_z * tiles_per_z;
+        d_mt = r / p.n_tiles; d_nt = r - d_mt * p.n_tiles;
+      }
+      auto advance = [&](int& nt_, int& mt_, int& z_, int& sp_) {
+        nt_ += d_nt;
+        int c = nt_ >= p.n_tiles ? 1 : 0;
+        nt_ -= c ? p.n_tiles : 0;
+        mt_ += d_mt + c;
+        c = mt_ >= p.m_tiles ? 1 : 0;
+        mt_ -= c ? p.m_tiles : 0;
+        z_ += d_z + c;
+        c = z_ >= p.batch ? 1 : 0;
+        z_ -= c ? p.batch : 0;
+        sp_ += d_sp + c;
+      };
+      // bias values of this warp's columns of tile `nt_`, one value per lane and chunk
+      auto fetch_bias = [&](int nt_, float (&b)[4]) {
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+          const int n = nt_ * p.bn + (hsel + 2 * i) * 32 + lane;
+          b[i] = (i < nch && p.bias && n < p.N) ? p.bias[n] : 0.f;
+        }
+      };
+      float bnext[4];
+      if (w_first < p.total_work) {
+        fetch_bias(nt, bnext);
+#pragma unroll
+        for (int i = 0; i < 4; i++) bias_s[i * 32 + lane] = bnext[i];
+        __syncwarp();
+      }
+      for (int w = w_first; w < p.total_work && ok; w += w_step, tile++) {
+        const int zo = p.hdiv == 1 ? z : z / p.hdiv, zi = p.hdiv == 1 ? 0 : z - zo * p.hdiv;
+        const uint32_t acc = tile & 1, use = tile >> 1;
+        const int m_warp = mt * mt_rows + (int)cta_rank * BM + q * 32;  // first row of this warp
+        const int m = m_warp + lane;
+        const bool row_ok = m < p.M;
+        const long long zoff = zo * p.d_bo + zi * p.d_bi;
+        const long long off0 = zoff + (long long)m * p.ldd;
+        const int n_base = nt * p.bn;
+        const float* bias_t = bias_s + (tile & 1) * 128;
+        const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
+        auto chunk_n0 = [&](int i) { return n_base + (hsel + 2 * i) * 32; };
+        auto chunk_ok = [&](int i) { return i < nch && chunk_n0(i) < p.N; };
+        auto prefetch_x = [&](int i, uint4 (&x)[4]) {
+          if (kHasXf && row_ok) {
+            const uint4* src = reinterpret_cast<const uint4*>(xsrc + off0 + chunk_n0(i));
+#pragma unroll
+            for (int j = 0; j < 4; j++) x[j] = src[j];
+          }
+        };
+        // the next work item and its bias (the loads travel while this tile is worked on)
+        int nt2 = nt, mt2 = mt, z2 = z, sp2 = sp;
+        advance(nt2, mt2, z2, sp2);
+        const bool more = w + w_step < p.total_work;
+        if (more) fetch_bias(nt2, bnext);
+        uint4 x[4];
+        const bool c0ok = chunk_ok(0);
+        if (c0ok) prefetch_x(0, x);
+        if (!mbar_wait(smem_u32(&tfull_bar[acc]), use & 1, abort_flag, p.status)) { ok = false; break; }
+        tc_fence_after();
+        auto release_acc = [&]() {  // every TMEM read of this tile has returned
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) {
+            if (kPair && !leader) mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[acc]), 0));
+            else mbar_arrive(smem_u32(&tempty_bar[acc]));
+          }
+        };
+        auto work = [&](const uint32_t (&a)[32], int i, bool has_next) {
+          uint4 xc[4];
+          if constexpr (kHasXf) {
+#pragma unroll
+            for (int j = 0; j < 4; j++) xc[j] = x[j];
+            if (has_next) prefetch_x(i + 1, x);
+          }
+          const int n0 = chunk_n0(i);
+          epi_chunk<kMode>(p, a, xc, bias_t + i * 32, stg, lane, zoff, m_warp, n0, p.direct && n0 + 32 <= p.N);  // warp-uniform
+        };
+        if (c0ok && kHasXf) {
+          // the flavours with a row-shaped extra operand have no registers to spare for a second
+          // chunk in flight
+          uint32_t ra[32];
+          for (int i = 0;; i++) {
+            const bool v1 = chunk_ok(i + 1);
+            tc_ld32_issue(trow + (hsel + 2 * i) * 32, ra);
+            tc_ld32_wait(ra);
+            if (!v1) release_acc();
+            work(ra, i, v1);
+            if (!v1) break;
+          }
+        } else if (c0ok) {
+          uint32_t ra[32], rb[32];
+          tc_ld32_issue(trow + hsel * 32, ra);
+          for (int i = 0;; i += 2) {
+            const bool v1 = chunk_ok(i + 1);
+            tc_ld32_wait(ra);
+            if (v1) tc_ld32_issue(trow + (hsel + 2 * (i + 1)) * 32, rb); else release_acc();
+            work(ra, i, v1);
+            if (!v1) break;
+            const bool v2 = chunk_ok(i + 2);
+            tc_ld32_wait(rb);
+            if (v2) tc_ld32_issue(trow + (hsel + 2 * (i + 2)) * 32, ra); else release_acc();
+            work(rb, i + 1, v2);
+            if (!v2) break;
+          }
+        } else {
+          release_acc();
+        }
+        if (more) {
+          float* bias_n = bias_s + ((tile + 1) & 1) * 128;
+#pragma unroll
+          for (int i = 0; i < 4; i++) bias_n[i * 32 + lane] = bnext[i];
+          __syncwarp();
+        }
+        nt = nt2; mt = mt2; z = z2; sp = sp2;
+      }
+    } else
     for (int w = w_first; w < p.total_work && ok; w += w_step, tile++) {
       const int split = w / per_split;
       int r = w - split * per_split;
@@ -546,7 +726,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             // the extra operand of the next chunk travels while this chunk is worked on
             if (has_next) prefetch_x(i + 1, x);
           }
-          epi_chunk<kMode>(p, a, xc, bias_s + i * 32, stg, lane, zoff, m_warp, n0);
+          epi_chunk<kMode>(p, a, xc, bias_s + i * 32, stg, lane, zoff, m_warp, n0, false);
           return;
         }
         const long long off = off0 + n0;
@@ -711,7 +891,10 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   // from L2 (about 117 is what an SM was measured to take) and has six instead of four stages in
   // flight.
   const int variant = g_tile_variant.load();
-  bool pair = variant != 1 && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0;
+  // Small products (under ~30 GFLOP, e.g. 16384 x 768 x 768) measured 5-10 % faster on single CTAs.
+  const double flops = 2.0 * d.M * d.N * (double)d.K * d.batch;
+  bool pair = variant != 1 && p.bn == 256 && d.M > BM && d.act != 3 && num_sms % 2 == 0 &&
+              (variant == 2 || flops >= 30e9);
   // share of the SMs that the last wave of tiles keeps busy
   auto wave_eff = [](long long work, int units_) {
     const long long waves = (work + units_ - 1) / units_;
@@ -793,6 +976,13 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   auto al16 = [](const void* q) { return ((uintptr_t)q & 15) == 0; };
   p.vec_ok = (d.ldd % 8 == 0 && d.d_bo % 8 == 0 && d.d_bi % 8 == 0 && al16(d.D) && al16(d.aux) &&
               al16(d.residual) && al16(d.bias)) ? 1 : 0;
+  // straight-from-register row stores write 32 bytes at a time
+  auto al32 = [](const void* q) { return ((uintptr_t)q & 31) == 0; };
+  const long long esz = d.d_fp32 ? 4 : 2;
+  p.direct = (p.vec_ok && al32(d.D) && (d.ldd * esz) % 32 == 0 && (d.d_bo * esz) % 32 == 0 && (d.d_bi * esz) % 32 == 0 &&
+              !(d.d_fp32 && d.accumulate) &&  // vector reductions do better as whole row segments
+              (!d.aux || d.act != 1 || (al32(d.aux) && (d.ldd * 2) % 32 == 0 && (d.d_bo * 2) % 32 == 0 && (d.d_bi * 2) % 32 == 0)))
+                 ? 1 : 0;
   // instruction descriptor: fp32 accumulate, bf16 x bf16, operand majors, N and M of the tile
   p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)p.a_mn << 15) | ((uint32_t)p.b_mn << 16) |
             ((uint32_t)(p.bn >> 3) << 17) | ((uint32_t)(tile_m >> 4) << 24);
