@@ -170,7 +170,7 @@ def run_reference(args, cfg):
 # ------------------------------------------------------------------------------------------------
 def make_model(cfg, torch, stream=None):
     from paper_2011_13635_b200.binding import Mslt
-    m = Mslt.from_config(cfg, stream=stream)
+    m = Mslt.from_config(cfg, stream=stream, max_trainable=cfg.trainable)
     m.set_params(I.make_weights(cfg, variant="bench"))
     m.mslt_set_trainable(cfg.trainable)
     m.mslt_set_optimizer(**I.ADAM_DEFAULTS)

@@ -61,6 +61,10 @@ typedef struct {
   int32_t dtype;       /* 0: fp32 everywhere; 1: bf16 weights/activations, fp32 master */
                        /*    weights, gradients and Adam state                         */
   float ln_eps;        /* LayerNorm epsilon (BERT: 1e-12)                              */
+  int32_t max_trainable; /* most top layers that will ever be trainable at once; 0 = max_layers.  Only */
+                       /* trainable layers keep their activations for the backward pass (Section    */
+                       /* 3.2: the bottom layers run forward only), so the workspace holds this many  */
+                       /* saved-activation slots: BERT-Base 9 + 3 needs 3 of them, not 12             */
 } mslt_arch;
 
 /* Adam with decoupled weight decay (decay on matrices and tables only). */
@@ -69,12 +73,19 @@ typedef struct {
   int32_t bias_correction; /* 1: divide m, v by (1 - beta^t)                           */
 } mslt_opt;
 
-/* Bytes of device memory the caller must provide for this architecture. */
+/*
+ * Bytes of device memory the caller must provide for this architecture: the parameter block
+ * (master weights, gradients, optimizer state and bf16 copies of every layer up to max_layers: the
+ * stack grows in place when layers are added, Section 3.2) and the workspace (two activation
+ * buffers for the forward-only bottom layers, saved activations for max_trainable top layers, the
+ * output layer's buffers).
+ */
 int mslt_query_bytes(const mslt_arch* arch, size_t* param_bytes, size_t* workspace_bytes);
 
 /*
  * Creates a context with init_layers encoder layers, all trainable (in the first
- * stage every parameter is trained, Section 3.2).  dev_params / dev_workspace:
+ * stage every parameter is trained, Section 3.2); if max_trainable is smaller than
+ * init_layers, the top max_trainable layers are trainable instead.  dev_params / dev_workspace:
  * device, at least the queried sizes, 256-byte aligned; the library zeroes
  * both.  Parameters are left at zero: set them with mslt_set_param.
  * cuda_stream: a cudaStream_t (NULL = the default stream).  *out: host.
@@ -98,12 +109,16 @@ int mslt_add_layers(mslt_ctx* ctx, int32_t k);
  * Moves the frozen/trainable boundary (Section 3.2): layers [L-top_k, L) and
  * the output layer (MLM transform, its LayerNorm, decoder bias) are trained;
  * top_k == L also trains the embeddings (word table shared with the decoder,
- * position table, embedding LayerNorm).  0 <= top_k <= L.  Zeroes the
- * optimizer state.
+ * position table, embedding LayerNorm).  0 <= top_k <= L (MSLT_ERR_STATE otherwise) and
+ * top_k <= max_trainable (MSLT_ERR_SIZE otherwise).  Zeroes the optimizer state.
  */
 int mslt_set_trainable(mslt_ctx* ctx, int32_t top_k);
 
-/* Hyper-parameters used from the next step on (learning-rate schedules are the caller's). */
+/*
+ * Hyper-parameters used from the next step on.  The paper trains with a warm-up of the learning
+ * rate over the first 10 000 steps of a stage and a smaller rate in the final joint retraining
+ * (Sections 4.2, 5.2): such schedules are the caller's, who sets the rate before each step.
+ */
 int mslt_set_optimizer(mslt_ctx* ctx, const mslt_opt* opt);
 
 /*
@@ -132,7 +147,9 @@ int mslt_step(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens,
 int mslt_read_loss(mslt_ctx* ctx, float* loss_out);
 
 /*
- * Forward only, nothing saved at any layer, no update.
+ * Forward only, nothing saved at any layer, no update: the pass that the bottom layers of a stage
+ * take part in (Section 3.2, "only participate in forward computation"), here through the whole
+ * stack and optionally through the output layer, e.g. for evaluation between stages.
  *   d_hidden_out  device [B,S,H] in the compute dtype (float or bf16), or NULL
  *   d_mlm_positions device [B,P] or NULL; d_logits_out device [B*P, vocab] fp32 or NULL
  *   (rows of empty slots are computed from a zero feature row).
@@ -231,6 +248,13 @@ int mslt_debug_starve_next_gemm(int32_t on);
 /* The same hook for the fused attention kernels: the NEXT mslt_op_attention / mslt_op_attention_bwd
  * call (or attention launch inside a step) runs with an idle producer and a 20 ms wait limit. */
 int mslt_debug_starve_next_attention(int32_t on);
+
+/*
+ * Environment switches read once per process, for debugging and A/B measurements only (they
+ * change speed, not results beyond rounding): MSLT_BF16_CUDA_CORES=1 sends dtype-1 contractions
+ * to the plain CUDA-core kernel; MSLT_UNFUSED_ATTENTION=1 runs attention as batched contractions
+ * with a separate softmax instead of the fused kernels.
+ */
 
 /*
  * Measurement hook: how the dtype-1 contraction kernel tiles its output from now on, process
@@ -333,7 +357,9 @@ int mslt_op_attention_bwd(const void* d_qkv, const void* d_probs, const void* d_
  *
  * The call itself, and everything under it, calls no cudaMalloc, cudaFree or allocating library
  * routine.  The first call on each device looks up the array's device address (the device must be
- * current, as for any call here); make that first call outside any stream capture.
+ * current, as for any call here) and may make the driver load the library's image onto that
+ * device; make that first call outside any stream capture.  Later calls take no device memory at
+ * all.
  * All calls on one GPU share the one array, which keeps whatever the last call left in it; each
  * call overwrites what it reads, so nothing needs clearing, but two calls that overlap in time on
  * the same GPU (different streams or threads) race on it and give undefined results: serialise

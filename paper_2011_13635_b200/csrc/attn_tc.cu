@@ -1014,16 +1014,49 @@ static std::atomic<int> g_attn_starve{0};
 void attn_starve_next(int on) { g_attn_starve.store(on ? 1 : 0); }
 long long attn_launches() { return g_attn_launches.load(); }
 
+namespace {
+// per-device facts and one-time kernel attributes (a process may drive several GPUs)
+struct AttnDevice {
+  int num_sms = 0, smem_optin = 0;
+  bool attr_fwd = false, attr_long = false, attr_bwd = false;
+};
+constexpr int kMaxDevices = 64;
+AttnDevice g_adev[kMaxDevices];
+std::mutex g_adev_mu;
+AttnDevice* attn_device(char* err) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
+    snprintf(err, 256, "attention: no CUDA device");
+    return nullptr;
+  }
+  std::lock_guard<std::mutex> lock(g_adev_mu);
+  AttnDevice& a = g_adev[dev];
+  if (a.num_sms == 0) {
+    cudaDeviceGetAttribute(&a.num_sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaDeviceGetAttribute(&a.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    if (a.num_sms <= 0) { snprintf(err, 256, "attention: no CUDA device"); return nullptr; }
+  }
+  return &a;
+}
+// opts a kernel in to the large dynamic shared memory size once per device
+template <typename K>
+int attn_opt_in(K kernel, bool* done, int smem_optin, char* err) {
+  std::lock_guard<std::mutex> lock(g_adev_mu);
+  if (*done) return 0;
+  cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
+  if (e != cudaSuccess) { snprintf(err, 256, "attention: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
+  *done = true;
+  return 0;
+}
+}  // namespace
+
 int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens, int B, int S, int A, int d,
                     float scale, int* status, cudaStream_t st, char* err) {
-  static int num_sms = 0, smem_optin = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (num_sms <= 0) { snprintf(err, 256, "attention: no CUDA device"); return MSLT_ERR_CUDA; }
-  }
+  // the test hook is used up by this call even if an argument check below rejects it
+  const bool starve = g_attn_starve.exchange(0) != 0;
+  AttnDevice* adev = attn_device(err);
+  if (!adev) return MSLT_ERR_CUDA;
+  const int num_sms = adev->num_sms, smem_optin = adev->smem_optin;
   if (d != 64 || S < 1 || S > 512 || B < 1 || A < 1 || !status) {
     snprintf(err, 256, "attention: the fused kernel needs head width 64 and 1 <= S <= 512");
     return MSLT_ERR_ARG;
@@ -1041,7 +1074,7 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
   p.fast_p = (probs != nullptr && S % 32 == 0) ? row_fast(probs, S) : 0;
   p.wait_limit = WAIT_LIMIT_CYCLES;
   p.status = status;
-  if (g_attn_starve.exchange(0)) {  // armed by mslt_debug_starve_next_attention
+  if (starve) {  // armed by mslt_debug_starve_next_attention
     p.starve = 1;
     p.wait_limit = 40000000ll;  // about 20 ms
   }
@@ -1064,12 +1097,8 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
     const size_t smem_long = 2 * (size_t)AT_TILE_BYTES + (size_t)AL_KV_STAGES * AL_KV_BYTES + AL_P_BYTES +
                              NUM_EPI_WARPS * AT_STAGING + 2 * 2 * 128 * sizeof(float2) + 1024 + 256;
     if ((int)smem_long > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
-    static bool attr_long = false;
-    if (!attr_long) {
-      cudaError_t e = cudaFuncSetAttribute(attn_fwd_long_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
-      if (e != cudaSuccess) { snprintf(err, 256, "attention: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
-      attr_long = true;
-    }
+    rc = attn_opt_in(attn_fwd_long_kernel, &adev->attr_long, smem_optin, err);
+    if (rc) return rc;
     const int grid_long = p.items < num_sms ? p.items : num_sms;
     attn_fwd_long_kernel<<<grid_long, NUM_THREADS, smem_long, st>>>(mq.map, mk.map, mv.map, p);
     cudaError_t e = cudaGetLastError();
@@ -1079,12 +1108,8 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
   }
   const size_t smem_bytes = (size_t)AT_STAGES * AT_STAGE_BYTES + NUM_EPI_WARPS * AT_STAGING + 1024 + 256;
   if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
-    if (e != cudaSuccess) { snprintf(err, 256, "attention: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
-    attr_set = true;
-  }
+  rc = attn_opt_in(attn_fwd_kernel, &adev->attr_fwd, smem_optin, err);
+  if (rc) return rc;
   const int grid = p.items < num_sms ? p.items : num_sms;
   attn_fwd_kernel<<<grid, NUM_THREADS, smem_bytes, st>>>(mq.map, mk.map, mv.map, p);
   cudaError_t e = cudaGetLastError();
@@ -1095,14 +1120,11 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
 
 int attn_bwd_launch(const void* qkv, const void* probs, const void* dctx, void* dqkv, int B, int S, int A, int d,
                     float scale, int* status, cudaStream_t st, char* err) {
-  static int num_sms = 0, smem_optin = 0;
-  if (num_sms == 0) {
-    int dev = 0;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&num_sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaDeviceGetAttribute(&smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-    if (num_sms <= 0) { snprintf(err, 256, "attention: no CUDA device"); return MSLT_ERR_CUDA; }
-  }
+  // the test hook is used up by this call even if an argument check below rejects it
+  const bool starve = g_attn_starve.exchange(0) != 0;
+  AttnDevice* adev = attn_device(err);
+  if (!adev) return MSLT_ERR_CUDA;
+  const int num_sms = adev->num_sms, smem_optin = adev->smem_optin;
   if (d != 64 || S < 8 || S > 128 || S % 8 || B < 1 || A < 1 || !status || !qkv || !probs || !dctx || !dqkv) {
     snprintf(err, 256, "attention backward: the fused kernel needs head width 64 and S a multiple of 8 in [8, 128]");
     return MSLT_ERR_ARG;
@@ -1116,7 +1138,7 @@ int attn_bwd_launch(const void* qkv, const void* probs, const void* dctx, void* 
   p.fast = 0;  // direct 32-byte row stores measured slower here (58 vs 54 us): three 128-byte pieces per row
   p.wait_limit = WAIT_LIMIT_CYCLES;
   p.status = status;
-  if (g_attn_starve.exchange(0)) {  // armed by mslt_debug_starve_next_attention
+  if (starve) {  // armed by mslt_debug_starve_next_attention
     p.starve = 1;
     p.wait_limit = 40000000ll;  // about 20 ms
   }
@@ -1144,12 +1166,8 @@ int attn_bwd_launch(const void* qkv, const void* probs, const void* dctx, void* 
   }
   const size_t smem_bytes = (size_t)2 * AB_STAGE_BYTES + NUM_EPI_WARPS * AT_STAGING + 1024 + 256;
   if ((int)smem_bytes > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
-  static bool attr_set = false;
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(attn_bwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin);
-    if (e != cudaSuccess) { snprintf(err, 256, "attention: cudaFuncSetAttribute: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
-    attr_set = true;
-  }
+  rc = attn_opt_in(attn_bwd_kernel, &adev->attr_bwd, smem_optin, err);
+  if (rc) return rc;
   const int grid = p.items < num_sms ? p.items : num_sms;
   attn_bwd_kernel<<<grid, NUM_THREADS, smem_bytes, st>>>(mq.map, mk.map, mv.map, mc.map, mp.map, p);
   cudaError_t e = cudaGetLastError();

@@ -865,6 +865,8 @@ std::mutex g_dev_mu;
 }  // namespace
 
 int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* err) {
+  // the test hook is used up by this call even if an argument check below rejects it
+  const bool starve = g_starve_next.exchange(0) != 0;
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) {
     snprintf(err, 256, "gemm: no CUDA device");
@@ -967,7 +969,7 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   p.aux = (bf16*)d.aux; p.residual = (const bf16*)d.residual; p.status = status;
   p.seq_lens = d.seq_lens;
   p.wait_limit = WAIT_LIMIT_CYCLES;
-  if (g_starve_next.exchange(0)) {  // armed by mslt_debug_starve_next_gemm
+  if (starve) {  // armed by mslt_debug_starve_next_gemm
     p.starve = 1;
     p.wait_limit = 40000000ll;  // about 20 ms
   }

@@ -530,7 +530,10 @@ __global__ void slots_prepare_kernel(const int* __restrict__ positions,
     const int pos = positions[r];
     const int lab = labels ? labels[r] : 0;
     bool ok = pos >= 0 && lab >= 0;
-    if (pos >= S) { bad |= ST_BAD_POSITION; ok = false; }
+    // a position at or beyond the sequence's length would read a padded row, whose content is unspecified
+    int len = S;
+    if (seq_lens != nullptr) len = min(max(seq_lens[b], 1), S);
+    if (pos >= len) { bad |= ST_BAD_POSITION; ok = false; }
     if (lab >= V) { bad |= ST_BAD_LABEL; ok = false; }
     rowsrc[r] = ok ? b * S + pos : -1;
     rowlabel[r] = ok ? lab : -1;

@@ -141,6 +141,8 @@ int check_arch(const mslt_arch* a) {
     return fail(MSLT_ERR_ARG, "max_seq must be a multiple of 8 in [8, 512]");
   if (a->max_pos < a->max_seq) return fail(MSLT_ERR_ARG, "max_pos < max_seq");
   if (!(a->ln_eps >= 0.f)) return fail(MSLT_ERR_ARG, "ln_eps must be >= 0");
+  if (a->max_trainable < 0 || a->max_trainable > a->max_layers)
+    return fail(MSLT_ERR_ARG, "need 0 <= max_trainable <= max_layers");
   return 0;
 }
 
@@ -176,6 +178,9 @@ void build_tensor_table(const mslt_arch& a, std::vector<Tensor>& out, int64_t& t
 
 constexpr int64_t kAdamChunk = 8192;
 
+// saved-activation slots: one per layer that may be trainable at the same time
+int trainable_slots(const mslt_arch& a) { return a.max_trainable > 0 ? a.max_trainable : a.max_layers; }
+
 // Lays out the workspace; with base == nullptr only the size is computed.
 void plan_workspace(const mslt_arch& a, const std::vector<Tensor>& tensors, char* base,
                     Workspace& w) {
@@ -210,8 +215,10 @@ void plan_workspace(const mslt_arch& a, const std::vector<Tensor>& tensors, char
     b.st1 = (float*)take(T * 2 * 4); b.st2 = (float*)take(T * 2 * 4);
   };
   take_layer(w.scratch);
-  w.layer.resize(a.max_layers);
-  for (int l = 0; l < a.max_layers; l++) take_layer(w.layer[l]);
+  // Only the trainable top layers save activations (the bottom layers run forward only and share
+  // the scratch slot above): trainable layer l of a step uses slot l - (L - top_k).
+  w.layer.resize(trainable_slots(a));
+  for (int l = 0; l < trainable_slots(a); l++) take_layer(w.layer[l]);
   w.z0 = take(T * H * E);
   w.st0 = (float*)take(T * 2 * 4);
   w.hm = take(R * H * E); w.ut = take(R * H * E); w.gt = take(R * H * E); w.tm = take(R * H * E);
@@ -662,7 +669,7 @@ int mslt_create(const mslt_arch* arch, void* dev_params, size_t param_bytes, voi
   c->st = (cudaStream_t)cuda_stream;
   c->opt = {1e-3f, 0.9f, 0.999f, 1e-6f, 0.01f, 1};
   c->L = arch->init_layers;
-  c->top_k = c->L;
+  c->top_k = std::min(c->L, trainable_slots(*arch));
   c->t_step = 0;
   c->launches = 0;
   c->timing = false;
@@ -729,6 +736,9 @@ int mslt_add_layers(mslt_ctx* c, int32_t k) {
 int mslt_set_trainable(mslt_ctx* c, int32_t top_k) {
   if (!c) return fail(MSLT_ERR_ARG, "null context");
   if (top_k < 0 || top_k > c->L) return fail(MSLT_ERR_STATE, "set_trainable: need 0 <= top_k <= L");
+  if (top_k > trainable_slots(c->a))
+    return fail(MSLT_ERR_SIZE, "set_trainable: top_k = %d exceeds max_trainable = %d, the number of saved-activation "
+                "slots the workspace was sized for", top_k, trainable_slots(c->a));
   c->top_k = top_k;
   return reset_optimizer(c);
 }
@@ -777,8 +787,9 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   const char* boundary = cur;  // the only output of the frozen prefix
   mark(c, 1);
   for (int l = first; l < c->L; l++) {
-    TRY(layer_forward(c, l, cur, w.layer[l], w.layer[l].xout, true, B, S, d_seq_lens));
-    cur = w.layer[l].xout;
+    LayerBuf& slot = w.layer[l - first];
+    TRY(layer_forward(c, l, cur, slot, slot.xout, true, B, S, d_seq_lens));
+    cur = slot.xout;
   }
   mark(c, 2);
   TRY(head_forward(c, cur, R, true));
@@ -790,9 +801,9 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   char* dx = w.dxa;
   char* dx_other = w.dxb;
   for (int l = c->L - 1; l >= first; l--) {
-    const void* x_in = l == first ? (const void*)boundary : (const void*)w.layer[l - 1].xout;
+    const void* x_in = l == first ? (const void*)boundary : (const void*)w.layer[l - 1 - first].xout;
     const bool need_dx = l > first || full;
-    TRY(layer_backward(c, l, x_in, w.layer[l], dx, dx_other, need_dx, B, S));
+    TRY(layer_backward(c, l, x_in, w.layer[l - first], dx, dx_other, need_dx, B, S));
     if (need_dx) std::swap(dx, dx_other);
   }
   if (full) {

@@ -49,7 +49,8 @@ def bf16_round(x: np.ndarray) -> np.ndarray:
     return ((u + bias) >> 16).astype(np.uint16)
 
 
-def build_pair(cfg: I.StageConfig, lr: float, max_layers=None, init_layers=None, seed=None, **opt):
+def build_pair(cfg: I.StageConfig, lr: float, max_layers=None, init_layers=None, seed=None,
+               max_trainable: int = 0, **opt):
     """(library context, oracle) with identical weights, boundary and hyper-parameters."""
     from paper_2011_13635_b200.binding import Mslt
     L0 = cfg.layers if init_layers is None else init_layers
@@ -61,7 +62,7 @@ def build_pair(cfg: I.StageConfig, lr: float, max_layers=None, init_layers=None,
     # both sides get the same numbers: the C ABI carries hyper-parameters as float32
     hyper = {k: (float(np.float32(v)) if k != "bias_correction" else v) for k, v in hyper.items()}
     oracle.set_optimizer(**hyper)
-    m = Mslt.from_config(cfg, init_layers=L0, max_layers=max_layers or cfg.layers)
+    m = Mslt.from_config(cfg, init_layers=L0, max_layers=max_layers or cfg.layers, max_trainable=max_trainable)
     m.set_params(w)
     m.mslt_set_optimizer(**hyper)
     if init_layers is None:

@@ -39,6 +39,18 @@ def test_host_side_validation(binding):
         with pytest.raises(binding.MsltError) as ei:
             binding.mslt_query_bytes(b)
         assert ei.value.code == -1, field
+    # saved activations are reserved for the layers that can be trainable at once: 9 + 3 needs 3 slots
+    a3 = binding.Arch(768, 12, 3072, 30522, 512, 3, 12, 128, 128, 20, 1, 1e-12, 3)
+    pb3, wb3 = binding.mslt_query_bytes(a3)
+    T, H, F, A, S = 128 * 128, 768, 3072, 12, 128
+    slot = 2 * (3 * T * H + 128 * A * S * S + 5 * T * H + 2 * T * F)      # bf16 bytes of one layer's slot
+    assert pb3 == pb
+    assert 9 * slot <= wb - wb3 <= 9 * slot * 1.01
+    assert wb3 < 0.45 * wb
+    a3.max_trainable = 13
+    with pytest.raises(binding.MsltError) as ei:
+        binding.mslt_query_bytes(a3)
+    assert ei.value.code == -1
     # fp32 path has no bf16 copy
     a32 = binding.Arch(128, 2, 512, 1024, 64, 2, 2, 8, 64, 10, 0, 1e-12)
     pb32, _ = binding.mslt_query_bytes(a32)

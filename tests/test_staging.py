@@ -54,6 +54,30 @@ def test_schedule_of_stages_matches_oracle(cfg):
 
 
 @pytest.mark.parametrize("cfg", [CFG32, CFG16], ids=["fp32", "bf16"])
+def test_saved_activation_slots_only_for_the_trainable_layers(cfg):
+    """A context sized for two trainable layers out of four: smaller workspace, same results, and a
+    request for more trainable layers than it has slots for is refused."""
+    from paper_2011_13635_b200 import binding as Bd
+    lr = 1e-3 if cfg.dtype == "fp32" else 1e-4
+    m, oracle = PT.build_pair(cfg, lr=lr, max_trainable=2)
+    assert m.num_layers == 4 and m.num_trainable == 2
+    full_ws = Bd.mslt_query_bytes(Bd.Arch(cfg.hidden, cfg.heads, cfg.ffn, cfg.vocab, cfg.max_pos, 4, 4, cfg.batch,
+                                          cfg.seq, cfg.pred, 0 if cfg.dtype == "fp32" else 1, 1e-12, 0))[1]
+    assert m.workspace_bytes < full_ws
+    seed = I.config_seed(cfg)
+    for s in range(2):
+        PT.compare_step(m, oracle, cfg, I.make_batch(cfg, seed=seed + s), PT.TOL[cfg.dtype])
+    m.mslt_set_trainable(1)
+    oracle.set_trainable(1)
+    PT.compare_step(m, oracle, cfg, I.make_batch(cfg, seed=seed + 2), PT.TOL[cfg.dtype])
+    with pytest.raises(Bd.MsltError) as ei:
+        m.mslt_set_trainable(3)
+    assert ei.value.code == -2 and "max_trainable" in str(ei.value)
+    assert m.num_trainable == 1
+    m.close()
+
+
+@pytest.mark.parametrize("cfg", [CFG32, CFG16], ids=["fp32", "bf16"])
 def test_truncation_leaves_top_gradients_unchanged(cfg):
     """Gradients of the trainable slice from a staged step equal the same tensors' gradients
     from an all-trainable step at identical weights."""

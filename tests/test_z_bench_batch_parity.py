@@ -19,7 +19,7 @@ pytestmark = pytest.mark.gpu
 def test_base_stage_batch_128_whole_step_against_the_oracle():
     cfg = I.CONFIGS["base_stage"]
     assert (cfg.batch, cfg.seq, cfg.layers, cfg.trainable) == (128, 128, 12, 3)
-    m, oracle = PT.build_pair(cfg, lr=1e-4)
+    m, oracle = PT.build_pair(cfg, lr=1e-4, max_trainable=cfg.trainable)     # as bench.py creates it
     rep = []
     PT.compare_step(m, oracle, cfg, I.make_batch(cfg), PT.TOL[cfg.dtype], rep)
     r = rep[0]
