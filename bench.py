@@ -5,9 +5,13 @@
 One "step" is one pass of the whole hot path (frozen-prefix forward, trainable forward and
 backward, MLM head and loss, Adam on the trainable slice) over one synthetic batch.  The path
 does not shard: with N > 1 every rank runs an independent replica on its own batch (no
-collective on the data path) and the aggregate throughput is reported.
+collective on the data path) and the aggregate throughput is reported; started without a
+launcher, `--gpus N` starts its N processes itself.
 
-Prints ONE JSON line (rank 0).
+Prints ONE JSON line (rank 0).  The headline is the BERT-Base stage configuration (9 frozen + 3
+trainable layers); at one GPU the line also carries a `configs` record with every stage
+configuration timed the same way, the contraction kernel's rate against both measured cuBLAS
+figures, and the memory-bound kernels one at a time.
 """
 from __future__ import annotations
 
@@ -157,10 +161,14 @@ def run_reference(args, cfg):
         return
     n_seq = 2
     base, dt = cpu_baseline(cfg, n_seq, steps=args.steps, warmup=args.warmup)
+    conf = describe(cfg)
+    conf["sample"] = (f"each step is the oracle on {n_seq} of the {cfg.batch} sequences of the batch (full "
+                      "architecture); value = those sequences per second")
+    conf["launch"] = "numpy float64 on the host cores"
     line = dict(impl="reference", metric=METRIC, value=base["value"], unit=UNIT, n_gpus=args.gpus,
                 steps=args.steps, warmup=args.warmup, ms_per_step=1e3 * dt / args.steps,
                 higher_is_better=True, scaling="weak", vs_baseline=None, dtype="f64", data="synthetic",
-                config=describe(cfg), cpu_baseline=base,
+                config=conf, cpu_baseline=base,
                 e2e=dict(value=base["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0))
     print(json.dumps(line))
 
@@ -225,16 +233,23 @@ def aggregate(ms_local: float, batch_per_rank: int, steps: int, world: int, dist
     return ms, batch_per_rank * world * steps / (ms * 1e-3)
 
 
-def run_ours(args, cfg):
-    import torch
-    import torch.distributed as dist
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    torch.cuda.set_device(local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+# DRAM bytes per launch of the contraction kernel from ncu captures of single launches (summaries
+# and commands under profiles/); None where the kernel has changed since the counters were taken.
+GEMM_DRAM_BYTES_PER_LAUNCH = None
 
+
+def gemm_peaks(peaks, clocks):
+    """Which measured cuBLAS figure the step's contractions are held against: the burst figure when
+    the sampled SM clock stayed near its maximum, the sustained one when it shows the power-capped
+    regime (both fractions are printed either way)."""
+    mhz, mx = clocks.get("sm_mhz"), clocks.get("sm_max_mhz")
+    capped = bool(mhz and mx and mhz < 0.9 * mx)
+    return ("sustained" if capped else "burst"), peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+
+
+def measure(cfg, args, torch, dist, world, rank, local, steps, warmup, headline):
+    """Times `steps` steps of one configuration on this rank's GPU.  Returns the JSON record of the
+    configuration (rank 0 adds the per-kernel passes) and, for the headline, the e2e figures."""
     def sync():
         torch.cuda.synchronize()
         if world > 1:
@@ -254,105 +269,199 @@ def run_ours(args, cfg):
         raise RuntimeError("non-finite loss")
 
     with ClockSampler(local) as clk:
-        ms, launches, graph = time_steps(m, dev, torch, args.steps, args.warmup, sync, args.graph)
+        ms, launches, graph = time_steps(m, dev, torch, steps, warmup, sync, args.graph)
     loss_end = m.mslt_read_loss()
-    ms, value = aggregate(ms, cfg.batch, args.steps, world, dist, "cuda")
+    ms, value = aggregate(ms, cfg.batch, steps, world, dist, "cuda" if world > 1 else "cpu")
+    clocks = clk.summary()
+    rec = dict(ms_per_step=ms / steps, value=value, unit=UNIT, steps=steps, warmup=warmup,
+               gpu_launches=int(launches), launches_per_step=launches / steps, clocks=clocks,
+               loss=dict(first=loss0, last=loss_end), workspace_gb=m.workspace_bytes / 1e9,
+               param_block_gb=m.param_bytes / 1e9)
 
-    # end to end: pinned host inputs copied in, loss read back, every step
-    sync()
-    with torch.cuda.stream(stream):
-        t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
-        t0.record(stream)
-        for _ in range(args.steps):
-            for d_, p_ in zip(dev, pinned):
-                if d_ is not None:
-                    d_.copy_(p_, non_blocking=True)
-            if graph is not None:
-                graph.replay()
-                m.mslt_read_loss()
-            else:
-                m.mslt_step(*dev)
-        t1.record(stream)
+    e2e = None
+    if headline:
+        # end to end: pinned host inputs copied in, loss read back, every step
         sync()
-    _, e2e_value = aggregate(t0.elapsed_time(t1), cfg.batch, args.steps, world, dist, "cuda")
-    e2e = dict(value=e2e_value, unit=UNIT,
-               h2d_bytes_per_step=int(sum(a.nbytes for a in host if a is not None)),
-               d2h_bytes_per_step=16)
+        with torch.cuda.stream(stream):
+            t0 = torch.cuda.Event(enable_timing=True); t1 = torch.cuda.Event(enable_timing=True)
+            t0.record(stream)
+            for _ in range(steps):
+                for d_, p_ in zip(dev, pinned):
+                    if d_ is not None:
+                        d_.copy_(p_, non_blocking=True)
+                if graph is not None:
+                    graph.replay()
+                    m.mslt_read_loss()
+                else:
+                    m.mslt_step(*dev)
+            t1.record(stream)
+            sync()
+        _, e2e_value = aggregate(t0.elapsed_time(t1), cfg.batch, steps, world, dist, "cuda" if world > 1 else "cpu")
+        e2e = dict(value=e2e_value, unit=UNIT,
+                   h2d_bytes_per_step=int(sum(a.nbytes for a in host if a is not None)),
+                   d2h_bytes_per_step=16)
     del graph
-
-    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
-                warmup=args.warmup, ms_per_step=ms / args.steps, higher_is_better=True, scaling="weak",
-                vs_baseline=None, dtype=cfg.dtype, data="synthetic", config=describe(cfg), e2e=e2e,
-                gpu_launches=int(launches), clocks=clk.summary(),
-                loss=dict(first=loss0, last=loss_end))
 
     if rank == 0:
         peaks = measured_peaks()
-        # per-kernel pass: the same steps again with an event pair around every contraction
+        # per-kernel pass: the same steps again with an event pair around every launch
         m.mslt_set_timing(2)
         m.mslt_get_kernel_profile()
-        n_prof = max(1, min(args.steps, 5))
+        n_prof = max(1, min(steps, 5))
         with torch.cuda.stream(stream):
             for _ in range(n_prof):
                 m.mslt_step(*dev, sync=False)
         torch.cuda.synchronize()
         prof = m.mslt_get_kernel_profile()
-        phases = m.mslt_get_timings()
+        rec["phases_ms"] = m.mslt_get_timings()
         m.mslt_set_timing(0)
         lin, att = prof["linear"], prof["attention"]
         lin_tflops = lin["work"] / (lin["ms"] * 1e-3) / 1e12 if lin["ms"] > 0 else 0.0
-        peak = peaks["bf16_tflops_sustained"] if cfg.dtype == "bf16" else None
         if cfg.dtype == "bf16":
-            line["roofline"] = dict(
+            regime, burst, sustained = gemm_peaks(peaks, clocks)
+            peak = burst if regime == "burst" else sustained
+            rec["roofline"] = dict(
                 bound="tensor", kernel="gemm_tc_kernel (linear-layer products of the step)",
-                achieved=lin_tflops, peak=peak, unit="TFLOP/s", frac=lin_tflops / peak, traffic=None,
-                peak_source=f"{peaks['source']}: cuBLAS bf16 sustained (kernel timed inside a long step)",
+                achieved=lin_tflops, peak=peak, unit="TFLOP/s", frac=lin_tflops / peak,
+                traffic=GEMM_DRAM_BYTES_PER_LAUNCH,
+                peak_source=f"{peaks['source']}: cuBLAS bf16 8192^3, {regime} figure (median SM clock "
+                            f"{clocks.get('sm_mhz')} of {clocks.get('sm_max_mhz')} MHz in the timed region)",
+                frac_of_burst=lin_tflops / burst, frac_of_sustained=lin_tflops / sustained,
+                peak_burst=burst, peak_sustained=sustained,
                 launches_per_step=lin["launches"] / n_prof,
                 avg_launch_us=1e3 * lin["ms"] / max(lin["launches"], 1),
+                launch_us_x_sm_mhz=(1e3 * lin["ms"] / max(lin["launches"], 1)) * (clocks.get("sm_mhz") or 0.0),
                 flops_per_step=lin["work"] / n_prof,
-                share_of_step_time=lin["ms"] / n_prof / (ms / args.steps))
+                share_of_step_time=lin["ms"] / n_prof / (ms / steps))
         else:
-            line["roofline"] = dict(bound="alu", kernel="gemm_simt_kernel", achieved=lin_tflops, peak=None,
-                                    unit="TFLOP/s", frac=None, traffic=None)
-        # attention: fused kernels (HBM-bound) where the sequence fits one tile, batched products otherwise
-        line["attention"] = dict(
+            rec["roofline"] = dict(bound="alu", kernel="gemm_simt_kernel", achieved=lin_tflops, peak=None,
+                                   unit="TFLOP/s", frac=None, traffic=None,
+                                   note="fp32 CUDA-core path of the small configuration: launch-bound")
+        # attention: fused kernels (HBM-bound) where they apply, batched products otherwise
+        rec["attention"] = dict(
             tflops=att["work"] / (att["ms"] * 1e-3) / 1e12 if att["ms"] > 0 else 0.0,
             ms_per_step=att["ms"] / n_prof, launches_per_step=att["launches"] / n_prof)
-        line["phases_ms"] = phases
-        line["hbm_kernels"] = {
-            k: dict(gbs=v["work"] / (v["ms"] * 1e-3) / 1e9, frac_of_measured_copy=v["work"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        rec["hbm_kernels"] = {
+            k: dict(gbs=v["work"] / (v["ms"] * 1e-3) / 1e9,
+                    frac_of_measured_copy=v["work"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
                     ms_per_step=v["ms"] / n_prof, launches_per_step=v["launches"] / n_prof)
             for k, v in prof.items() if k not in ("linear", "attention") and v["ms"] > 0}
-        line["step_tflops"] = step_flops(cfg) / (ms / args.steps * 1e-3) / 1e12
-        m.close()
-        del m
-        torch.cuda.empty_cache()
-        if world == 1 and args.ratio and cfg.name == "base_stage":
-            full = I.CONFIGS["base_full"]
-            mf = make_model(full, torch, stream)
-            k = max(3, min(args.steps, 10))
-            ms_f, _, gf = time_steps(mf, dev, torch, k, 3, sync, args.graph)
-            del gf
-            line["stage_vs_full"] = dict(
-                staged_ms=ms / args.steps, full_ms=ms_f / k, ratio=(ms / args.steps) / (ms_f / k),
-                note="step time of 9 frozen + 3 trainable layers over all 12 trainable, same shapes, "
-                     "data and seed, one GPU, no communication")
-            mf.close()
+        rec["step_tflops"] = step_flops(cfg) / (ms / steps * 1e-3) / 1e12
+    m.close()
+    del m
+    torch.cuda.empty_cache()
+    return rec, e2e
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    rec, e2e = measure(cfg, args, torch, dist, world, rank, local, args.steps, args.warmup, True)
+    line = dict(metric=METRIC, value=rec["value"], unit=UNIT, n_gpus=world, steps=args.steps,
+                warmup=args.warmup, ms_per_step=rec["ms_per_step"], higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype=cfg.dtype, data="synthetic", config=describe(cfg), e2e=e2e,
+                gpu_launches=rec["gpu_launches"], clocks=rec["clocks"], loss=rec["loss"])
+    if rank == 0:
+        for k in ("roofline", "attention", "phases_ms", "hbm_kernels", "step_tflops", "workspace_gb", "param_block_gb"):
+            if k in rec:
+                line[k] = rec[k]
+        peaks = measured_peaks()
+        if world == 1 and args.all_configs:
+            # every stage configuration, timed the same way (fewer steps); spec ratio from the two
+            # BERT-Base ones
+            short = max(10, args.steps // 4)
+            per = {cfg.name: rec}
+            for name in ("tiny", "base_stage", "base_full", "large_stage", "large_long"):
+                if name in per:
+                    continue
+                per[name], _ = measure(I.CONFIGS[name], args, torch, dist, world, rank, local, short, 3, False)
+            line["configs"] = {
+                n: dict(ms_per_step=r["ms_per_step"], sequences_per_s=r["value"], steps=r["steps"],
+                        launches_per_step=r["launches_per_step"], clocks=r["clocks"],
+                        gemm_tflops=r["roofline"]["achieved"],
+                        gemm_frac_of_burst=r["roofline"].get("frac_of_burst"),
+                        gemm_frac_of_sustained=r["roofline"].get("frac_of_sustained"),
+                        attention_ms=r["attention"]["ms_per_step"], phases_ms=r["phases_ms"],
+                        step_tflops=r["step_tflops"], workspace_gb=r["workspace_gb"],
+                        hbm_kernels={k: round(v["frac_of_measured_copy"], 3) for k, v in r["hbm_kernels"].items()})
+                for n, r in per.items()}
+            if "base_stage" in per and "base_full" in per:
+                a, b = per["base_stage"]["ms_per_step"], per["base_full"]["ms_per_step"]
+                line["stage_vs_full"] = dict(
+                    staged_ms=a, full_ms=b, ratio=a / b,
+                    note="step time of 9 frozen + 3 trainable layers over all 12 trainable, same shapes, "
+                         "data and seed, one GPU, no communication")
         if world == 1 and cfg.dtype == "bf16" and cfg.seq <= 512 and args.isolated:
-            # the same kernels one at a time, back to back on rotating buffers larger than L2: no
-            # event pair per launch, so short kernels are not understated as in hbm_kernels
+            # the memory-bound kernels one at a time, back to back on rotating buffers larger than L2:
+            # no event pair per launch, so short kernels are not understated as in hbm_kernels
             from paper_2011_13635_b200 import op_bench
-            recs = op_bench.main(["--rows", str(cfg.batch * cfg.seq), "--hidden", str(cfg.hidden), "--ffn", str(cfg.ffn),
-                                  "--heads", str(cfg.heads), "--seq", str(cfg.seq), "--batch", str(cfg.batch),
-                                  "--iters", "20", "--only", "attention,ln,colsum"], emit=None)
+            with ClockSampler(local) as clk2:
+                recs = op_bench.main(["--rows", str(cfg.batch * cfg.seq), "--hidden", str(cfg.hidden), "--ffn", str(cfg.ffn),
+                                      "--heads", str(cfg.heads), "--seq", str(cfg.seq), "--batch", str(cfg.batch),
+                                      "--iters", "20", "--only", "attention,ln,colsum,ce"], emit=None)
             line["hbm_kernels_alone"] = {
-                r["kernel"]: dict(us=r["us"], gbs=r["gbs"], frac_of_measured_copy=r["gbs"] / peaks["hbm_gbs"])
+                r["kernel"]: dict(us=r["us"], gbs=r["gbs"], frac_of_measured_copy=r["gbs"] / peaks["hbm_gbs"],
+                                  dram_bytes_ncu=HBM_DRAM_BYTES_NCU.get(r["kernel"]))
                 for r in recs}
+            line["hbm_kernels_alone"]["clocks"] = clk2.summary()
             torch.cuda.empty_cache()
         if world == 1:
-            n_seq = args.cpu_seqs
-            line["cpu_baseline"], _ = cpu_baseline(cfg, n_seq)
+            line["cpu_baseline"], _ = cpu_baseline(cfg, args.cpu_seqs)
         print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+# DRAM bytes per launch of the memory-bound kernels at the op_bench sizes, from one-kernel ncu captures
+# (profiles/); keys are op_bench's kernel names.  Empty until the captures are taken for this build.
+HBM_DRAM_BYTES_NCU = {}
+
+
+# ------------------------------------------------------------------------------------------------
+# N replicas on N GPUs when started as a plain `python bench.py --gpus N`
+# ------------------------------------------------------------------------------------------------
+def free_port() -> int:
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    return port
+
+
+def launch_replicas(n: int, argv):
+    """Starts n copies of this script, one per GPU (RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* set as a
+    launcher would), waits for them and returns the worst exit code.  Rank 0 prints the JSON line."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__), *argv], env=env))
+    return max(abs(p.wait()) for p in procs)
+
+
+def run_selftest_cpu(args):
+    """The launcher and the aggregation without a GPU: every rank pretends its timed region took
+    10 * (rank + 1) ms and the ranks meet over gloo."""
+    import torch.distributed as dist
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    if world > 1:
+        dist.init_process_group("gloo", init_method=f"tcp://{os.environ['MASTER_ADDR']}:{os.environ['MASTER_PORT']}",
+                                rank=rank, world_size=world)
+    cfg = I.CONFIGS[args.config]
+    ms, value = aggregate(10.0 * (rank + 1), cfg.batch, args.steps, world, dist, "cpu")
+    if rank == 0:
+        print(json.dumps(dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps,
+                              ms_per_step=ms / args.steps, selftest="cpu")))
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -361,12 +470,14 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="base_stage", choices=sorted(I.CONFIGS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-seqs", type=int, default=8, help="sequences in the oracle's timed sample")
-    ap.add_argument("--no-ratio", dest="ratio", action="store_false")
+    ap.add_argument("--no-ratio", "--one-config", dest="all_configs", action="store_false",
+                    help="time only the headline configuration (no `configs` record, no staged : full ratio)")
+    ap.add_argument("--selftest-cpu", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--no-isolated", dest="isolated", action="store_false",
                     help="skip the one-kernel-at-a-time bandwidth figures")
     ap.add_argument("--no-graph", dest="graph", action="store_false",
@@ -374,7 +485,12 @@ def main():
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     cfg = I.CONFIGS[args.config]
-    if args.impl == "reference":
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        # not under a launcher: start the replicas ourselves, one process per GPU
+        sys.exit(launch_replicas(args.gpus, sys.argv[1:]))
+    if args.selftest_cpu:
+        run_selftest_cpu(args)
+    elif args.impl == "reference":
         run_reference(args, cfg)
     else:
         run_ours(args, cfg)

@@ -135,6 +135,28 @@ def adam_update(w, g, m, v, t: int, lr, beta1, beta2, eps, weight_decay, bias_co
     return w, m, v
 
 
+def lamb_update(w, g, m, v, t: int, lr, beta1, beta2, eps, weight_decay, bias_correction: bool):
+    """One LAMB step on one tensor (the optimizer of the paper's experiments, Section 4.1; You
+    et al., "Large batch optimization for deep learning", Algorithm 2 with the identity as scaling
+    function).  The Adam direction plus decoupled decay, r = m_hat / (sqrt(v_hat) + eps) + wd * w,
+    is rescaled per tensor by the trust ratio ||w|| / ||r|| (Euclidean norms over the whole
+    tensor; the ratio is 1 when either norm is 0):  w <- w - lr * (||w|| / ||r||) * r.
+    t is the step count after this update.  Returns (w, m, v)."""
+    m = beta1 * m + (1.0 - beta1) * g
+    v = beta2 * v + (1.0 - beta2) * g * g
+    if bias_correction:
+        mh = m / (1.0 - beta1 ** t)
+        vh = v / (1.0 - beta2 ** t)
+    else:
+        mh, vh = m, v
+    r = mh / (np.sqrt(vh) + eps) + weight_decay * w
+    wn = math.sqrt(float(np.sum(w * w)))
+    rn = math.sqrt(float(np.sum(r * r)))
+    ratio = wn / rn if (wn > 0.0 and rn > 0.0) else 1.0
+    w = w - lr * ratio * r
+    return w, m, v
+
+
 # ----------------------------------------------------------------------------
 # the model
 # ----------------------------------------------------------------------------
@@ -160,7 +182,7 @@ class MsltOracle:
         self.V = self.p["emb.word"].shape[0]
         self.top_k = self.L
         self.opt = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01,
-                        bias_correction=1)
+                        bias_correction=1, lamb=0)
         self.grads: Dict[str, np.ndarray] = {}
         self._reset_optimizer()
 
@@ -345,13 +367,14 @@ class MsltOracle:
 
     # -- one training step ------------------------------------------------------------
     def step(self, tokens, seq_lens, positions, labels) -> float:
-        """Forward, truncated backward, Adam on the trainable tensors only."""
+        """Forward, truncated backward, Adam (or LAMB, opt["lamb"] = 1) on the trainable tensors only."""
         loss, g = self.loss_and_grads(tokens, seq_lens, positions, labels)
         self.t += 1
         o = self.opt
+        update = lamb_update if o.get("lamb") else adam_update
         for n in self.trainable_names():
             wd = o["weight_decay"] if self.p[n].ndim == 2 else 0.0
-            self.p[n], self.m[n], self.v[n] = adam_update(
+            self.p[n], self.m[n], self.v[n] = update(
                 self.p[n], g[n], self.m[n], self.v[n], self.t, o["lr"], o["beta1"], o["beta2"],
                 o["eps"], wd, bool(o["bias_correction"]))
         return loss

@@ -477,3 +477,79 @@ def test_batches_follow_the_recipe():
     a = I.make_batch(I.scaled(I.CONFIGS["base_stage"], batch=2))
     b = I.make_batch(I.scaled(I.CONFIGS["base_full"], batch=2))
     assert all(np.array_equal(x, y) for x, y in zip(a, b))         # same seed, same data
+
+
+# -- LAMB (the optimizer of the paper's experiments, Section 4.1) -----------------------------------
+
+def _lamb_by_hand(w, g, m, v, t, lr, b1, b2, eps, wd, bc):
+    """The same rule element by element with plain Python floats."""
+    n = len(w)
+    m2 = [b1 * m[i] + (1 - b1) * g[i] for i in range(n)]
+    v2 = [b2 * v[i] + (1 - b2) * g[i] * g[i] for i in range(n)]
+    c1 = 1 - b1 ** t if bc else 1.0
+    c2 = 1 - b2 ** t if bc else 1.0
+    r = [(m2[i] / c1) / (math.sqrt(v2[i] / c2) + eps) + wd * w[i] for i in range(n)]
+    wn = math.sqrt(sum(x * x for x in w)); rn = math.sqrt(sum(x * x for x in r))
+    ratio = wn / rn if wn > 0 and rn > 0 else 1.0
+    return [w[i] - lr * ratio * r[i] for i in range(n)], m2, v2
+
+
+def test_lamb_closed_forms():
+    rng = np.random.default_rng(16)
+    n = 40
+    w = rng.standard_normal(n); g = rng.standard_normal(n) * 3
+    z = np.zeros(n)
+    lr, eps = 0.00088, 1e-6
+    # brute force, with history and decay
+    m0 = rng.standard_normal(n) * 0.1; v0 = np.abs(rng.standard_normal(n)) * 0.1
+    got = O.lamb_update(w, g, m0, v0, 5, lr, 0.9, 0.999, eps, 0.01, True)
+    want = _lamb_by_hand(list(w), list(g), list(m0), list(v0), 5, lr, 0.9, 0.999, eps, 0.01, True)
+    for a, b in zip(got, want):
+        np.testing.assert_allclose(a, np.array(b), rtol=1e-12, atol=1e-15)
+    # first step, no decay: the direction is g / (|g| + eps), one unit per element, so the step of every
+    # element has size lr * ||w|| / sqrt(n) (up to eps / |g|) whatever the size of the gradient
+    w1, _, _ = O.lamb_update(w, g, z, z, 1, lr, 0.9, 0.999, eps, 0.0, True)
+    r = g / (np.abs(g) + eps)
+    np.testing.assert_allclose(w1 - w, -lr * np.linalg.norm(w) / np.linalg.norm(r) * r, atol=1e-15)
+    big = np.abs(g) > 1e-2
+    np.testing.assert_allclose(np.abs(w1 - w)[big], lr * np.linalg.norm(w) / math.sqrt(n), rtol=2e-4)
+    # the update does not change when the gradient is rescaled (eps aside) ...
+    w1b, _, _ = O.lamb_update(w, 100.0 * g, z, z, 1, lr, 0.9, 0.999, 0.0 + 1e-30, 0.0, True)
+    w1c, _, _ = O.lamb_update(w, g, z, z, 1, lr, 0.9, 0.999, 0.0 + 1e-30, 0.0, True)
+    np.testing.assert_allclose(w1b, w1c, atol=1e-14)
+    # ... and scales with the weights: the step is relative to ||w||
+    w3, _, _ = O.lamb_update(3.0 * w, g, z, z, 1, lr, 0.9, 0.999, eps, 0.0, True)
+    np.testing.assert_allclose(w3 - 3.0 * w, 3.0 * (w1 - w), atol=1e-14)
+    # the norm of the whole step is lr * ||w|| exactly (that is what the trust ratio does)
+    assert abs(np.linalg.norm(w1 - w) - lr * np.linalg.norm(w)) < 1e-14
+    wd_step, _, _ = O.lamb_update(w, g, m0, v0, 7, lr, 0.9, 0.999, eps, 0.05, True)
+    assert abs(np.linalg.norm(wd_step - w) - lr * np.linalg.norm(w)) < 1e-14
+    # zero gradient and no decay: nothing moves; zero gradient with decay: pure shrink by lr (ratio = 1 / wd)
+    w4, _, _ = O.lamb_update(w, z, z, z, 1, lr, 0.9, 0.999, eps, 0.0, True)
+    assert np.array_equal(w4, w)
+    w5, _, _ = O.lamb_update(w, z, z, z, 1, lr, 0.9, 0.999, eps, 0.1, True)
+    np.testing.assert_allclose(w5, w * (1 - lr), atol=1e-15)
+    # a tensor of zeros has no norm to be relative to: trust ratio 1, i.e. a plain Adam step
+    w6, _, _ = O.lamb_update(z, g, z, z, 1, lr, 0.9, 0.999, eps, 0.0, True)
+    w6a, _, _ = O.adam_update(z, g, z, z, 1, lr, 0.9, 0.999, eps, 0.0, True)
+    np.testing.assert_allclose(w6, w6a, atol=1e-18)
+    # moments are Adam's
+    _, mm, vv = O.lamb_update(w, g, m0, v0, 5, lr, 0.9, 0.999, eps, 0.01, True)
+    _, ma, va = O.adam_update(w, g, m0, v0, 5, lr, 0.9, 0.999, eps, 0.01, True)
+    assert np.array_equal(mm, ma) and np.array_equal(vv, va)
+
+
+def test_step_with_lamb_updates_every_trainable_tensor_by_its_own_norm():
+    m = tiny_model(top_k=1)
+    lr = 0.00088
+    m.set_optimizer(lr=lr, weight_decay=0.0, lamb=1)
+    tok, lens, pos, lab = tiny_batch()
+    before = {k: v.copy() for k, v in m.p.items()}
+    m.step(tok, lens, pos, lab)
+    names = set(m.trainable_names())
+    for k in before:
+        if k in names:
+            # the trust ratio is per tensor: each tensor's step has norm lr * its own norm
+            assert abs(np.linalg.norm(m.p[k] - before[k]) - lr * np.linalg.norm(before[k])) < 1e-12, k
+        else:
+            assert np.array_equal(m.p[k], before[k]), k
