@@ -67,10 +67,17 @@ typedef struct {
                        /* saved-activation slots: BERT-Base 9 + 3 needs 3 of them, not 12             */
 } mslt_arch;
 
-/* Adam with decoupled weight decay (decay on matrices and tables only). */
+/*
+ * Optimizer of the trainable parameters.  Adam with decoupled weight decay (decay on matrices and
+ * tables only), or, with lamb = 1, LAMB, the optimizer of the paper's experiments (Section 4.1,
+ * learning rate 0.00088): the same direction r = m_hat / (sqrt(v_hat) + eps) + decay * w, scaled
+ * for every tensor by its trust ratio ||w|| / ||r|| (Euclidean norms over the tensor; 1 when
+ * either norm is 0), w <- w - lr * ratio * r.
+ */
 typedef struct {
   float lr, beta1, beta2, eps, weight_decay;
   int32_t bias_correction; /* 1: divide m, v by (1 - beta^t)                           */
+  int32_t lamb;            /* 0: Adam; 1: LAMB                                         */
 } mslt_opt;
 
 /*

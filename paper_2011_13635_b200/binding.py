@@ -31,7 +31,7 @@ class Arch(C.Structure):
 
 class Opt(C.Structure):
     _fields_ = [("lr", C.c_float), ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float),
-                ("weight_decay", C.c_float), ("bias_correction", C.c_int32)]
+                ("weight_decay", C.c_float), ("bias_correction", C.c_int32), ("lamb", C.c_int32)]
 
 
 class GemmDesc(C.Structure):
@@ -264,8 +264,8 @@ class Mslt:
         _check(lib.mslt_set_trainable(self.h, top_k))
 
     def mslt_set_optimizer(self, lr, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01,
-                           bias_correction=1):
-        o = Opt(lr, beta1, beta2, eps, weight_decay, int(bias_correction))
+                           bias_correction=1, lamb=0):
+        o = Opt(lr, beta1, beta2, eps, weight_decay, int(bias_correction), int(lamb))
         _check(lib.mslt_set_optimizer(self.h, C.byref(o)))
 
     # -- the hot path -------------------------------------------------------------------------

@@ -892,6 +892,85 @@ adam_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ w,
   }
 }
 
+// LAMB, first kernel: new moments, and the per-tensor sums of w^2 and r^2
+__global__ void __launch_bounds__(256)
+lamb_moments_kernel(const AdamChunk* __restrict__ chunks, const float* __restrict__ w,
+                    const float* __restrict__ g, float* __restrict__ m, float* __restrict__ v, AdamHyper h,
+                    const float* __restrict__ bc, float* __restrict__ norms) {
+  h.bc1 = bc[0];
+  h.bc2 = bc[1];
+  const AdamChunk ch = chunks[blockIdx.x];
+  const float decay = h.weight_decay * ch.decay;
+  float sw = 0.f, sr = 0.f;
+  for (int i = threadIdx.x * 4; i < ch.count; i += 256 * 4) {
+    const int64_t o = ch.offset + i;
+    const float4 wv = *reinterpret_cast<const float4*>(w + o);
+    const float4 gv = *reinterpret_cast<const float4*>(g + o);
+    float4 mv = *reinterpret_cast<float4*>(m + o);
+    float4 vv = *reinterpret_cast<float4*>(v + o);
+    const float* wp = &wv.x; const float* gp = &gv.x; float* mp = &mv.x; float* vp = &vv.x;
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const float mm = h.beta1 * mp[e] + h.omb1 * gp[e];
+      const float vn = h.beta2 * vp[e] + h.omb2 * gp[e] * gp[e];
+      const float r = (mm * h.bc1) / (sqrtf(vn * h.bc2) + h.eps) + decay * wp[e];
+      sw += wp[e] * wp[e];
+      sr += r * r;
+      mp[e] = mm;
+      vp[e] = vn;
+    }
+    *reinterpret_cast<float4*>(m + o) = mv;
+    *reinterpret_cast<float4*>(v + o) = vv;
+  }
+  __shared__ float red[2][8];
+  sw = warp_sum(sw);
+  sr = warp_sum(sr);
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = sw; red[1][threadIdx.x >> 5] = sr; }
+  __syncthreads();
+  if (threadIdx.x < 32) {
+    float a = threadIdx.x < 8 ? red[0][threadIdx.x] : 0.f, b = threadIdx.x < 8 ? red[1][threadIdx.x] : 0.f;
+    a = warp_sum(a);
+    b = warp_sum(b);
+    if (threadIdx.x == 0) {
+      atomicAdd(norms + 2 * ch.tensor, a);
+      atomicAdd(norms + 2 * ch.tensor + 1, b);
+    }
+  }
+}
+
+// LAMB, second kernel: the step, scaled by the tensor's trust ratio
+__global__ void __launch_bounds__(256)
+lamb_apply_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ w, const float* __restrict__ m,
+                  const float* __restrict__ v, bf16* __restrict__ wb, AdamHyper h,
+                  const float* __restrict__ bc, const float* __restrict__ norms) {
+  h.bc1 = bc[0];
+  h.bc2 = bc[1];
+  const AdamChunk ch = chunks[blockIdx.x];
+  const float decay = h.weight_decay * ch.decay;
+  const float wn = sqrtf(norms[2 * ch.tensor]), rn = sqrtf(norms[2 * ch.tensor + 1]);
+  const float step = h.lr * ((wn > 0.f && rn > 0.f) ? wn / rn : 1.f);
+  for (int i = threadIdx.x * 4; i < ch.count; i += 256 * 4) {
+    const int64_t o = ch.offset + i;
+    float4 wv = *reinterpret_cast<float4*>(w + o);
+    const float4 mv = *reinterpret_cast<const float4*>(m + o);
+    const float4 vv = *reinterpret_cast<const float4*>(v + o);
+    float* wp = &wv.x; const float* mp = &mv.x; const float* vp = &vv.x;
+#pragma unroll
+    for (int e = 0; e < 4; e++) {
+      const float r = (mp[e] * h.bc1) / (sqrtf(vp[e] * h.bc2) + h.eps) + decay * wp[e];
+      wp[e] = wp[e] - step * r;
+    }
+    *reinterpret_cast<float4*>(w + o) = wv;
+    if (wb != nullptr) {
+      __nv_bfloat162 lo = __floats2bfloat162_rn(wv.x, wv.y), hi = __floats2bfloat162_rn(wv.z, wv.w);
+      uint2 pk;
+      pk.x = *reinterpret_cast<uint32_t*>(&lo);
+      pk.y = *reinterpret_cast<uint32_t*>(&hi);
+      *reinterpret_cast<uint2*>(wb + o) = pk;
+    }
+  }
+}
+
 // d[i] *= gelu'(u[i]) (MLM transform backward)
 template <typename T>
 __global__ void dgelu_kernel(T* __restrict__ d, const T* __restrict__ u, int64_t n) {
@@ -1059,6 +1138,16 @@ void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g
   adam_tick_kernel<<<1, 1, 0, st>>>(t_dev, bc_dev, h.beta1, h.beta2, bias_correction);
   if (n_chunks <= 0) return;
   adam_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, g, m, v, (bf16*)wb, h, bc_dev);
+}
+
+void launch_lamb(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,
+                 void* wb, const AdamHyper& h, int* t_dev, float* bc_dev, int bias_correction,
+                 float* norms, int n_tensors, cudaStream_t st) {
+  adam_tick_kernel<<<1, 1, 0, st>>>(t_dev, bc_dev, h.beta1, h.beta2, bias_correction);
+  if (n_chunks <= 0) return;
+  cudaMemsetAsync(norms, 0, (size_t)n_tensors * 2 * sizeof(float), st);
+  lamb_moments_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, g, m, v, h, bc_dev, norms);
+  lamb_apply_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, m, v, (bf16*)wb, h, bc_dev, norms);
 }
 
 void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st) {

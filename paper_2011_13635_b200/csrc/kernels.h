@@ -11,6 +11,8 @@ struct AdamChunk {
   int64_t offset;  // element offset into the parameter arena (multiple of 4)
   int32_t count;   // elements in this chunk (multiple of 4)
   float decay;     // 1 for matrices and tables, 0 for vectors
+  int32_t tensor;  // index of the tensor the chunk belongs to (LAMB sums its norms per tensor)
+  int32_t pad_;
 };
 struct AdamHyper {
   float lr, beta1, beta2, eps, weight_decay;
@@ -51,6 +53,13 @@ void launch_embed_scatter(bool bf, const void* dz, const int* tokens, float* dwo
 void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,
                  void* wb, const AdamHyper& h, int* t_dev, float* bc_dev, int bias_correction,
                  cudaStream_t st);
+// LAMB on the same chunk table: the Adam direction r = m_hat / (sqrt(v_hat) + eps) + decay * w is
+// scaled per tensor by ||w|| / ||r|| (1 when either norm is 0).  Two kernels: the first updates m and
+// v and sums w^2 and r^2 of every tensor into norms[2 * tensor] / [2 * tensor + 1] (zeroed here);
+// the second forms r again from the new moments and applies the step.  n_tensors: entries of norms.
+void launch_lamb(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,
+                 void* wb, const AdamHyper& h, int* t_dev, float* bc_dev, int bias_correction,
+                 float* norms, int n_tensors, cudaStream_t st);
 // d[i] *= gelu'(u[i]); n a multiple of the vector width
 void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st);
 void launch_f32_to_bf16(const float* src, void* dst, int64_t n, cudaStream_t st);

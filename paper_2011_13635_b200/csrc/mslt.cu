@@ -72,6 +72,7 @@ struct Workspace {
   int* scalars;  // [0] status, [1] n_valid, [2] inv_n (float), [3] loss (float), [4] Adam step count,
                  // [5], [6] Adam bias corrections (float)
   int *rowsrc, *rowlabel;
+  float* norms;  // LAMB: sums of w^2 and r^2 per tensor
   AdamChunk* chunks;
   int64_t max_chunks;
   char *xa, *xb;
@@ -206,6 +207,7 @@ void plan_workspace(const mslt_arch& a, const std::vector<Tensor>& tensors, char
   w.max_chunks = 0;
   for (const Tensor& t : tensors) w.max_chunks += (t.padded + kAdamChunk - 1) / kAdamChunk;
   w.chunks = (AdamChunk*)take(w.max_chunks * sizeof(AdamChunk));
+  w.norms = (float*)take(tensors.size() * 2 * sizeof(float));
   w.xa = take(T * H * E);
   w.xb = take(T * H * E);
   auto take_layer = [&](LayerBuf& b) {
@@ -267,13 +269,16 @@ float* G(const mslt_ctx* c, int64_t off) { return c->grad + off; }
 
 int rebuild_chunks(mslt_ctx* c) {
   std::vector<AdamChunk> h;
-  for (const Tensor& t : c->tensors) {
+  for (size_t ti = 0; ti < c->tensors.size(); ti++) {
+    const Tensor& t = c->tensors[ti];
     if (t.layer >= c->L || !is_trainable(c, t)) continue;
     for (int64_t o = 0; o < t.padded; o += kAdamChunk) {
       AdamChunk ch;
       ch.offset = t.offset + o;
       ch.count = (int32_t)std::min<int64_t>(kAdamChunk, t.padded - o);
       ch.decay = t.rank == 2 ? 1.f : 0.f;
+      ch.tensor = (int32_t)ti;
+      ch.pad_ = 0;
       h.push_back(ch);
     }
   }
@@ -667,7 +672,7 @@ int mslt_create(const mslt_arch* arch, void* dev_params, size_t param_bytes, voi
   c->bf = arch->dtype == 1;
   c->esz = c->bf ? 2 : 4;
   c->st = (cudaStream_t)cuda_stream;
-  c->opt = {1e-3f, 0.9f, 0.999f, 1e-6f, 0.01f, 1};
+  c->opt = {1e-3f, 0.9f, 0.999f, 1e-6f, 0.01f, 1, 0};
   c->L = arch->init_layers;
   c->top_k = std::min(c->L, trainable_slots(*arch));
   c->t_step = 0;
@@ -747,6 +752,7 @@ int mslt_set_optimizer(mslt_ctx* c, const mslt_opt* o) {
   if (!c || !o) return fail(MSLT_ERR_ARG, "null pointer");
   if (!(o->beta1 >= 0.f && o->beta1 < 1.f && o->beta2 >= 0.f && o->beta2 < 1.f && o->eps > 0.f))
     return fail(MSLT_ERR_ARG, "bad Adam hyper-parameters");
+  if (o->lamb != 0 && o->lamb != 1) return fail(MSLT_ERR_ARG, "lamb must be 0 or 1");
   c->opt = *o;
   return 0;
 }
@@ -820,8 +826,15 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   h.omb1 = (float)(1.0 - (double)c->opt.beta1);
   h.omb2 = (float)(1.0 - (double)c->opt.beta2);
   h.bc1 = h.bc2 = 1.f;  // formed on the device from the step count kept there
-  KL(PC_ADAM, 30.0 * c->n_chunks * kAdamChunk, launch_adam(w.chunks, c->n_chunks, c->master, c->grad, c->m, c->v, c->wb, h, w.scalars + 4,
-                 (float*)(w.scalars + 5), c->opt.bias_correction, c->st));
+  if (c->opt.lamb) {
+    KL(PC_ADAM, 42.0 * c->n_chunks * kAdamChunk, launch_lamb(w.chunks, c->n_chunks, c->master, c->grad, c->m, c->v, c->wb, h,
+                   w.scalars + 4, (float*)(w.scalars + 5), c->opt.bias_correction, w.norms, (int)c->tensors.size(), c->st));
+    c->launches += 2;  // step-count kernel, moments kernel, update kernel
+  } else {
+    KL(PC_ADAM, 30.0 * c->n_chunks * kAdamChunk, launch_adam(w.chunks, c->n_chunks, c->master, c->grad, c->m, c->v, c->wb, h, w.scalars + 4,
+                   (float*)(w.scalars + 5), c->opt.bias_correction, c->st));
+    c->launches++;  // step-count kernel and update kernel
+  }
   mark(c, 5);
   if (c->timing && c->have_events) {
     CUDA_TRY(cudaEventSynchronize(c->ev[5]));

@@ -14,8 +14,8 @@ pytestmark = pytest.mark.gpu
 TINY = I.CONFIGS["tiny"]
 
 
-def _run(cfg, steps, lr, batch_seed=None):
-    m, oracle = PT.build_pair(cfg, lr=lr)
+def _run(cfg, steps, lr, batch_seed=None, **opt):
+    m, oracle = PT.build_pair(cfg, lr=lr, **opt)
     tol = PT.TOL[cfg.dtype]
     rep = []
     for s in range(steps):
@@ -46,6 +46,12 @@ def test_fp32_ragged_shapes_with_padding():
     _run(I.scaled(cfg, trainable=3), steps=2, lr=1e-3)
 
 
+def test_fp32_lamb_staged_and_all_trainable():
+    """LAMB at the learning rate of the paper's experiments (Section 4.1): per-tensor trust ratios."""
+    _run(TINY, steps=3, lr=0.00088, lamb=1)
+    _run(I.scaled(TINY, trainable=2), steps=2, lr=0.00088, lamb=1, weight_decay=0.0)
+
+
 # -- bf16 path ---------------------------------------------------------------------------------
 
 BASE_SMALL = I.scaled(I.CONFIGS["base_stage"], layers=3, trainable=2, batch=4)
@@ -59,6 +65,11 @@ def test_bf16_base_shapes_staged():
 
 def test_bf16_base_shapes_all_trainable():
     _run(I.scaled(BASE_SMALL, layers=2, trainable=2, batch=3), steps=2, lr=1e-4)
+
+
+def test_bf16_lamb_base_shapes():
+    _run(BASE_SMALL, steps=2, lr=0.00088, lamb=1)
+    _run(I.scaled(BASE_SMALL, layers=2, trainable=2, batch=2), steps=1, lr=0.00088, lamb=1)
 
 
 def test_bf16_head_only():
