@@ -268,11 +268,35 @@ def measure(cfg, args, torch, dist, world, rank, local, steps, warmup, headline)
     if not np.isfinite(loss0):
         raise RuntimeError("non-finite loss")
 
+    dp = None
+    if args.data_parallel:
+        # every rank takes its own share of the global batch; the gradients of the trainable slice are
+        # all-reduced bucket by bucket while the backward pass goes on (steps run eagerly)
+        from paper_2011_13635_b200.data_parallel import DataParallelStep
+        dp = DataParallelStep(m, dist if world > 1 else None)
     with ClockSampler(local) as clk:
-        ms, launches, graph = time_steps(m, dev, torch, steps, warmup, sync, args.graph)
+        if dp is None:
+            ms, launches, graph = time_steps(m, dev, torch, steps, warmup, sync, args.graph)
+        else:
+            graph = None
+            with torch.cuda.stream(m.stream):
+                for _ in range(warmup):
+                    dp.step(*dev, read_loss=False)
+                sync()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                before = m.launch_count
+                e0.record(m.stream)
+                for _ in range(steps):
+                    dp.step(*dev, read_loss=False)
+                e1.record(m.stream)
+                sync()
+            ms, launches = e0.elapsed_time(e1), m.launch_count - before
     loss_end = m.mslt_read_loss()
     ms, value = aggregate(ms, cfg.batch, steps, world, dist, "cuda" if world > 1 else "cpu")
     clocks = clk.summary()
+    if dp is not None:
+        args.dp_note = dict(buckets=len(dp.buckets), gradient_bytes_per_step=dp.bytes_exchanged,
+                            of_all_parameters_bytes=4 * sum(int(np.prod(i["shape"])) for i in m.tensors().values()))
     rec = dict(ms_per_step=ms / steps, value=value, unit=UNIT, steps=steps, warmup=warmup,
                gpu_launches=int(launches), launches_per_step=launches / steps, clocks=clocks,
                loss=dict(first=loss0, last=loss_end), workspace_gb=m.workspace_bytes / 1e9,
@@ -292,6 +316,8 @@ def measure(cfg, args, torch, dist, world, rank, local, steps, warmup, headline)
                 if graph is not None:
                     graph.replay()
                     m.mslt_read_loss()
+                elif dp is not None:
+                    dp.step(*dev)
                 else:
                     m.mslt_step(*dev)
             t1.record(stream)
@@ -368,12 +394,17 @@ def run_ours(args, cfg):
                 warmup=args.warmup, ms_per_step=rec["ms_per_step"], higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype=cfg.dtype, data="synthetic", config=describe(cfg), e2e=e2e,
                 gpu_launches=rec["gpu_launches"], clocks=rec["clocks"], loss=rec["loss"])
+    if args.data_parallel:
+        line["config"]["parallelism"] = (f"data parallel over {world} GPU(s): all-reduce (NCCL) of the trainable "
+                                         "gradient slice only, bucket by bucket behind the backward pass")
+        line["config"]["launch"] = "eager launches (the exchange hooks run on the host)"
+        line["data_parallel"] = getattr(args, "dp_note", None)
     if rank == 0:
         for k in ("roofline", "attention", "phases_ms", "hbm_kernels", "step_tflops", "workspace_gb", "param_block_gb"):
             if k in rec:
                 line[k] = rec[k]
         peaks = measured_peaks()
-        if world == 1 and args.all_configs:
+        if world == 1 and args.all_configs and not args.data_parallel:
             # every stage configuration, timed the same way (fewer steps); spec ratio from the two
             # BERT-Base ones
             short = max(10, args.steps // 4)
@@ -478,6 +509,9 @@ def main():
     ap.add_argument("--no-ratio", "--one-config", dest="all_configs", action="store_false",
                     help="time only the headline configuration (no `configs` record, no staged : full ratio)")
     ap.add_argument("--selftest-cpu", action="store_true", help=argparse.SUPPRESS)
+    ap.add_argument("--data-parallel", action="store_true",
+                    help="N workers train ONE model: gradients of the trainable slice are all-reduced (the default "
+                         "is N independent replicas)")
     ap.add_argument("--no-isolated", dest="isolated", action="store_false",
                     help="skip the one-kernel-at-a-time bandwidth figures")
     ap.add_argument("--no-graph", dest="graph", action="store_false",

@@ -150,6 +150,43 @@ int mslt_step(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens,
               const int32_t* d_mlm_positions, const int32_t* d_mlm_labels, int32_t B, int32_t S,
               int32_t P, float* loss_out);
 
+/*
+ * The same step in two halves, for data-parallel training (Section 3.1, last paragraph, and Section
+ * 4.1: every worker takes a share of the batch, and only the gradients of the trainable top layers
+ * and the output layer are exchanged; those of the bottom layers are neither computed nor
+ * communicated).  mslt_step_backward runs forward, loss and backward and leaves the gradients of
+ * the trainable parameters in the gradient arena; the caller sums them over the workers;
+ * mslt_step_apply then runs the optimizer.  Between the two calls only the gradient buckets may be
+ * touched (no mslt_step, mslt_set_trainable or mslt_add_layers: MSLT_ERR_STATE).
+ *   d_total_valid  device int32 or NULL: number of valid MLM slots over ALL workers' batches.  With
+ *                  it the loss and the gradients are divided by that count, so that the SUM over
+ *                  workers of the returned losses and of the gradients is exactly the mean loss of
+ *                  the concatenated batch and its gradient.  NULL: this batch's own count.
+ * Other arguments as for mslt_step.
+ */
+int mslt_step_backward(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens,
+                       const int32_t* d_mlm_positions, const int32_t* d_mlm_labels, int32_t B, int32_t S,
+                       int32_t P, const int32_t* d_total_valid, float* loss_out);
+int mslt_step_apply(mslt_ctx* ctx);
+
+/*
+ * Gradient buckets: the trainable gradients as a few contiguous fp32 device ranges, numbered in
+ * the order in which mslt_step_backward completes them: 0 the output layer, 1..top_k the trainable
+ * layers from the top down, then the embeddings when every layer is trainable.  The frozen layers
+ * have no bucket: that is the communication the method saves.
+ */
+int mslt_num_grad_buckets(const mslt_ctx* ctx);
+int mslt_grad_bucket(mslt_ctx* ctx, int32_t index, float** d_ptr, int64_t* count);
+/*
+ * Overlap of the exchange with the rest of the backward pass: if a hook is set, mslt_step_backward
+ * calls fn(user, bucket) on the host as soon as the kernels that complete that bucket have been
+ * enqueued; comm_stream (a cudaStream_t) has been made to wait for them, so a reduction enqueued on
+ * it by the hook runs while the layers below are still in their backward pass.  mslt_step_apply
+ * makes the context's stream wait for everything enqueued on comm_stream.  fn = NULL clears it.
+ */
+typedef void (*mslt_bucket_fn)(void* user, int32_t bucket);
+int mslt_set_bucket_hook(mslt_ctx* ctx, void* comm_stream, mslt_bucket_fn fn, void* user);
+
 /* Synchronises the stream and returns the loss of the last mslt_step (host pointer). */
 int mslt_read_loss(mslt_ctx* ctx, float* loss_out);
 

@@ -48,7 +48,8 @@ class GemmDesc(C.Structure):
 
 
 EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers", "mslt_set_trainable",
-           "mslt_set_optimizer", "mslt_step", "mslt_read_loss", "mslt_forward", "mslt_num_layers",
+           "mslt_set_optimizer", "mslt_step", "mslt_step_backward", "mslt_step_apply", "mslt_num_grad_buckets",
+           "mslt_grad_bucket", "mslt_set_bucket_hook", "mslt_read_loss", "mslt_forward", "mslt_num_layers",
            "mslt_num_trainable", "mslt_num_tensors", "mslt_tensor_info", "mslt_get_param",
            "mslt_set_param", "mslt_get_param_raw", "mslt_get_grad", "mslt_get_opt_state",
            "mslt_launch_count", "mslt_set_timing", "mslt_get_timings", "mslt_get_kernel_profile",
@@ -68,6 +69,13 @@ lib.mslt_query_bytes.argtypes = [C.POINTER(Arch), C.POINTER(C.c_size_t), C.POINT
 lib.mslt_create.argtypes = [C.POINTER(Arch), C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t,
                             C.c_void_p, C.POINTER(C.c_void_p)]
 lib.mslt_destroy.argtypes = [C.c_void_p]
+BUCKET_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_int32)
+lib.mslt_step_backward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
+                                   C.c_int32, C.c_void_p, C.POINTER(C.c_float)]
+lib.mslt_step_apply.argtypes = [C.c_void_p]
+lib.mslt_num_grad_buckets.argtypes = [C.c_void_p]
+lib.mslt_grad_bucket.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64)]
+lib.mslt_set_bucket_hook.argtypes = [C.c_void_p, C.c_void_p, BUCKET_FN, C.c_void_p]
 lib.mslt_add_layers.argtypes = [C.c_void_p, C.c_int32]
 lib.mslt_set_trainable.argtypes = [C.c_void_p, C.c_int32]
 lib.mslt_set_optimizer.argtypes = [C.c_void_p, C.POINTER(Opt)]
@@ -278,6 +286,42 @@ class Mslt:
         _check(lib.mslt_step(self.h, tokens.data_ptr(), _ptr(seq_lens), mlm_positions.data_ptr(),
                              mlm_labels.data_ptr(), B, S, P, C.byref(loss) if sync else None))
         return loss.value if sync else None
+
+    def mslt_step_backward(self, tokens, seq_lens, mlm_positions, mlm_labels, total_valid=None, sync: bool = True):
+        """Forward, loss and backward only; total_valid: int32 CUDA tensor of one element (valid slots
+        over all workers) or None.  Returns this worker's share of the loss when sync."""
+        B, S = tokens.shape
+        P = mlm_positions.shape[1]
+        loss = C.c_float()
+        _check(lib.mslt_step_backward(self.h, tokens.data_ptr(), _ptr(seq_lens), mlm_positions.data_ptr(),
+                                      mlm_labels.data_ptr(), B, S, P, _ptr(total_valid),
+                                      C.byref(loss) if sync else None))
+        return loss.value if sync else None
+
+    def mslt_step_apply(self):
+        _check(lib.mslt_step_apply(self.h))
+
+    def grad_buckets(self):
+        """The trainable gradients as float32 CUDA tensors that alias the gradient arena, in the order
+        in which a backward pass completes them (output layer, layers top-down, embeddings)."""
+        torch = self.torch
+        flat = self._params.view(torch.float32)
+        out = []
+        for i in range(lib.mslt_num_grad_buckets(self.h)):
+            ptr, cnt = C.c_void_p(), C.c_int64()
+            _check(lib.mslt_grad_bucket(self.h, i, C.byref(ptr), C.byref(cnt)))
+            first = (ptr.value - self._params.data_ptr()) // 4
+            out.append(flat[first:first + cnt.value])
+        return out
+
+    def mslt_set_bucket_hook(self, comm_stream, fn):
+        """fn(bucket_index) is called on the host when a bucket's kernels are enqueued; None clears."""
+        if fn is None:
+            self._hook = None
+            _check(lib.mslt_set_bucket_hook(self.h, None, BUCKET_FN(), None))
+            return
+        self._hook = BUCKET_FN(lambda user, i: fn(int(i)))      # keep the callback object alive
+        _check(lib.mslt_set_bucket_hook(self.h, C.c_void_p(comm_stream.cuda_stream), self._hook, None))
 
     def mslt_read_loss(self) -> float:
         loss = C.c_float()

@@ -780,6 +780,11 @@ __global__ void loss_reduce_kernel(const float* __restrict__ nll, int R,
   }
 }
 
+__global__ void override_inv_n_kernel(const int* __restrict__ total_valid, float* __restrict__ inv_n) {
+  const int n = *total_valid;
+  *inv_n = n > 0 ? 1.0f / (float)n : 0.f;
+}
+
 // ---------------------------------------------------------------------------------------
 // Column sums (bias gradients): out[n] += sum_rows x[row, n].
 // ---------------------------------------------------------------------------------------
@@ -1108,6 +1113,10 @@ void launch_cross_entropy(bool bf, const float* logits, int64_t ldl, const int* 
   else
     DISPATCH_T(bf, (cross_entropy_kernel<T><<<R, 256, 0, st>>>(logits, ldl, rowlabel, inv_n,
                                                               (T*)dlogits, ldd, nll, V)));
+}
+
+void launch_override_inv_n(const int* total_valid, float* inv_n, cudaStream_t st) {
+  override_inv_n_kernel<<<1, 1, 0, st>>>(total_valid, inv_n);
 }
 
 void launch_loss_reduce(const float* nll, int R, const float* inv_n, float* loss, cudaStream_t st) {

@@ -61,6 +61,8 @@ void launch_lamb(const AdamChunk* chunks, int n_chunks, float* w, const float* g
                  void* wb, const AdamHyper& h, int* t_dev, float* bc_dev, int bias_correction,
                  float* norms, int n_tensors, cudaStream_t st);
 // d[i] *= gelu'(u[i]); n a multiple of the vector width
+// data-parallel steps: the loss normaliser becomes 1 / *total_valid (0 when that count is 0)
+void launch_override_inv_n(const int* total_valid, float* inv_n, cudaStream_t st);
 void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st);
 void launch_f32_to_bf16(const float* src, void* dst, int64_t n, cudaStream_t st);
 

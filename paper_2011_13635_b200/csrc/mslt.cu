@@ -115,6 +115,14 @@ struct mslt_ctx {
   struct PRec { int cls; double flops; };
   std::vector<PRec> prec;
   double prof[10][3];  // per kernel class: launches, work (flops or bytes), ms
+  // data-parallel hook: called on the host each time the kernels that finish a gradient bucket have
+  // been enqueued (the communication stream already waits for them)
+  cudaStream_t comm;
+  mslt_bucket_fn bucket_fn;
+  void* bucket_user;
+  std::vector<cudaEvent_t> bev;
+  cudaEvent_t comm_done;
+  bool pending_update;  // mslt_step_backward ran, mslt_step_apply has not yet
 };
 
 namespace {
@@ -610,6 +618,28 @@ int zero_trainable_grads(mslt_ctx* c) {
   return 0;
 }
 
+// Gradient buckets in the order in which a step completes them: the output layer, the trainable
+// layers from the top down, then (only when everything trains) the embeddings.  Each is one contiguous
+// range of the fp32 gradient arena.
+int num_buckets(const mslt_ctx* c) { return 1 + c->top_k + (c->top_k == c->L ? 1 : 0); }
+void bucket_range(const mslt_ctx* c, int i, int64_t* off, int64_t* cnt) {
+  if (i == 0) { *off = c->head_off; *cnt = c->head_cnt; }
+  else if (i <= c->top_k) { *off = c->layer0_off + (int64_t)(c->L - i) * c->layer_cnt; *cnt = c->layer_cnt; }
+  else { *off = c->emb_off; *cnt = c->emb_cnt; }
+}
+int bucket_done(mslt_ctx* c, int i) {
+  if (!c->bucket_fn) return 0;
+  while ((int)c->bev.size() <= i) {
+    cudaEvent_t e;
+    CUDA_TRY(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+    c->bev.push_back(e);
+  }
+  CUDA_TRY(cudaEventRecord(c->bev[i], c->st));
+  CUDA_TRY(cudaStreamWaitEvent(c->comm, c->bev[i], 0));
+  c->bucket_fn(c->bucket_user, i);
+  return 0;
+}
+
 int check_batch(mslt_ctx* c, int B, int S, int P) {
   if (B < 1 || S < 1 || P < 0) return fail(MSLT_ERR_ARG, "bad batch shape");
   if (B > c->a.max_batch || S > c->a.max_seq || P > c->a.max_pred)
@@ -680,6 +710,11 @@ int mslt_create(const mslt_arch* arch, void* dev_params, size_t param_bytes, voi
   c->timing = false;
   c->have_events = false;
   c->profile = 0;
+  c->comm = nullptr;
+  c->bucket_fn = nullptr;
+  c->bucket_user = nullptr;
+  c->comm_done = nullptr;
+  c->pending_update = false;
   memset(c->prof, 0, sizeof(c->prof));
   c->Vp = (int)pad_to(arch->vocab, 8);
   build_tensor_table(*arch, c->tensors, c->n_elems);
@@ -719,6 +754,8 @@ int mslt_destroy(mslt_ctx* c) {
   if (c->have_events)
     for (int i = 0; i < 6; i++) cudaEventDestroy(c->ev[i]);
   for (cudaEvent_t e : c->pev) cudaEventDestroy(e);
+  for (cudaEvent_t e : c->bev) cudaEventDestroy(e);
+  if (c->comm_done) cudaEventDestroy(c->comm_done);
   delete c;
   return 0;
 }
@@ -740,6 +777,7 @@ int mslt_add_layers(mslt_ctx* c, int32_t k) {
 
 int mslt_set_trainable(mslt_ctx* c, int32_t top_k) {
   if (!c) return fail(MSLT_ERR_ARG, "null context");
+  if (c->pending_update) return fail(MSLT_ERR_STATE, "set_trainable: a step is waiting for mslt_step_apply");
   if (top_k < 0 || top_k > c->L) return fail(MSLT_ERR_STATE, "set_trainable: need 0 <= top_k <= L");
   if (top_k > trainable_slots(c->a))
     return fail(MSLT_ERR_SIZE, "set_trainable: top_k = %d exceeds max_trainable = %d, the number of saved-activation "
@@ -757,10 +795,15 @@ int mslt_set_optimizer(mslt_ctx* c, const mslt_opt* o) {
   return 0;
 }
 
-int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
-              const int32_t* d_pos, const int32_t* d_lab, int32_t B, int32_t S, int32_t P,
-              float* loss_out) {
+static int apply_update(mslt_ctx* c);
+
+// forward, loss and backward of one step; the optimizer runs too unless `defer_update`
+static int step_impl(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
+                     const int32_t* d_pos, const int32_t* d_lab, int32_t B, int32_t S, int32_t P,
+                     const int32_t* d_total_valid, bool defer_update, float* loss_out) {
   if (!c || !d_tokens || !d_pos || !d_lab) return fail(MSLT_ERR_ARG, "null pointer");
+  if (c->pending_update)
+    return fail(MSLT_ERR_STATE, "mslt_step_backward was called: call mslt_step_apply before the next step");
   TRY(check_batch(c, B, S, P));
   if (P < 1) return fail(MSLT_ERR_ARG, "P must be >= 1");
   Workspace& w = c->ws;
@@ -779,6 +822,8 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   mark(c, 0);
   KL(PC_OTHER, 16.0 * B * P, launch_slots_prepare(d_pos, d_lab, d_seq_lens, B, S, P, V, w.rowsrc, w.rowlabel, w.scalars + 1,
                           inv_n, status, c->st));
+  if (d_total_valid)  // the mean runs over the valid slots of every rank's batch
+    KL(PC_OTHER, 8.0, launch_override_inv_n(d_total_valid, inv_n, c->st));
   // embeddings, then the frozen prefix: forward only, two buffers, nothing kept but the output
   KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_embed_ln(c->bf, d_tokens, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
                      Wv(c, toff(c, -1, "emb.ln.gamma")), Wv(c, toff(c, -1, "emb.ln.beta")), w.xa,
@@ -803,6 +848,7 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   KL(PC_OTHER, 4.0 * R, launch_loss_reduce(w.nll, R, inv_n, loss, c->st));
   TRY(zero_trainable_grads(c));
   TRY(head_backward(c, B, S, P, full));
+  TRY(bucket_done(c, 0));
   mark(c, 3);
   char* dx = w.dxa;
   char* dx_other = w.dxb;
@@ -811,14 +857,46 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
     const bool need_dx = l > first || full;
     TRY(layer_backward(c, l, x_in, w.layer[l - first], dx, dx_other, need_dx, B, S));
     if (need_dx) std::swap(dx, dx_other);
+    TRY(bucket_done(c, c->L - l));
   }
   if (full) {
     KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, dx, w.z0, w.st0, Wv(c, toff(c, -1, "emb.ln.gamma")), w.dz2,
                      G(c, toff(c, -1, "emb.ln.gamma")), G(c, toff(c, -1, "emb.ln.beta")), nullptr, T, H, c->st));
     KL(PC_OTHER, 1.0 * T * H * c->esz, launch_embed_scatter(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
                             G(c, toff(c, -1, "emb.pos")), T, S, H, V, c->st));
+    TRY(bucket_done(c, c->top_k + 1));
   }
   mark(c, 4);
+  if (defer_update) {
+    c->pending_update = true;
+    return finish(c, loss_out);
+  }
+  TRY(apply_update(c));
+  mark(c, 5);
+  if (c->timing && c->have_events) {
+    CUDA_TRY(cudaEventSynchronize(c->ev[5]));
+    for (int i = 0; i < 5; i++) cudaEventElapsedTime(&c->phase_ms[i], c->ev[i], c->ev[i + 1]);
+  }
+  if (c->profile) {
+    CUDA_TRY(cudaStreamSynchronize(c->st));
+    for (size_t i = 0; i < c->prec.size(); i++) {
+      float ms = 0.f;
+      cudaEventElapsedTime(&ms, c->pev[2 * i], c->pev[2 * i + 1]);
+      double* a = c->prof[c->prec[i].cls];
+      a[0] += 1.0; a[1] += c->prec[i].flops; a[2] += ms;
+    }
+  }
+  return finish(c, loss_out);
+}
+
+// the optimizer on the trainable slice (Adam or LAMB), after any gradient exchange
+static int apply_update(mslt_ctx* c) {
+  Workspace& w = c->ws;
+  if (c->bucket_fn && c->comm) {  // the reductions enqueued on the communication stream come first
+    if (!c->comm_done) CUDA_TRY(cudaEventCreateWithFlags(&c->comm_done, cudaEventDisableTiming));
+    CUDA_TRY(cudaEventRecord(c->comm_done, c->comm));
+    CUDA_TRY(cudaStreamWaitEvent(c->st, c->comm_done, 0));
+  }
   c->t_step += 1;
   AdamHyper h;
   h.lr = c->opt.lr; h.beta1 = c->opt.beta1; h.beta2 = c->opt.beta2; h.eps = c->opt.eps;
@@ -835,21 +913,49 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
                    (float*)(w.scalars + 5), c->opt.bias_correction, c->st));
     c->launches++;  // step-count kernel and update kernel
   }
-  mark(c, 5);
-  if (c->timing && c->have_events) {
-    CUDA_TRY(cudaEventSynchronize(c->ev[5]));
-    for (int i = 0; i < 5; i++) cudaEventElapsedTime(&c->phase_ms[i], c->ev[i], c->ev[i + 1]);
-  }
-  if (c->profile) {
-    CUDA_TRY(cudaStreamSynchronize(c->st));
-    for (size_t i = 0; i < c->prec.size(); i++) {
-      float ms = 0.f;
-      cudaEventElapsedTime(&ms, c->pev[2 * i], c->pev[2 * i + 1]);
-      double* a = c->prof[c->prec[i].cls];
-      a[0] += 1.0; a[1] += c->prec[i].flops; a[2] += ms;
-    }
-  }
-  return finish(c, loss_out);
+  return 0;
+}
+
+int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
+              const int32_t* d_pos, const int32_t* d_lab, int32_t B, int32_t S, int32_t P,
+              float* loss_out) {
+  return step_impl(c, d_tokens, d_seq_lens, d_pos, d_lab, B, S, P, nullptr, false, loss_out);
+}
+
+int mslt_step_backward(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
+                       const int32_t* d_pos, const int32_t* d_lab, int32_t B, int32_t S, int32_t P,
+                       const int32_t* d_total_valid, float* loss_out) {
+  return step_impl(c, d_tokens, d_seq_lens, d_pos, d_lab, B, S, P, d_total_valid, true, loss_out);
+}
+
+int mslt_step_apply(mslt_ctx* c) {
+  if (!c) return fail(MSLT_ERR_ARG, "null context");
+  if (!c->pending_update) return fail(MSLT_ERR_STATE, "mslt_step_apply without a preceding mslt_step_backward");
+  c->pending_update = false;
+  TRY(apply_update(c));
+  CUDA_TRY(cudaGetLastError());
+  return 0;
+}
+
+int mslt_num_grad_buckets(const mslt_ctx* c) { return c ? num_buckets(c) : MSLT_ERR_ARG; }
+
+int mslt_grad_bucket(mslt_ctx* c, int32_t i, float** d_ptr, int64_t* count) {
+  if (!c || !d_ptr || !count) return fail(MSLT_ERR_ARG, "null pointer");
+  if (i < 0 || i >= num_buckets(c)) return fail(MSLT_ERR_ARG, "no such gradient bucket");
+  int64_t off, cnt;
+  bucket_range(c, i, &off, &cnt);
+  *d_ptr = c->grad + off;
+  *count = cnt;
+  return 0;
+}
+
+int mslt_set_bucket_hook(mslt_ctx* c, void* comm_stream, mslt_bucket_fn fn, void* user) {
+  if (!c) return fail(MSLT_ERR_ARG, "null context");
+  if (fn && !comm_stream) return fail(MSLT_ERR_ARG, "a hook needs a communication stream");
+  c->comm = (cudaStream_t)comm_stream;
+  c->bucket_fn = fn;
+  c->bucket_user = user;
+  return 0;
 }
 
 int mslt_read_loss(mslt_ctx* c, float* loss_out) {
