@@ -172,11 +172,15 @@ class MsltOracle:
     """BERT stack with a frozen/trainable boundary, in float64."""
 
     def __init__(self, params: Dict[str, np.ndarray], heads: int, ln_eps: float = 1e-12,
-                 max_layers: Optional[int] = None):
+                 max_layers: Optional[int] = None, share_group: int = 1):
+        """share_group = g > 1: the grouped parameter sharing of Section 3.3 (the paper's change to
+        ALBERT): encoder layers l with the same l // g use one parameter block, named
+        "layer.<l // g>."; a stage adds one or more whole groups and only those train."""
         self.p: Dict[str, np.ndarray] = {k: np.array(v, dtype=F64) for k, v in params.items()}
         self.heads = heads
         self.eps = ln_eps
-        self.L = 1 + max(int(k.split(".")[1]) for k in self.p if k.startswith("layer."))
+        self.g = int(share_group)
+        self.L = self.g * (1 + max(int(k.split(".")[1]) for k in self.p if k.startswith("layer.")))
         self.max_layers = self.L if max_layers is None else max_layers
         self.H = self.p["emb.word"].shape[1]
         self.V = self.p["emb.word"].shape[0]
@@ -191,8 +195,8 @@ class MsltOracle:
         names: List[str] = []
         if self.top_k == self.L:
             names += list(EMB_TENSORS)
-        for l in range(self.L - self.top_k, self.L):
-            names += [f"layer.{l}.{t}" for t in LAYER_TENSORS]
+        for b in range((self.L - self.top_k) // self.g, self.L // self.g):
+            names += [f"layer.{b}.{t}" for t in LAYER_TENSORS]
         names += list(HEAD_TENSORS)
         return names
 
@@ -205,18 +209,18 @@ class MsltOracle:
         self.opt.update(kw)
 
     def set_trainable(self, top_k: int):
-        if not 0 <= top_k <= self.L:
-            raise ValueError("top_k out of range")
+        if not 0 <= top_k <= self.L or top_k % self.g:
+            raise ValueError("top_k out of range, or not a whole number of groups")
         self.top_k = top_k
         self._reset_optimizer()
 
     def add_layers(self, k: int):
         """New layer L+i is a copy of layer L-k+i (order preserved)."""
-        if not 1 <= k <= self.L or self.L + k > self.max_layers:
+        if not 1 <= k <= self.L or self.L + k > self.max_layers or k % self.g:
             raise ValueError("cannot add layers")
-        for i in range(k):
+        for i in range(k // self.g):
             for t in LAYER_TENSORS:
-                self.p[f"layer.{self.L + i}.{t}"] = self.p[f"layer.{self.L - k + i}.{t}"].copy()
+                self.p[f"layer.{self.L // self.g + i}.{t}"] = self.p[f"layer.{(self.L - k) // self.g + i}.{t}"].copy()
         self.L += k
         self.top_k = min(self.top_k, self.L)
         self._reset_optimizer()
@@ -229,7 +233,7 @@ class MsltOracle:
         return y, (xhat, rstd)
 
     def _layer_forward(self, l: int, x, seq_lens):
-        P = lambda t: self.p[f"layer.{l}.{t}"]
+        P = lambda t: self.p[f"layer.{l // self.g}.{t}"]
         B, S, H = x.shape
         A, d = self.heads, H // self.heads
         qkv = x @ P("qkv.weight").T + P("qkv.bias")                 # [B,S,3H]
@@ -327,22 +331,25 @@ class MsltOracle:
                     dx[b, hs["pos"][b, j]] += dhm[b, j]
 
         # trainable encoder layers, top-down; stop at the frozen boundary
+        def acc(name, value):          # layers of one group add their gradients into the shared block
+            g[name] = g[name] + value if name in g else value
+
         for l in range(self.L - 1, first - 1, -1):
-            P = lambda t: self.p[f"layer.{l}.{t}"]
+            P = lambda t: self.p[f"layer.{l // self.g}.{t}"]
             s = st[l]
-            n = f"layer.{l}."
-            dz2, g[n + "ln2.gamma"], g[n + "ln2.beta"] = layer_norm_backward(
-                dx, s["xh2"], s["rs2"], P("ln2.gamma"))
-            g[n + "ffn2.weight"] = np.einsum("bso,bsi->oi", dz2, s["g"])
-            g[n + "ffn2.bias"] = dz2.sum(axis=(0, 1))
+            n = f"layer.{l // self.g}."
+            dz2, dgam, dbet = layer_norm_backward(dx, s["xh2"], s["rs2"], P("ln2.gamma"))
+            acc(n + "ln2.gamma", dgam); acc(n + "ln2.beta", dbet)
+            acc(n + "ffn2.weight", np.einsum("bso,bsi->oi", dz2, s["g"]))
+            acc(n + "ffn2.bias", dz2.sum(axis=(0, 1)))
             du = (dz2 @ P("ffn2.weight")) * gelu_grad(s["u"])
-            g[n + "ffn1.weight"] = np.einsum("bso,bsi->oi", du, s["y"])
-            g[n + "ffn1.bias"] = du.sum(axis=(0, 1))
+            acc(n + "ffn1.weight", np.einsum("bso,bsi->oi", du, s["y"]))
+            acc(n + "ffn1.bias", du.sum(axis=(0, 1)))
             dy = du @ P("ffn1.weight") + dz2
-            dz1, g[n + "ln1.gamma"], g[n + "ln1.beta"] = layer_norm_backward(
-                dy, s["xh1"], s["rs1"], P("ln1.gamma"))
-            g[n + "out.weight"] = np.einsum("bso,bsi->oi", dz1, s["c"])
-            g[n + "out.bias"] = dz1.sum(axis=(0, 1))
+            dz1, dgam, dbet = layer_norm_backward(dy, s["xh1"], s["rs1"], P("ln1.gamma"))
+            acc(n + "ln1.gamma", dgam); acc(n + "ln1.beta", dbet)
+            acc(n + "out.weight", np.einsum("bso,bsi->oi", dz1, s["c"]))
+            acc(n + "out.bias", dz1.sum(axis=(0, 1)))
             dc = (dz1 @ P("out.weight")).reshape(B, S, A, d).transpose(0, 2, 1, 3)   # [B,A,S,d]
             dv = np.einsum("bhij,bhid->bhjd", s["p"], dc)
             dp = np.einsum("bhid,bhjd->bhij", dc, s["v"])
@@ -351,8 +358,8 @@ class MsltOracle:
             dk = np.einsum("bhij,bhid->bhjd", dsc, s["q"])
             dqkv = np.concatenate([t.transpose(0, 2, 1, 3).reshape(B, S, H) for t in (dq, dk, dv)],
                                   axis=-1)
-            g[n + "qkv.weight"] = np.einsum("bso,bsi->oi", dqkv, s["x"])
-            g[n + "qkv.bias"] = dqkv.sum(axis=(0, 1))
+            acc(n + "qkv.weight", np.einsum("bso,bsi->oi", dqkv, s["x"]))
+            acc(n + "qkv.bias", dqkv.sum(axis=(0, 1)))
             if l > first or full:
                 dx = dqkv @ P("qkv.weight") + dz1
 

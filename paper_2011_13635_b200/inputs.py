@@ -41,6 +41,7 @@ class StageConfig:
     dtype: str           # "fp32" or "bf16"
     varlen: Tuple[int, int] | None = None   # (lo, hi) inclusive, None = all S
     seed_index: int = 0
+    share_group: int = 1  # layers per shared parameter block (Section 3.3); 1 = every layer its own
 
     @property
     def frozen(self) -> int:
@@ -122,7 +123,7 @@ def param_shapes(cfg: StageConfig, n_layers: int | None = None) -> Dict[str, Tup
         "emb.word": (V, H), "emb.pos": (cfg.max_pos, H),
         "emb.ln.gamma": (H,), "emb.ln.beta": (H,),
     }
-    for i in range(L):
+    for i in range(L // cfg.share_group):   # one parameter block per group of layers
         p = f"layer.{i}."
         d[p + "qkv.weight"] = (3 * H, H)
         d[p + "qkv.bias"] = (3 * H,)

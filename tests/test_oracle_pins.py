@@ -553,3 +553,85 @@ def test_step_with_lamb_updates_every_trainable_tensor_by_its_own_norm():
             assert abs(np.linalg.norm(m.p[k] - before[k]) - lr * np.linalg.norm(before[k])) < 1e-12, k
         else:
             assert np.array_equal(m.p[k], before[k]), k
+
+
+# -- grouped parameter sharing (Section 3.3: the paper's change to ALBERT) ------------------------------
+
+SHARED = I.scaled(TINY, layers=4, trainable=2, share_group=2, seed_index=78)
+
+
+def _unshared_twin(m):
+    """The same network with every layer given its own copy of its group's block."""
+    w = {k: v.copy() for k, v in m.p.items() if not k.startswith("layer.")}
+    for l in range(m.L):
+        for t in O.LAYER_TENSORS:
+            w[f"layer.{l}.{t}"] = m.p[f"layer.{l // m.g}.{t}"].copy()
+    return O.MsltOracle(w, m.heads, ln_eps=m.eps)
+
+
+@pytest.mark.parametrize("top_k", [2, 4])
+def test_shared_group_gradient_is_the_sum_over_its_layers(top_k):
+    w = I.make_weights(SHARED, seed=5, variant="parity", std=0.3)
+    assert "layer.1.qkv.weight" in w and "layer.2.qkv.weight" not in w      # two blocks for four layers
+    m = O.MsltOracle(w, SHARED.heads, share_group=2)
+    assert m.L == 4
+    m.set_trainable(top_k)
+    tok, lens, pos, lab = tiny_batch(SHARED)
+    twin = _unshared_twin(m)
+    twin.set_trainable(top_k)
+    # same function of the same numbers ...
+    h, _ = m.forward(tok, lens)
+    h2, _ = twin.forward(tok, lens)
+    assert np.array_equal(h, h2)
+    loss, g = m.loss_and_grads(tok, lens, pos, lab)
+    loss2, g2 = twin.loss_and_grads(tok, lens, pos, lab)
+    assert loss == loss2
+    # ... and the gradient of a shared block is the sum of the gradients its layers would get alone
+    assert set(g) == set(m.trainable_names())
+    for b in range((4 - top_k) // 2, 2):
+        for t in O.LAYER_TENSORS:
+            np.testing.assert_allclose(g[f"layer.{b}.{t}"], g2[f"layer.{2 * b}.{t}"] + g2[f"layer.{2 * b + 1}.{t}"],
+                                       rtol=0, atol=1e-13)
+    for n in O.HEAD_TENSORS:
+        np.testing.assert_allclose(g[n], g2[n], rtol=0, atol=1e-14)
+
+
+def test_shared_group_gradients_match_finite_differences():
+    w = I.make_weights(SHARED, seed=5, variant="parity", std=0.3)
+    m = O.MsltOracle(w, SHARED.heads, share_group=2)
+    m.set_trainable(2)
+    tok, lens, pos, lab = tiny_batch(SHARED)
+    _, g = m.loss_and_grads(tok, lens, pos, lab)
+    h = 1e-5
+    for name in ("layer.1.qkv.weight", "layer.1.ln1.gamma", "layer.1.ffn2.bias", "layer.1.out.weight"):
+        wt = m.p[name]
+        fd = np.zeros_like(wt)
+        it = np.nditer(wt, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = wt[idx]
+            wt[idx] = keep + h; lp = m.loss(tok, lens, pos, lab)
+            wt[idx] = keep - h; lm = m.loss(tok, lens, pos, lab)
+            wt[idx] = keep
+            fd[idx] = (lp - lm) / (2 * h)
+        assert np.abs(fd - g[name]).max() / max(np.abs(fd).max(), 1e-8) < 1e-6, name
+
+
+def test_shared_groups_stack_and_train_by_whole_groups():
+    cfg = I.scaled(SHARED, layers=2)
+    w = I.make_weights(cfg, seed=5, variant="parity", std=0.3)
+    m = O.MsltOracle(w, cfg.heads, max_layers=4, share_group=2)
+    assert m.L == 2 and m.trainable_names().count("layer.0.qkv.weight") == 1
+    with pytest.raises(ValueError):
+        m.add_layers(1)                       # half a group
+    with pytest.raises(ValueError):
+        m.set_trainable(1)
+    m.add_layers(2)                           # the new group starts as a copy of the top group
+    assert m.L == 4 and np.array_equal(m.p["layer.1.ffn1.weight"], m.p["layer.0.ffn1.weight"])
+    m.set_trainable(2)
+    assert "layer.1.ffn1.weight" in m.trainable_names() and "layer.0.ffn1.weight" not in m.trainable_names()
+    before = {k: v.copy() for k, v in m.p.items()}
+    m.step(*tiny_batch(SHARED))
+    for k in before:                          # only the new group and the output layer move
+        moved = not np.array_equal(before[k], m.p[k])
+        assert moved == (k.startswith("layer.1.") or k.startswith("head.")), k
