@@ -65,6 +65,11 @@ typedef struct {
                        /* trainable layers keep their activations for the backward pass (Section    */
                        /* 3.2: the bottom layers run forward only), so the workspace holds this many  */
                        /* saved-activation slots: BERT-Base 9 + 3 needs 3 of them, not 12             */
+  int32_t share_group; /* grouped parameter sharing (Section 3.3, the paper's change to ALBERT): encoder  */
+                       /* layers l with the same l / share_group use ONE parameter block, their weight   */
+                       /* gradients add up, and stages add and train whole groups.  0 or 1: every layer  */
+                       /* has its own parameters.  init_layers, max_layers and every k / top_k below     */
+                       /* must be multiples of it; tensors are named by block: "layer.<block>.<name>"    */
 } mslt_arch;
 
 /*

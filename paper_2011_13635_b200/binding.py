@@ -26,7 +26,8 @@ class Arch(C.Structure):
     _fields_ = [("hidden", C.c_int32), ("heads", C.c_int32), ("ffn", C.c_int32), ("vocab", C.c_int32),
                 ("max_pos", C.c_int32), ("init_layers", C.c_int32), ("max_layers", C.c_int32),
                 ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("max_pred", C.c_int32),
-                ("dtype", C.c_int32), ("ln_eps", C.c_float), ("max_trainable", C.c_int32)]
+                ("dtype", C.c_int32), ("ln_eps", C.c_float), ("max_trainable", C.c_int32),
+                ("share_group", C.c_int32)]
 
 
 class Opt(C.Structure):
@@ -229,14 +230,14 @@ class Mslt:
 
     def __init__(self, *, hidden, heads, ffn, vocab, max_pos, init_layers, max_layers, max_batch,
                  max_seq, max_pred, dtype: str, ln_eps: float = 1e-12, max_trainable: int = 0,
-                 device="cuda:0", stream=None):
+                 share_group: int = 1, device="cuda:0", stream=None):
         import torch
         self.torch = torch
         if not torch.cuda.is_available():
             raise MsltError(-4, "no CUDA device: this library has no CPU path")
         self.device = torch.device(device)
         self.arch = Arch(hidden, heads, ffn, vocab, max_pos, init_layers, max_layers, max_batch,
-                         max_seq, max_pred, {"fp32": 0, "bf16": 1}[dtype], ln_eps, max_trainable)
+                         max_seq, max_pred, {"fp32": 0, "bf16": 1}[dtype], ln_eps, max_trainable, share_group)
         self.dtype = dtype
         pb, wb = mslt_query_bytes(self.arch)
         with torch.cuda.device(self.device):
@@ -254,7 +255,8 @@ class Mslt:
         return cls(hidden=cfg.hidden, heads=cfg.heads, ffn=cfg.ffn, vocab=cfg.vocab,
                    max_pos=cfg.max_pos, init_layers=cfg.layers if init_layers is None else init_layers,
                    max_layers=cfg.layers if max_layers is None else max_layers,
-                   max_batch=cfg.batch, max_seq=cfg.seq, max_pred=cfg.pred, dtype=cfg.dtype, **kw)
+                   max_batch=cfg.batch, max_seq=cfg.seq, max_pred=cfg.pred, dtype=cfg.dtype,
+                   share_group=getattr(cfg, "share_group", 1), **kw)
 
     def close(self):
         if getattr(self, "h", None):

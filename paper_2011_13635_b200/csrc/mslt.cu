@@ -57,7 +57,7 @@ struct Tensor {
   int64_t count;   // elements
   int64_t padded;  // elements reserved (multiple of 64)
   int64_t offset;  // element offset in every arena
-  int layer;       // >= 0 encoder layer, -1 embeddings, -2 head
+  int layer;       // >= 0 parameter block of encoder layers (= layer index without sharing), -1 embeddings, -2 head
 };
 
 // Saved activations of one encoder layer (also the scratch of a frozen layer).
@@ -152,8 +152,15 @@ int check_arch(const mslt_arch* a) {
   if (!(a->ln_eps >= 0.f)) return fail(MSLT_ERR_ARG, "ln_eps must be >= 0");
   if (a->max_trainable < 0 || a->max_trainable > a->max_layers)
     return fail(MSLT_ERR_ARG, "need 0 <= max_trainable <= max_layers");
+  if (a->share_group < 0) return fail(MSLT_ERR_ARG, "share_group must be >= 0");
+  if (a->share_group > 1 && (a->init_layers % a->share_group || a->max_layers % a->share_group ||
+                             a->max_trainable % a->share_group))
+    return fail(MSLT_ERR_ARG, "init_layers, max_layers and max_trainable must be multiples of share_group");
   return 0;
 }
+
+// layers per shared parameter block (Section 3.3); layer l reads block l / group
+int group_of(const mslt_arch& a) { return a.share_group > 1 ? a.share_group : 1; }
 
 void build_tensor_table(const mslt_arch& a, std::vector<Tensor>& out, int64_t& total) {
   const int64_t H = a.hidden, F = a.ffn, V = a.vocab;
@@ -171,7 +178,7 @@ void build_tensor_table(const mslt_arch& a, std::vector<Tensor>& out, int64_t& t
   add("emb.pos", 2, a.max_pos, H, -1);
   add("emb.ln.gamma", 1, H, 0, -1);
   add("emb.ln.beta", 1, H, 0, -1);
-  for (int l = 0; l < a.max_layers; l++) {
+  for (int l = 0; l < a.max_layers / group_of(a); l++) {  // one block per group of layers
     const std::string p = "layer." + std::to_string(l) + ".";
     const int64_t rows[12] = {3 * H, H, F, H, 3 * H, H, H, H, F, H, H, H};
     const int64_t cols[4] = {H, H, H, F};
@@ -253,18 +260,19 @@ const Tensor* find(const mslt_ctx* c, const char* name) {
   auto it = c->by_name.find(name);
   if (it == c->by_name.end()) return nullptr;
   const Tensor* t = &c->tensors[it->second];
-  if (t->layer >= c->L) return nullptr;
+  if (t->layer >= c->L / group_of(c->a)) return nullptr;
   return t;
 }
 bool is_trainable(const mslt_ctx* c, const Tensor& t) {
   if (t.layer == -2) return true;
   if (t.layer == -1) return c->top_k == c->L;
-  return t.layer >= c->L - c->top_k && t.layer < c->L;
+  const int g = group_of(c->a);
+  return t.layer >= (c->L - c->top_k) / g && t.layer < c->L / g;
 }
 int64_t toff(const mslt_ctx* c, int layer, const char* n) {
   if (layer >= 0) {
     for (int i = 0; i < 12; i++)
-      if (strcmp(n, kLayerNames[i]) == 0) return c->tensors[4 + 12 * layer + i].offset;
+      if (strcmp(n, kLayerNames[i]) == 0) return c->tensors[4 + 12 * (layer / group_of(c->a)) + i].offset;
   }
   return c->tensors[c->by_name.at(n)].offset;
 }
@@ -279,7 +287,7 @@ int rebuild_chunks(mslt_ctx* c) {
   std::vector<AdamChunk> h;
   for (size_t ti = 0; ti < c->tensors.size(); ti++) {
     const Tensor& t = c->tensors[ti];
-    if (t.layer >= c->L || !is_trainable(c, t)) continue;
+    if (t.layer >= c->L / group_of(c->a) || !is_trainable(c, t)) continue;
     for (int64_t o = 0; o < t.padded; o += kAdamChunk) {
       AdamChunk ch;
       ch.offset = t.offset + o;
@@ -612,8 +620,8 @@ int zero_trainable_grads(mslt_ctx* c) {
   const int first = c->L - c->top_k;
   if (c->top_k == c->L) CUDA_TRY(cudaMemsetAsync(c->grad + c->emb_off, 0, c->emb_cnt * 4, c->st));
   if (c->top_k > 0)
-    CUDA_TRY(cudaMemsetAsync(c->grad + c->layer0_off + (int64_t)first * c->layer_cnt, 0,
-                             (size_t)c->top_k * c->layer_cnt * 4, c->st));
+    CUDA_TRY(cudaMemsetAsync(c->grad + c->layer0_off + (int64_t)(first / group_of(c->a)) * c->layer_cnt, 0,
+                             (size_t)(c->top_k / group_of(c->a)) * c->layer_cnt * 4, c->st));
   CUDA_TRY(cudaMemsetAsync(c->grad + c->head_off, 0, c->head_cnt * 4, c->st));
   return 0;
 }
@@ -621,10 +629,13 @@ int zero_trainable_grads(mslt_ctx* c) {
 // Gradient buckets in the order in which a step completes them: the output layer, the trainable
 // layers from the top down, then (only when everything trains) the embeddings.  Each is one contiguous
 // range of the fp32 gradient arena.
-int num_buckets(const mslt_ctx* c) { return 1 + c->top_k + (c->top_k == c->L ? 1 : 0); }
+int num_buckets(const mslt_ctx* c) { return 1 + c->top_k / group_of(c->a) + (c->top_k == c->L ? 1 : 0); }
 void bucket_range(const mslt_ctx* c, int i, int64_t* off, int64_t* cnt) {
   if (i == 0) { *off = c->head_off; *cnt = c->head_cnt; }
-  else if (i <= c->top_k) { *off = c->layer0_off + (int64_t)(c->L - i) * c->layer_cnt; *cnt = c->layer_cnt; }
+  else if (i <= c->top_k / group_of(c->a)) {  // parameter blocks from the top down
+    *off = c->layer0_off + (int64_t)(c->L / group_of(c->a) - i) * c->layer_cnt;
+    *cnt = c->layer_cnt;
+  }
   else { *off = c->emb_off; *cnt = c->emb_cnt; }
 }
 int bucket_done(mslt_ctx* c, int i) {
@@ -734,7 +745,7 @@ int mslt_create(const mslt_arch* arch, void* dev_params, size_t param_bytes, voi
   c->layer0_off = c->tensors[c->by_name.at("layer.0.qkv.weight")].offset;
   c->emb_cnt = c->layer0_off;
   c->head_off = c->tensors[c->by_name.at("head.transform.weight")].offset;
-  c->layer_cnt = (c->head_off - c->layer0_off) / arch->max_layers;
+  c->layer_cnt = (c->head_off - c->layer0_off) / (arch->max_layers / group_of(*arch));
   c->head_cnt = c->n_elems - c->head_off;
   cudaError_t e = cudaMemsetAsync(dev_params, 0, param_bytes_for(*arch, c->n_elems), c->st);
   if (e == cudaSuccess) e = cudaMemsetAsync(dev_workspace, 0, c->ws.bytes, c->st);
@@ -762,12 +773,15 @@ int mslt_destroy(mslt_ctx* c) {
 
 int mslt_add_layers(mslt_ctx* c, int32_t k) {
   if (!c) return fail(MSLT_ERR_ARG, "null context");
+  const int g = group_of(c->a);
+  if (c->pending_update) return fail(MSLT_ERR_STATE, "add_layers: a step is waiting for mslt_step_apply");
   if (k < 1 || k > c->L) return fail(MSLT_ERR_STATE, "add_layers: need 1 <= k <= L (k=%d, L=%d)", k, c->L);
+  if (k % g) return fail(MSLT_ERR_STATE, "add_layers: k = %d is not a whole number of shared groups of %d layers", k, g);
   if (c->L + k > c->a.max_layers)
     return fail(MSLT_ERR_STATE, "add_layers: L + k = %d exceeds max_layers = %d", c->L + k, c->a.max_layers);
-  const int64_t src = c->layer0_off + (int64_t)(c->L - k) * c->layer_cnt;
-  const int64_t dst = c->layer0_off + (int64_t)c->L * c->layer_cnt;
-  const int64_t n = (int64_t)k * c->layer_cnt;
+  const int64_t src = c->layer0_off + (int64_t)((c->L - k) / g) * c->layer_cnt;
+  const int64_t dst = c->layer0_off + (int64_t)(c->L / g) * c->layer_cnt;
+  const int64_t n = (int64_t)(k / g) * c->layer_cnt;
   CUDA_TRY(cudaMemcpyAsync(c->master + dst, c->master + src, n * 4, cudaMemcpyDeviceToDevice, c->st));
   if (c->bf)
     CUDA_TRY(cudaMemcpyAsync(c->wb + dst * 2, c->wb + src * 2, n * 2, cudaMemcpyDeviceToDevice, c->st));
@@ -779,6 +793,8 @@ int mslt_set_trainable(mslt_ctx* c, int32_t top_k) {
   if (!c) return fail(MSLT_ERR_ARG, "null context");
   if (c->pending_update) return fail(MSLT_ERR_STATE, "set_trainable: a step is waiting for mslt_step_apply");
   if (top_k < 0 || top_k > c->L) return fail(MSLT_ERR_STATE, "set_trainable: need 0 <= top_k <= L");
+  if (top_k % group_of(c->a))
+    return fail(MSLT_ERR_STATE, "set_trainable: top_k = %d is not a whole number of shared groups", top_k);
   if (top_k > trainable_slots(c->a))
     return fail(MSLT_ERR_SIZE, "set_trainable: top_k = %d exceeds max_trainable = %d, the number of saved-activation "
                 "slots the workspace was sized for", top_k, trainable_slots(c->a));
@@ -857,14 +873,15 @@ static int step_impl(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_
     const bool need_dx = l > first || full;
     TRY(layer_backward(c, l, x_in, w.layer[l - first], dx, dx_other, need_dx, B, S));
     if (need_dx) std::swap(dx, dx_other);
-    TRY(bucket_done(c, c->L - l));
+    if (l % group_of(c->a) == 0)  // the lowest layer of a parameter block completes its gradients
+      TRY(bucket_done(c, (c->L - l) / group_of(c->a)));
   }
   if (full) {
     KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, dx, w.z0, w.st0, Wv(c, toff(c, -1, "emb.ln.gamma")), w.dz2,
                      G(c, toff(c, -1, "emb.ln.gamma")), G(c, toff(c, -1, "emb.ln.beta")), nullptr, T, H, c->st));
     KL(PC_OTHER, 1.0 * T * H * c->esz, launch_embed_scatter(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
                             G(c, toff(c, -1, "emb.pos")), T, S, H, V, c->st));
-    TRY(bucket_done(c, c->top_k + 1));
+    TRY(bucket_done(c, c->top_k / group_of(c->a) + 1));
   }
   mark(c, 4);
   if (defer_update) {
@@ -1000,15 +1017,15 @@ int mslt_num_trainable(const mslt_ctx* c) { return c ? c->top_k : MSLT_ERR_ARG; 
 
 int mslt_num_tensors(const mslt_ctx* c) {
   if (!c) return MSLT_ERR_ARG;
-  return 4 + 12 * c->L + 5;
+  return 4 + 12 * (c->L / group_of(c->a)) + 5;
 }
 
 static const Tensor* tensor_by_index(const mslt_ctx* c, int i) {
-  const int n_layer_t = 12 * c->L;
+  const int n_layer_t = 12 * (c->L / group_of(c->a));
   if (i < 0) return nullptr;
   if (i < 4 + n_layer_t) return &c->tensors[i];
   i -= 4 + n_layer_t;
-  if (i < 5) return &c->tensors[4 + 12 * c->a.max_layers + i];
+  if (i < 5) return &c->tensors[4 + 12 * (c->a.max_layers / group_of(c->a)) + i];
   return nullptr;
 }
 

@@ -55,7 +55,8 @@ def build_pair(cfg: I.StageConfig, lr: float, max_layers=None, init_layers=None,
     from paper_2011_13635_b200.binding import Mslt
     L0 = cfg.layers if init_layers is None else init_layers
     w = I.make_weights(cfg, seed=seed, variant="parity", n_layers=L0)
-    oracle = O.MsltOracle(w, cfg.heads, ln_eps=1e-12, max_layers=max_layers or cfg.layers)
+    oracle = O.MsltOracle(w, cfg.heads, ln_eps=1e-12, max_layers=max_layers or cfg.layers,
+                          share_group=cfg.share_group)
     hyper = dict(I.ADAM_DEFAULTS)
     hyper.update(opt)
     hyper["lr"] = lr

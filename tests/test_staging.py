@@ -54,6 +54,41 @@ def test_schedule_of_stages_matches_oracle(cfg):
 
 
 @pytest.mark.parametrize("cfg", [CFG32, CFG16], ids=["fp32", "bf16"])
+def test_grouped_parameter_sharing_schedule_matches_oracle(cfg):
+    """Section 3.3: layers of a group share one parameter block; a stage adds a group and trains only
+    that group and the output layer; the shared block's gradient is the sum over its layers."""
+    from paper_2011_13635_b200 import binding as Bd
+    cfg = I.scaled(cfg, share_group=2)
+    lr = 1e-3 if cfg.dtype == "fp32" else 1e-4
+    tol = PT.TOL[cfg.dtype]
+    m, oracle = PT.build_pair(cfg, lr=lr, init_layers=2, max_layers=4)
+    assert m.num_layers == 2 and len([n for n in m.tensors() if n.startswith("layer.")]) == 12   # one block
+    seed = I.config_seed(cfg)
+    PT.compare_step(m, oracle, cfg, I.make_batch(cfg, seed=seed), tol)            # both layers feed block 0
+    with pytest.raises(Bd.MsltError) as ei:
+        m.mslt_add_layers(1)
+    assert ei.value.code == -3
+    m.mslt_add_layers(2)
+    oracle.add_layers(2)
+    assert m.num_layers == 4
+    assert np.array_equal(m.mslt_get_param("layer.1.ffn2.weight"), m.mslt_get_param("layer.0.ffn2.weight"))
+    with pytest.raises(Bd.MsltError) as ei:
+        m.mslt_set_trainable(1)
+    assert ei.value.code == -3
+    m.mslt_set_trainable(2)
+    oracle.set_trainable(2)
+    info = m.tensors()
+    assert info["layer.1.qkv.weight"]["trainable"] and not info["layer.0.qkv.weight"]["trainable"]
+    for s in (1, 2):
+        PT.compare_step(m, oracle, cfg, I.make_batch(cfg, seed=seed + s), tol)
+    assert len(m.grad_buckets()) == 2                                              # output layer + one group
+    m.mslt_set_trainable(4)
+    oracle.set_trainable(4)
+    PT.compare_step(m, oracle, cfg, I.make_batch(cfg, seed=seed + 3), tol)
+    m.close()
+
+
+@pytest.mark.parametrize("cfg", [CFG32, CFG16], ids=["fp32", "bf16"])
 def test_saved_activation_slots_only_for_the_trainable_layers(cfg):
     """A context sized for two trainable layers out of four: smaller workspace, same results, and a
     request for more trainable layers than it has slots for is refused."""
