@@ -166,6 +166,11 @@ LAYER_TENSORS = ("qkv.weight", "qkv.bias", "out.weight", "out.bias", "ln1.gamma"
 HEAD_TENSORS = ("head.transform.weight", "head.transform.bias", "head.ln.gamma", "head.ln.beta",
                 "head.decoder.bias")
 EMB_TENSORS = ("emb.word", "emb.pos", "emb.ln.gamma", "emb.ln.beta")
+# next-sentence-prediction objective (Section 4.1: "the same MLM and NSP objectives" as BERT): a
+# segment (token-type) table in the embeddings, a tanh pooler on the first token and a two-way
+# classifier.  Present only when the parameter set holds them.
+NSP_EMB_TENSORS = ("emb.type",)
+NSP_HEAD_TENSORS = ("head.pooler.weight", "head.pooler.bias", "head.nsp.weight", "head.nsp.bias")
 
 
 class MsltOracle:
@@ -184,6 +189,7 @@ class MsltOracle:
         self.max_layers = self.L if max_layers is None else max_layers
         self.H = self.p["emb.word"].shape[1]
         self.V = self.p["emb.word"].shape[0]
+        self.nsp = "head.nsp.weight" in self.p
         self.top_k = self.L
         self.opt = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01,
                         bias_correction=1, lamb=0)
@@ -194,10 +200,10 @@ class MsltOracle:
     def trainable_names(self) -> List[str]:
         names: List[str] = []
         if self.top_k == self.L:
-            names += list(EMB_TENSORS)
+            names += list(EMB_TENSORS) + (list(NSP_EMB_TENSORS) if self.nsp else [])
         for b in range((self.L - self.top_k) // self.g, self.L // self.g):
             names += [f"layer.{b}.{t}" for t in LAYER_TENSORS]
-        names += list(HEAD_TENSORS)
+        names += list(HEAD_TENSORS) + (list(NSP_HEAD_TENSORS) if self.nsp else [])
         return names
 
     def _reset_optimizer(self):
@@ -226,9 +232,12 @@ class MsltOracle:
         self._reset_optimizer()
 
     # -- forward ------------------------------------------------------------------
-    def _embed(self, tokens):
+    def _embed(self, tokens, segments=None):
         S = tokens.shape[1]
         z = self.p["emb.word"][tokens] + self.p["emb.pos"][:S][None, :, :]
+        if self.nsp:
+            seg = np.zeros_like(tokens) if segments is None else np.asarray(segments)
+            z = z + self.p["emb.type"][seg]
         y, xhat, rstd = layer_norm(z, self.p["emb.ln.gamma"], self.p["emb.ln.beta"], self.eps)
         return y, (xhat, rstd)
 
@@ -252,14 +261,14 @@ class MsltOracle:
                      xh2=xh2, rs2=rs2)
         return xo, stash
 
-    def encode(self, tokens, seq_lens=None, keep_from: Optional[int] = None):
+    def encode(self, tokens, seq_lens=None, keep_from: Optional[int] = None, segments=None):
         """Hidden states after the last layer, [B,S,H].  Frozen and trainable
         layers run the same forward function; stashes are kept only for layers
         >= keep_from."""
         tokens = np.asarray(tokens)
         B, S = tokens.shape
         seq_lens = np.full((B,), S) if seq_lens is None else np.asarray(seq_lens)
-        x, emb_stash = self._embed(tokens)
+        x, emb_stash = self._embed(tokens, segments)
         stashes = {}
         for l in range(self.L):
             x, st = self._layer_forward(l, x, seq_lens)
@@ -279,24 +288,39 @@ class MsltOracle:
         logits = tm @ self.p["emb.word"].T + self.p["head.decoder.bias"]
         return logits, dict(hm=hm, ut=ut, xh=xh, rs=rs, tm=tm, ok=ok.reshape(-1), pos=pos)
 
-    def forward(self, tokens, seq_lens=None, positions=None):
+    def _nsp_forward(self, x, nsp_labels):
+        """Pooler and two-way classifier on the first token of every sequence; mean cross-entropy
+        over the sequences whose label is >= 0."""
+        cls = x[:, 0, :]
+        up = cls @ self.p["head.pooler.weight"].T + self.p["head.pooler.bias"]
+        pooled = np.tanh(up)
+        logits = pooled @ self.p["head.nsp.weight"].T + self.p["head.nsp.bias"]      # [B,2]
+        lab = np.asarray(nsp_labels)
+        loss, dlogits = cross_entropy(logits, lab, int((lab >= 0).sum()))
+        return loss, dlogits, dict(cls=cls, pooled=pooled, logits=logits)
+
+    def forward(self, tokens, seq_lens=None, positions=None, segments=None):
         """(hidden [B,S,H], logits [B*P,V] or None): the inference-only path."""
-        x, _, _ = self.encode(tokens, seq_lens)
+        x, _, _ = self.encode(tokens, seq_lens, segments=segments)
         if positions is None:
             return x, None
         positions = np.asarray(positions)
         logits, _ = self._head_forward(x, positions, np.zeros_like(positions))
         return x, logits
 
-    def loss(self, tokens, seq_lens, positions, labels) -> float:
-        x, _, _ = self.encode(tokens, seq_lens)
+    def loss(self, tokens, seq_lens, positions, labels, segments=None, nsp_labels=None) -> float:
+        """MLM loss, plus the NSP loss when nsp_labels are given."""
+        x, _, _ = self.encode(tokens, seq_lens, segments=segments)
         positions, labels = np.asarray(positions), np.asarray(labels)
         logits, hs = self._head_forward(x, positions, labels)
         lab = np.where(hs["ok"], labels.reshape(-1), -1)
-        return cross_entropy(logits, lab, int(hs["ok"].sum()))[0]
+        total = cross_entropy(logits, lab, int(hs["ok"].sum()))[0]
+        if self.nsp and nsp_labels is not None:
+            total += self._nsp_forward(x, nsp_labels)[0]
+        return total
 
     # -- forward + backward, gradients for the trainable tensors only -------------------
-    def loss_and_grads(self, tokens, seq_lens, positions, labels):
+    def loss_and_grads(self, tokens, seq_lens, positions, labels, segments=None, nsp_labels=None):
         tokens = np.asarray(tokens)
         positions, labels = np.asarray(positions), np.asarray(labels)
         B, S = tokens.shape
@@ -305,7 +329,7 @@ class MsltOracle:
         seq_lens = np.full((B,), S) if seq_lens is None else np.asarray(seq_lens)
         first = self.L - self.top_k                       # first trainable layer
         full = self.top_k == self.L
-        x, emb_stash, st = self.encode(tokens, seq_lens, keep_from=first)
+        x, emb_stash, st = self.encode(tokens, seq_lens, keep_from=first, segments=segments)
         logits, hs = self._head_forward(x, positions, labels)
         lab = np.where(hs["ok"], labels.reshape(-1), -1)
         n_valid = int(hs["ok"].sum())
@@ -329,6 +353,22 @@ class MsltOracle:
             for j in range(positions.shape[1]):
                 if okm[b, j]:
                     dx[b, hs["pos"][b, j]] += dhm[b, j]
+
+        self.losses = dict(mlm=loss, nsp=0.0)
+        if self.nsp:
+            for n in NSP_HEAD_TENSORS:
+                g[n] = np.zeros_like(self.p[n])
+            if nsp_labels is not None:
+                # second objective: loss = MLM + NSP; its gradient enters the last hidden state at token 0
+                nsp_loss, dl2, ns = self._nsp_forward(x, nsp_labels)
+                loss = loss + nsp_loss
+                self.losses["nsp"] = nsp_loss
+                g["head.nsp.weight"] = dl2.T @ ns["pooled"]
+                g["head.nsp.bias"] = dl2.sum(axis=0)
+                dup = (dl2 @ self.p["head.nsp.weight"]) * (1.0 - ns["pooled"] ** 2)
+                g["head.pooler.weight"] = dup.T @ ns["cls"]
+                g["head.pooler.bias"] = dup.sum(axis=0)
+                dx[:, 0, :] += dup @ self.p["head.pooler.weight"]
 
         # trainable encoder layers, top-down; stop at the frozen boundary
         def acc(name, value):          # layers of one group add their gradients into the shared block
@@ -369,13 +409,17 @@ class MsltOracle:
             g["emb.pos"] = np.zeros_like(self.p["emb.pos"])
             g["emb.pos"][:S] = dz0.sum(axis=0)
             np.add.at(g["emb.word"], tokens.reshape(-1), dz0.reshape(B * S, H))
+            if self.nsp:
+                seg = np.zeros_like(tokens) if segments is None else np.asarray(segments)
+                g["emb.type"] = np.zeros_like(self.p["emb.type"])
+                np.add.at(g["emb.type"], seg.reshape(-1), dz0.reshape(B * S, H))
         self.grads = g
         return loss, g
 
     # -- one training step ------------------------------------------------------------
-    def step(self, tokens, seq_lens, positions, labels) -> float:
+    def step(self, tokens, seq_lens, positions, labels, segments=None, nsp_labels=None) -> float:
         """Forward, truncated backward, Adam (or LAMB, opt["lamb"] = 1) on the trainable tensors only."""
-        loss, g = self.loss_and_grads(tokens, seq_lens, positions, labels)
+        loss, g = self.loss_and_grads(tokens, seq_lens, positions, labels, segments, nsp_labels)
         self.t += 1
         o = self.opt
         update = lamb_update if o.get("lamb") else adam_update

@@ -42,6 +42,7 @@ class StageConfig:
     varlen: Tuple[int, int] | None = None   # (lo, hi) inclusive, None = all S
     seed_index: int = 0
     share_group: int = 1  # layers per shared parameter block (Section 3.3); 1 = every layer its own
+    nsp: bool = False     # next-sentence-prediction head and segment embeddings (Section 4.1)
 
     @property
     def frozen(self) -> int:
@@ -123,6 +124,8 @@ def param_shapes(cfg: StageConfig, n_layers: int | None = None) -> Dict[str, Tup
         "emb.word": (V, H), "emb.pos": (cfg.max_pos, H),
         "emb.ln.gamma": (H,), "emb.ln.beta": (H,),
     }
+    if cfg.nsp:
+        d["emb.type"] = (2, H)
     for i in range(L // cfg.share_group):   # one parameter block per group of layers
         p = f"layer.{i}."
         d[p + "qkv.weight"] = (3 * H, H)
@@ -142,7 +145,26 @@ def param_shapes(cfg: StageConfig, n_layers: int | None = None) -> Dict[str, Tup
     d["head.ln.gamma"] = (H,)
     d["head.ln.beta"] = (H,)
     d["head.decoder.bias"] = (V,)
+    if cfg.nsp:
+        d["head.pooler.weight"] = (H, H)
+        d["head.pooler.bias"] = (H,)
+        d["head.nsp.weight"] = (2, H)
+        d["head.nsp.bias"] = (2,)
     return d
+
+
+def make_nsp(cfg: StageConfig, seq_lens: np.ndarray, seed: int | None = None):
+    """segment ids [B,S] (0 up to a random split point inside the sequence, 1 after it, 0 on the
+    padding) and next-sentence labels [B] in {0, 1}; all int32."""
+    seed = config_seed(cfg) if seed is None else seed
+    r = _rng(seed, 4)
+    seg = np.zeros((cfg.batch, cfg.seq), dtype=np.int32)
+    for b in range(cfg.batch):
+        n = int(seq_lens[b])
+        cut = int(r.integers(1, max(2, n)))
+        seg[b, cut:n] = 1
+    lab = r.integers(0, 2, size=(cfg.batch,)).astype(np.int32)
+    return seg, lab
 
 
 def make_weights(cfg: StageConfig, seed: int | None = None, variant: str = "parity",

@@ -635,3 +635,78 @@ def test_shared_groups_stack_and_train_by_whole_groups():
     for k in before:                          # only the new group and the output layer move
         moved = not np.array_equal(before[k], m.p[k])
         assert moved == (k.startswith("layer.1.") or k.startswith("head.")), k
+
+
+# -- next-sentence prediction and segment embeddings (Section 4.1: "the same MLM and NSP objectives") ----
+
+NSP = I.scaled(TINY, nsp=True, seed_index=79)
+
+
+def _nsp_case(top_k):
+    w = I.make_weights(NSP, seed=5, variant="parity", std=0.3)
+    m = O.MsltOracle(w, NSP.heads)
+    m.set_trainable(top_k)
+    tok, lens, pos, lab = tiny_batch(NSP)
+    seg, nlab = I.make_nsp(NSP, lens, seed=9)
+    assert seg.max() == 1 and seg.min() == 0
+    return m, (tok, lens, pos, lab, seg, nlab)
+
+
+@pytest.mark.parametrize("top_k", [0, 1, 2])
+def test_nsp_gradients_match_finite_differences(top_k):
+    m, batch = _nsp_case(top_k)
+    assert m.nsp
+    loss, g = m.loss_and_grads(*batch)
+    names = m.trainable_names()
+    assert set(g) == set(names) and "head.nsp.weight" in names
+    assert ("emb.type" in names) == (top_k == 2)
+    assert abs(loss - (m.losses["mlm"] + m.losses["nsp"])) < 1e-14 and m.losses["nsp"] > 0
+    h = 1e-5
+    for name in names:
+        wt = m.p[name]
+        fd = np.zeros_like(wt)
+        it = np.nditer(wt, flags=["multi_index"])
+        for _ in it:
+            idx = it.multi_index
+            keep = wt[idx]
+            wt[idx] = keep + h; lp = m.loss(*batch)
+            wt[idx] = keep - h; lm = m.loss(*batch)
+            wt[idx] = keep
+            fd[idx] = (lp - lm) / (2 * h)
+        assert np.abs(fd - g[name]).max() / max(np.abs(fd).max(), 1e-8) < 1e-6, name
+        if name != "emb.pos":
+            assert np.abs(g[name]).max() > 0, name
+
+
+def test_nsp_head_matches_torch_functional_and_zero_classifier_gives_log_two():
+    m, (tok, lens, pos, lab, seg, nlab) = _nsp_case(1)
+    x, _, _ = m.encode(tok, lens, segments=seg)
+    F = torch.nn.functional
+    T = lambda n: torch.from_numpy(m.p[n])
+    pooled = torch.tanh(F.linear(torch.from_numpy(x[:, 0, :]), T("head.pooler.weight"), T("head.pooler.bias")))
+    want = F.cross_entropy(F.linear(pooled, T("head.nsp.weight"), T("head.nsp.bias")),
+                           torch.from_numpy(nlab.astype(np.int64))).item()
+    assert abs(m._nsp_forward(x, nlab)[0] - want) < 1e-12
+    # embeddings with segments against torch
+    e = F.embedding(torch.from_numpy(tok.astype(np.int64)), T("emb.word")) + T("emb.pos")[: tok.shape[1]]
+    e = e + F.embedding(torch.from_numpy(seg.astype(np.int64)), T("emb.type"))
+    want_e = F.layer_norm(e, (NSP.hidden,), T("emb.ln.gamma"), T("emb.ln.beta"), eps=1e-12).numpy()
+    np.testing.assert_allclose(m._embed(tok, seg)[0], want_e, atol=1e-12, rtol=0)
+    # a zero classifier cannot tell the two classes apart: loss ln 2 exactly
+    m.p["head.nsp.weight"][:] = 0.0; m.p["head.nsp.bias"][:] = 0.0
+    assert abs(m._nsp_forward(x, nlab)[0] - math.log(2.0)) < 1e-15
+    # ignored labels drop out of the mean
+    nl2 = nlab.copy(); nl2[0] = -1
+    m2, _ = _nsp_case(1)
+    full = m2._nsp_forward(x, nlab)[0]
+    part = m2._nsp_forward(x, nl2)[0]
+    one = m2._nsp_forward(x[1:], nlab[1:])[0]
+    assert abs(part - one) < 1e-14 and abs(full - part) > 1e-6
+
+
+def test_without_nsp_labels_the_nsp_parameters_get_zero_gradient_and_mlm_is_unchanged():
+    m, (tok, lens, pos, lab, seg, nlab) = _nsp_case(1)
+    loss, g = m.loss_and_grads(tok, lens, pos, lab, seg, None)
+    assert loss == m.losses["mlm"] and m.losses["nsp"] == 0.0
+    for n in O.NSP_HEAD_TENSORS:
+        assert not g[n].any()
