@@ -70,6 +70,11 @@ typedef struct {
                        /* gradients add up, and stages add and train whole groups.  0 or 1: every layer  */
                        /* has its own parameters.  init_layers, max_layers and every k / top_k below     */
                        /* must be multiples of it; tensors are named by block: "layer.<block>.<name>"    */
+  int32_t nsp;         /* 1: the network also has BERT's second objective (Section 4.1, "the same MLM    */
+                       /* and NSP objectives"): a segment table "emb.type" [2,H] added to the embeddings  */
+                       /* (trained with them), a tanh pooler "head.pooler.*" on the first token and a    */
+                       /* two-way classifier "head.nsp.*" (part of the output layer, always trained);    */
+                       /* see mslt_step_nsp.  0: MLM only, these tensors do not exist                    */
 } mslt_arch;
 
 /*
@@ -154,6 +159,22 @@ int mslt_set_optimizer(mslt_ctx* ctx, const mslt_opt* opt);
 int mslt_step(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens,
               const int32_t* d_mlm_positions, const int32_t* d_mlm_labels, int32_t B, int32_t S,
               int32_t P, float* loss_out);
+
+/*
+ * mslt_step with both BERT objectives (needs arch.nsp = 1): loss = MLM loss + NSP loss, where the
+ * NSP loss is the mean two-way cross-entropy, over the sequences whose label is 0 or 1, of the
+ * classifier on tanh(pooler(first token's final hidden state)).
+ *   d_segment_ids  device [B,S] values in {0, 1}, or NULL (all 0): row of "emb.type" added to every
+ *                  token's embedding before the embedding LayerNorm
+ *   d_nsp_labels   device [B] in {0, 1}, other values = sequence ignored; NULL = no NSP term at all
+ *                  (the NSP parameters then get zero gradients)
+ * Everything else as mslt_step, which on an nsp context runs with segment 0 everywhere and no NSP
+ * term.  loss_out receives the sum of the two losses.
+ */
+int mslt_step_nsp(mslt_ctx* ctx, const int32_t* d_tokens, const int32_t* d_seq_lens,
+                  const int32_t* d_segment_ids, const int32_t* d_mlm_positions,
+                  const int32_t* d_mlm_labels, const int32_t* d_nsp_labels, int32_t B, int32_t S,
+                  int32_t P, float* loss_out);
 
 /*
  * The same step in two halves, for data-parallel training (Section 3.1, last paragraph, and Section

@@ -27,7 +27,7 @@ class Arch(C.Structure):
                 ("max_pos", C.c_int32), ("init_layers", C.c_int32), ("max_layers", C.c_int32),
                 ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("max_pred", C.c_int32),
                 ("dtype", C.c_int32), ("ln_eps", C.c_float), ("max_trainable", C.c_int32),
-                ("share_group", C.c_int32)]
+                ("share_group", C.c_int32), ("nsp", C.c_int32)]
 
 
 class Opt(C.Structure):
@@ -49,7 +49,7 @@ class GemmDesc(C.Structure):
 
 
 EXPORTS = ["mslt_query_bytes", "mslt_create", "mslt_destroy", "mslt_add_layers", "mslt_set_trainable",
-           "mslt_set_optimizer", "mslt_step", "mslt_step_backward", "mslt_step_apply", "mslt_num_grad_buckets",
+           "mslt_set_optimizer", "mslt_step", "mslt_step_nsp", "mslt_step_backward", "mslt_step_apply", "mslt_num_grad_buckets",
            "mslt_grad_bucket", "mslt_set_bucket_hook", "mslt_read_loss", "mslt_forward", "mslt_num_layers",
            "mslt_num_trainable", "mslt_num_tensors", "mslt_tensor_info", "mslt_get_param",
            "mslt_set_param", "mslt_get_param_raw", "mslt_get_grad", "mslt_get_opt_state",
@@ -74,6 +74,8 @@ BUCKET_FN = C.CFUNCTYPE(None, C.c_void_p, C.c_int32)
 lib.mslt_step_backward.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_int32,
                                    C.c_int32, C.c_void_p, C.POINTER(C.c_float)]
 lib.mslt_step_apply.argtypes = [C.c_void_p]
+lib.mslt_step_nsp.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                              C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_float)]
 lib.mslt_num_grad_buckets.argtypes = [C.c_void_p]
 lib.mslt_grad_bucket.argtypes = [C.c_void_p, C.c_int32, C.POINTER(C.c_void_p), C.POINTER(C.c_int64)]
 lib.mslt_set_bucket_hook.argtypes = [C.c_void_p, C.c_void_p, BUCKET_FN, C.c_void_p]
@@ -230,14 +232,14 @@ class Mslt:
 
     def __init__(self, *, hidden, heads, ffn, vocab, max_pos, init_layers, max_layers, max_batch,
                  max_seq, max_pred, dtype: str, ln_eps: float = 1e-12, max_trainable: int = 0,
-                 share_group: int = 1, device="cuda:0", stream=None):
+                 share_group: int = 1, nsp: bool = False, device="cuda:0", stream=None):
         import torch
         self.torch = torch
         if not torch.cuda.is_available():
             raise MsltError(-4, "no CUDA device: this library has no CPU path")
         self.device = torch.device(device)
         self.arch = Arch(hidden, heads, ffn, vocab, max_pos, init_layers, max_layers, max_batch,
-                         max_seq, max_pred, {"fp32": 0, "bf16": 1}[dtype], ln_eps, max_trainable, share_group)
+                         max_seq, max_pred, {"fp32": 0, "bf16": 1}[dtype], ln_eps, max_trainable, share_group, int(bool(nsp)))
         self.dtype = dtype
         pb, wb = mslt_query_bytes(self.arch)
         with torch.cuda.device(self.device):
@@ -256,7 +258,7 @@ class Mslt:
                    max_pos=cfg.max_pos, init_layers=cfg.layers if init_layers is None else init_layers,
                    max_layers=cfg.layers if max_layers is None else max_layers,
                    max_batch=cfg.batch, max_seq=cfg.seq, max_pred=cfg.pred, dtype=cfg.dtype,
-                   share_group=getattr(cfg, "share_group", 1), **kw)
+                   share_group=getattr(cfg, "share_group", 1), nsp=getattr(cfg, "nsp", False), **kw)
 
     def close(self):
         if getattr(self, "h", None):
@@ -287,6 +289,15 @@ class Mslt:
         loss = C.c_float()
         _check(lib.mslt_step(self.h, tokens.data_ptr(), _ptr(seq_lens), mlm_positions.data_ptr(),
                              mlm_labels.data_ptr(), B, S, P, C.byref(loss) if sync else None))
+        return loss.value if sync else None
+
+    def mslt_step_nsp(self, tokens, seq_lens, segment_ids, mlm_positions, mlm_labels, nsp_labels, sync: bool = True):
+        """The step with both objectives; segment_ids [B,S] and nsp_labels [B] int32 CUDA tensors or None."""
+        B, S = tokens.shape
+        P = mlm_positions.shape[1]
+        loss = C.c_float()
+        _check(lib.mslt_step_nsp(self.h, tokens.data_ptr(), _ptr(seq_lens), _ptr(segment_ids), mlm_positions.data_ptr(),
+                                 mlm_labels.data_ptr(), _ptr(nsp_labels), B, S, P, C.byref(loss) if sync else None))
         return loss.value if sync else None
 
     def mslt_step_backward(self, tokens, seq_lens, mlm_positions, mlm_labels, total_valid=None, sync: bool = True):

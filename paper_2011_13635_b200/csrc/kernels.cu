@@ -180,8 +180,9 @@ ln_fwd_kernel(const T* __restrict__ z, const float* __restrict__ gamma, const fl
 // Embedding: z = word[token] + pos[s]; optional stash of z; then LayerNorm.
 template <typename T>
 __global__ void __launch_bounds__(256)
-embed_ln_kernel(const int* __restrict__ tokens, const T* __restrict__ word,
-                const T* __restrict__ pos, const float* __restrict__ gamma,
+embed_ln_kernel(const int* __restrict__ tokens, const int* __restrict__ segments,
+                const T* __restrict__ word, const T* __restrict__ pos, const T* __restrict__ type,
+                const float* __restrict__ gamma,
                 const float* __restrict__ beta, T* __restrict__ y, T* __restrict__ zstash,
                 float* __restrict__ stats, int rows, int S, int H, int V, float eps,
                 int* __restrict__ status) {
@@ -197,6 +198,16 @@ embed_ln_kernel(const int* __restrict__ tokens, const T* __restrict__ word,
   }
   const T* wr = word + (int64_t)tok * H;
   const T* pr = pos + (int64_t)(row % S) * H;
+  // segment (token-type) row: table of two rows; ids outside {0, 1} are reported and read as 0
+  const T* tr = nullptr;
+  if (type != nullptr) {
+    int sg = segments ? segments[row] : 0;
+    if (sg < 0 || sg > 1) {
+      if (lane == 0) atomicOr(status, ST_BAD_TOKEN);
+      sg = 0;
+    }
+    tr = type + (int64_t)sg * H;
+  }
   float x[LN_MAXE];
 #pragma unroll
   for (int i = 0; i < NV; i++) {
@@ -205,6 +216,12 @@ embed_ln_kernel(const int* __restrict__ tokens, const T* __restrict__ word,
       float a[VN], b[VN];
       VecT<T>::load(wr + c, a);
       VecT<T>::load(pr + c, b);
+      if (tr != nullptr) {
+        float t3[VN];
+        VecT<T>::load(tr + c, t3);
+#pragma unroll
+        for (int e = 0; e < VN; e++) b[e] += t3[e];
+      }
       // round the sum to the storage type first: the backward pass normalises the stashed copy
 #pragma unroll
       for (int e = 0; e < VN; e++) a[e] = to_f<T>(from_f<T>(a[e] + b[e]));
@@ -897,6 +914,100 @@ adam_kernel(const AdamChunk* __restrict__ chunks, float* __restrict__ w,
   }
 }
 
+// ---------------------------------------------------------------------------------------
+// Next-sentence-prediction head (the second BERT objective): per sequence b, on the pooled first
+// token, logits = Wn pooled + bn (two classes), nll = logsumexp - logit[label], mean over the
+// sequences with label >= 0.  One block per sequence; it also forms the gradients of Wn and bn
+// (atomics into the zeroed arena) and, fused with the tanh derivative of the pooler, the gradient
+// at the pooler's pre-activation: dup = (dlogit . Wn) * (1 - pooled^2).
+// ---------------------------------------------------------------------------------------
+__global__ void nsp_prepare_kernel(const int* __restrict__ labels, int B, int S, int* __restrict__ rowsrc,
+                                   float* __restrict__ inv_n, const int* __restrict__ total_valid) {
+  __shared__ int cnt;
+  if (threadIdx.x == 0) cnt = 0;
+  __syncthreads();
+  int local = 0;
+  for (int b = threadIdx.x; b < B; b += blockDim.x) {
+    rowsrc[b] = b * S;  // the first token of sequence b
+    local += (labels != nullptr && labels[b] >= 0 && labels[b] <= 1) ? 1 : 0;
+  }
+  if (local) atomicAdd(&cnt, local);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const int n = total_valid ? *total_valid : cnt;
+    *inv_n = n > 0 ? 1.0f / (float)n : 0.f;
+  }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(128)
+nsp_head_kernel(const T* __restrict__ pooled, const float* __restrict__ wn, const float* __restrict__ bn,
+                const int* __restrict__ labels, const float* __restrict__ inv_n, T* __restrict__ dup,
+                float* __restrict__ dwn, float* __restrict__ dbn, float* __restrict__ loss, int H) {
+  const int b = blockIdx.x;
+  const T* pr = pooled + (int64_t)b * H;
+  float s0 = 0.f, s1 = 0.f;
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    const float p = to_f<T>(pr[c]);
+    s0 += p * wn[c];
+    s1 += p * wn[H + c];
+  }
+  __shared__ float red[2][4];
+  s0 = warp_sum(s0);
+  s1 = warp_sum(s1);
+  if ((threadIdx.x & 31) == 0) { red[0][threadIdx.x >> 5] = s0; red[1][threadIdx.x >> 5] = s1; }
+  __syncthreads();
+  const float l0 = red[0][0] + red[0][1] + red[0][2] + red[0][3] + bn[0];
+  const float l1 = red[1][0] + red[1][1] + red[1][2] + red[1][3] + bn[1];
+  const int lab = labels ? labels[b] : -1;
+  const bool ok = lab == 0 || lab == 1;
+  const float mx = fmaxf(l0, l1);
+  const float e0 = expf(l0 - mx), e1 = expf(l1 - mx);
+  const float lse = mx + logf(e0 + e1);
+  const float scale = ok ? *inv_n : 0.f;
+  const float d0 = (e0 / (e0 + e1) - (lab == 0 ? 1.f : 0.f)) * scale;
+  const float d1 = (e1 / (e0 + e1) - (lab == 1 ? 1.f : 0.f)) * scale;
+  if (threadIdx.x == 0 && ok) {
+    atomicAdd(loss, (lse - (lab == 0 ? l0 : l1)) * scale);
+    atomicAdd(dbn, d0);
+    atomicAdd(dbn + 1, d1);
+  }
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    const float p = to_f<T>(pr[c]);
+    dup[(int64_t)b * H + c] = from_f<T>((d0 * wn[c] + d1 * wn[H + c]) * (1.f - p * p));
+    if (ok) {
+      atomicAdd(dwn + c, d0 * p);
+      atomicAdd(dwn + H + c, d1 * p);
+    }
+  }
+}
+
+// y = tanh(x), elementwise
+template <typename T>
+__global__ void tanh_kernel(const T* __restrict__ x, T* __restrict__ y, int64_t n) {
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+    y[i] = from_f<T>(tanhf(to_f<T>(x[i])));
+}
+
+// Gradient of the two-row segment table: dtype[seg[t], c] += dz[t, c].  A thread owns a column of a
+// block of rows and keeps one sum per segment, so the table sees two atomics per thread.
+template <typename T>
+__global__ void __launch_bounds__(128)
+type_grad_kernel(const T* __restrict__ dz, const int* __restrict__ segments, float* __restrict__ dtype,
+                 int rows, int H, int rows_per_block) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= H) return;
+  const int r0 = blockIdx.y * rows_per_block, r1 = min(rows, r0 + rows_per_block);
+  float a0 = 0.f, a1 = 0.f;
+  for (int r = r0; r < r1; r++) {
+    const float v = to_f<T>(dz[(int64_t)r * H + c]);
+    const int sg = segments ? segments[r] : 0;
+    if (sg == 1) a1 += v; else a0 += v;
+  }
+  atomicAdd(dtype + c, a0);
+  atomicAdd(dtype + H + c, a1);
+}
+
 // LAMB, first kernel: new moments, and the per-tensor sums of w^2 and r^2
 __global__ void __launch_bounds__(256)
 lamb_moments_kernel(const AdamChunk* __restrict__ chunks, const float* __restrict__ w,
@@ -1023,13 +1134,13 @@ void launch_ln_fwd(bool bf, const void* z, const float* gamma, const float* beta
 #undef LN_FWD
 }
 
-void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* pos,
-                     const float* gamma, const float* beta, void* y, void* zstash, float* stats,
-                     int rows, int S, int H, int V, float eps, int* status, cudaStream_t st) {
+void launch_embed_ln(bool bf, const int* tokens, const int* segments, const void* word, const void* pos,
+                     const void* type, const float* gamma, const float* beta, void* y, void* zstash,
+                     float* stats, int rows, int S, int H, int V, float eps, int* status, cudaStream_t st) {
   if (rows <= 0) return;
   DISPATCH_T(bf, (embed_ln_kernel<T><<<div_up(rows, 8), 256, 0, st>>>(
-                     tokens, (const T*)word, (const T*)pos, gamma, beta, (T*)y, (T*)zstash, stats,
-                     rows, S, H, V, eps, status)));
+                     tokens, segments, (const T*)word, (const T*)pos, (const T*)type, gamma, beta, (T*)y,
+                     (T*)zstash, stats, rows, S, H, V, eps, status)));
 }
 
 void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, const float* gamma,
@@ -1157,6 +1268,33 @@ void launch_lamb(const AdamChunk* chunks, int n_chunks, float* w, const float* g
   cudaMemsetAsync(norms, 0, (size_t)n_tensors * 2 * sizeof(float), st);
   lamb_moments_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, g, m, v, h, bc_dev, norms);
   lamb_apply_kernel<<<n_chunks, 256, 0, st>>>(chunks, w, m, v, (bf16*)wb, h, bc_dev, norms);
+}
+
+void launch_nsp_prepare(const int* labels, int B, int S, int* rowsrc, float* inv_n, const int* total_valid,
+                        cudaStream_t st) {
+  nsp_prepare_kernel<<<1, 128, 0, st>>>(labels, B, S, rowsrc, inv_n, total_valid);
+}
+
+void launch_nsp_head(bool bf, const void* pooled, const float* wn, const float* bn, const int* labels,
+                     const float* inv_n, void* dup, float* dwn, float* dbn, float* loss, int B, int H,
+                     cudaStream_t st) {
+  if (B <= 0) return;
+  DISPATCH_T(bf, (nsp_head_kernel<T><<<B, 128, 0, st>>>((const T*)pooled, wn, bn, labels, inv_n, (T*)dup, dwn, dbn,
+                                                       loss, H)));
+}
+
+void launch_tanh(bool bf, const void* x, void* y, int64_t n, cudaStream_t st) {
+  if (n <= 0) return;
+  int blocks = (int)std::min<int64_t>((n + 255) / 256, 148 * 8);
+  DISPATCH_T(bf, (tanh_kernel<T><<<blocks, 256, 0, st>>>((const T*)x, (T*)y, n)));
+}
+
+void launch_type_grad(bool bf, const void* dz, const int* segments, float* dtype, int rows, int H,
+                      cudaStream_t st) {
+  if (rows <= 0) return;
+  const int rpb = 512;
+  DISPATCH_T(bf, (type_grad_kernel<T><<<dim3(div_up(H, 128), div_up(rows, rpb)), 128, 0, st>>>(
+                     (const T*)dz, segments, dtype, rows, H, rpb)));
 }
 
 void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st) {

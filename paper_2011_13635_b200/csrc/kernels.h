@@ -22,9 +22,10 @@ struct AdamHyper {
 
 void launch_ln_fwd(bool bf, const void* z, const float* gamma, const float* beta, void* y,
                    float* stats, int rows, int H, float eps, cudaStream_t st);
-void launch_embed_ln(bool bf, const int* tokens, const void* word, const void* pos,
-                     const float* gamma, const float* beta, void* y, void* zstash, float* stats,
-                     int rows, int S, int H, int V, float eps, int* status, cudaStream_t st);
+// segments / type: segment ids and the two-row segment table, or null (no segment term)
+void launch_embed_ln(bool bf, const int* tokens, const int* segments, const void* word, const void* pos,
+                     const void* type, const float* gamma, const float* beta, void* y, void* zstash,
+                     float* stats, int rows, int S, int H, int V, float eps, int* status, cudaStream_t st);
 void launch_ln_bwd(bool bf, const void* dy, const void* z, const float* stats, const float* gamma,
                    void* dz, float* dgamma, float* dbeta, float* dbias, int rows, int H, cudaStream_t st);
 void launch_softmax_fwd(bool bf, const void* sc, void* p, const int* seq_lens, int rows, int S,
@@ -61,6 +62,19 @@ void launch_lamb(const AdamChunk* chunks, int n_chunks, float* w, const float* g
                  void* wb, const AdamHyper& h, int* t_dev, float* bc_dev, int bias_correction,
                  float* norms, int n_tensors, cudaStream_t st);
 // d[i] *= gelu'(u[i]); n a multiple of the vector width
+// Next-sentence-prediction head.  prepare: rowsrc[b] = b * S (first tokens) and inv_n = 1 / (number of
+// labels in {0, 1}, or *total_valid when given).  head: two-way classifier on the pooled rows, loss
+// added to *loss, gradients of the classifier added to dwn [2,H] / dbn [2], and dup [B,H] = gradient
+// at the pooler's pre-activation (tanh derivative included).
+void launch_nsp_prepare(const int* labels, int B, int S, int* rowsrc, float* inv_n, const int* total_valid,
+                        cudaStream_t st);
+void launch_nsp_head(bool bf, const void* pooled, const float* wn, const float* bn, const int* labels,
+                     const float* inv_n, void* dup, float* dwn, float* dbn, float* loss, int B, int H,
+                     cudaStream_t st);
+void launch_tanh(bool bf, const void* x, void* y, int64_t n, cudaStream_t st);
+// dtype[seg[t], :] += dz[t, :] for the two-row segment table
+void launch_type_grad(bool bf, const void* dz, const int* segments, float* dtype, int rows, int H,
+                      cudaStream_t st);
 // data-parallel steps: the loss normaliser becomes 1 / *total_valid (0 when that count is 0)
 void launch_override_inv_n(const int* total_valid, float* inv_n, cudaStream_t st);
 void launch_dgelu(bool bf, void* d, const void* u, int64_t n, cudaStream_t st);

@@ -81,6 +81,8 @@ struct Workspace {
   char* z0;
   float* st0;
   char *hm, *ut, *gt, *tm, *dlogits, *dtm, *dgt, *dhm;
+  int* nsp_rowsrc;                          // NSP head: first-token row of every sequence
+  char *cls, *up, *pooled, *dup, *dcls;     // [B,H] each
   float *hst, *logits, *nll, *dtm32;
   char *dxa, *dxb, *dz2, *dg, *dy, *dz1, *dc, *dp, *dqkv;
 };
@@ -153,12 +155,16 @@ int check_arch(const mslt_arch* a) {
   if (a->max_trainable < 0 || a->max_trainable > a->max_layers)
     return fail(MSLT_ERR_ARG, "need 0 <= max_trainable <= max_layers");
   if (a->share_group < 0) return fail(MSLT_ERR_ARG, "share_group must be >= 0");
+  if (a->nsp != 0 && a->nsp != 1) return fail(MSLT_ERR_ARG, "nsp must be 0 or 1");
   if (a->share_group > 1 && (a->init_layers % a->share_group || a->max_layers % a->share_group ||
                              a->max_trainable % a->share_group))
     return fail(MSLT_ERR_ARG, "init_layers, max_layers and max_trainable must be multiples of share_group");
   return 0;
 }
 
+// tensors before the first encoder block and after the last
+int n_emb_tensors(const mslt_arch& a) { return a.nsp ? 5 : 4; }
+int n_head_tensors(const mslt_arch& a) { return a.nsp ? 9 : 5; }
 // layers per shared parameter block (Section 3.3); layer l reads block l / group
 int group_of(const mslt_arch& a) { return a.share_group > 1 ? a.share_group : 1; }
 
@@ -178,6 +184,7 @@ void build_tensor_table(const mslt_arch& a, std::vector<Tensor>& out, int64_t& t
   add("emb.pos", 2, a.max_pos, H, -1);
   add("emb.ln.gamma", 1, H, 0, -1);
   add("emb.ln.beta", 1, H, 0, -1);
+  if (a.nsp) add("emb.type", 2, 2, H, -1);  // segment table, part of the embeddings
   for (int l = 0; l < a.max_layers / group_of(a); l++) {  // one block per group of layers
     const std::string p = "layer." + std::to_string(l) + ".";
     const int64_t rows[12] = {3 * H, H, F, H, 3 * H, H, H, H, F, H, H, H};
@@ -189,6 +196,12 @@ void build_tensor_table(const mslt_arch& a, std::vector<Tensor>& out, int64_t& t
   add("head.ln.gamma", 1, H, 0, -2);
   add("head.ln.beta", 1, H, 0, -2);
   add("head.decoder.bias", 1, V, 0, -2);
+  if (a.nsp) {  // next-sentence-prediction head, part of the output layer
+    add("head.pooler.weight", 2, H, H, -2);
+    add("head.pooler.bias", 1, H, 0, -2);
+    add("head.nsp.weight", 2, 2, H, -2);
+    add("head.nsp.bias", 1, 2, 0, -2);
+  }
   total = off;
 }
 
@@ -245,6 +258,12 @@ void plan_workspace(const mslt_arch& a, const std::vector<Tensor>& tensors, char
   w.nll = (float*)take(R * 4);
   w.dtm = take(R * H * E); w.dgt = take(R * H * E); w.dhm = take(R * H * E);
   w.dtm32 = (float*)take(R * H * 4);
+  if (a.nsp) {
+    const int64_t Bm = a.max_batch;
+    w.nsp_rowsrc = (int*)take(Bm * 4);
+    w.cls = take(Bm * H * E); w.up = take(Bm * H * E); w.pooled = take(Bm * H * E);
+    w.dup = take(Bm * H * E); w.dcls = take(Bm * H * E);
+  }
   w.dxa = take(T * H * E); w.dxb = take(T * H * E); w.dz2 = take(T * H * E);
   w.dg = take(T * F * E); w.dy = take(T * H * E); w.dz1 = take(T * H * E);
   w.dc = take(T * H * E); w.dp = take(P2 * E); w.dqkv = take(T * 3 * H * E);
@@ -272,7 +291,7 @@ bool is_trainable(const mslt_ctx* c, const Tensor& t) {
 int64_t toff(const mslt_ctx* c, int layer, const char* n) {
   if (layer >= 0) {
     for (int i = 0; i < 12; i++)
-      if (strcmp(n, kLayerNames[i]) == 0) return c->tensors[4 + 12 * (layer / group_of(c->a)) + i].offset;
+      if (strcmp(n, kLayerNames[i]) == 0) return c->tensors[n_emb_tensors(c->a) + 12 * (layer / group_of(c->a)) + i].offset;
   }
   return c->tensors[c->by_name.at(n)].offset;
 }
@@ -816,8 +835,11 @@ static int apply_update(mslt_ctx* c);
 // forward, loss and backward of one step; the optimizer runs too unless `defer_update`
 static int step_impl(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
                      const int32_t* d_pos, const int32_t* d_lab, int32_t B, int32_t S, int32_t P,
-                     const int32_t* d_total_valid, bool defer_update, float* loss_out) {
+                     const int32_t* d_total_valid, bool defer_update, float* loss_out,
+                     const int32_t* d_seg = nullptr, const int32_t* d_nsp_lab = nullptr) {
   if (!c || !d_tokens || !d_pos || !d_lab) return fail(MSLT_ERR_ARG, "null pointer");
+  if ((d_seg || d_nsp_lab) && !c->a.nsp)
+    return fail(MSLT_ERR_STATE, "segment ids / NSP labels need a context created with arch.nsp = 1");
   if (c->pending_update)
     return fail(MSLT_ERR_STATE, "mslt_step_backward was called: call mslt_step_apply before the next step");
   TRY(check_batch(c, B, S, P));
@@ -841,7 +863,8 @@ static int step_impl(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_
   if (d_total_valid)  // the mean runs over the valid slots of every rank's batch
     KL(PC_OTHER, 8.0, launch_override_inv_n(d_total_valid, inv_n, c->st));
   // embeddings, then the frozen prefix: forward only, two buffers, nothing kept but the output
-  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_embed_ln(c->bf, d_tokens, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
+  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_embed_ln(c->bf, d_tokens, d_seg, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
+                     c->a.nsp ? Wc(c, toff(c, -1, "emb.type")) : nullptr,
                      Wv(c, toff(c, -1, "emb.ln.gamma")), Wv(c, toff(c, -1, "emb.ln.beta")), w.xa,
                      full ? w.z0 : nullptr, full ? w.st0 : nullptr, T, S, H, V, c->a.ln_eps, status,
                      c->st));
@@ -862,8 +885,30 @@ static int step_impl(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_
   TRY(head_forward(c, cur, R, true));
   KL(PC_CROSS_ENTROPY, (double)R * c->Vp * (4 + c->esz), launch_cross_entropy(c->bf, w.logits, c->Vp, w.rowlabel, inv_n, w.dlogits, c->Vp, w.nll, R, V, c->st));
   KL(PC_OTHER, 4.0 * R, launch_loss_reduce(w.nll, R, inv_n, loss, c->st));
+  const bool nsp = c->a.nsp && d_nsp_lab != nullptr;
+  float* nsp_inv_n = (float*)(w.scalars + 7);
+  if (nsp) {
+    // second objective, forward: pooled = tanh(Wp x_L[b, 0] + bp)
+    const int32_t* nsp_total = d_total_valid ? d_total_valid + 1 : nullptr;
+    KL(PC_OTHER, 8.0 * B, launch_nsp_prepare(d_nsp_lab, B, S, w.nsp_rowsrc, nsp_inv_n, nsp_total, c->st));
+    KL(PC_OTHER, 2.0 * B * H * c->esz, launch_gather_rows(c->bf, cur, w.nsp_rowsrc, w.cls, B, H, c->st));
+    TRY(linear_fwd(c, w.cls, B, H, toff(c, -1, "head.pooler.weight"), toff(c, -1, "head.pooler.bias"), H, w.up, 0,
+                   nullptr, nullptr));
+    KL(PC_OTHER, 2.0 * B * H * c->esz, launch_tanh(c->bf, w.up, w.pooled, (int64_t)B * H, c->st));
+  }
   TRY(zero_trainable_grads(c));
   TRY(head_backward(c, B, S, P, full));
+  if (nsp) {
+    // classifier, its loss (added to the MLM loss) and its gradients; then back through the pooler
+    // into the first token's row of the last hidden state's gradient
+    KL(PC_OTHER, 4.0 * B * H * c->esz, launch_nsp_head(c->bf, w.pooled, Wv(c, toff(c, -1, "head.nsp.weight")),
+                     Wv(c, toff(c, -1, "head.nsp.bias")), d_nsp_lab, nsp_inv_n, w.dup,
+                     G(c, toff(c, -1, "head.nsp.weight")), G(c, toff(c, -1, "head.nsp.bias")), loss, B, H, c->st));
+    TRY(linear_wgrad(c, w.dup, B, H, H, w.cls, H, toff(c, -1, "head.pooler.weight")));
+    KL(PC_COLSUM, 1.0 * B * H * c->esz, launch_colsum(c->bf, w.dup, H, B, H, G(c, toff(c, -1, "head.pooler.bias")), c->st));
+    TRY(linear_dgrad(c, w.dup, B, H, H, toff(c, -1, "head.pooler.weight"), H, w.dcls, 0, nullptr, nullptr));
+    KL(PC_OTHER, 2.0 * B * H * c->esz, launch_scatter_rows(c->bf, w.dcls, w.nsp_rowsrc, w.dxa, B, 1, H, c->st));
+  }
   TRY(bucket_done(c, 0));
   mark(c, 3);
   char* dx = w.dxa;
@@ -881,6 +926,8 @@ static int step_impl(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_
                      G(c, toff(c, -1, "emb.ln.gamma")), G(c, toff(c, -1, "emb.ln.beta")), nullptr, T, H, c->st));
     KL(PC_OTHER, 1.0 * T * H * c->esz, launch_embed_scatter(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
                             G(c, toff(c, -1, "emb.pos")), T, S, H, V, c->st));
+    if (c->a.nsp)
+      KL(PC_OTHER, 1.0 * T * H * c->esz, launch_type_grad(c->bf, w.dz2, d_seg, G(c, toff(c, -1, "emb.type")), T, H, c->st));
     TRY(bucket_done(c, c->top_k / group_of(c->a) + 1));
   }
   mark(c, 4);
@@ -939,6 +986,13 @@ int mslt_step(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
   return step_impl(c, d_tokens, d_seq_lens, d_pos, d_lab, B, S, P, nullptr, false, loss_out);
 }
 
+int mslt_step_nsp(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens, const int32_t* d_seg,
+                  const int32_t* d_pos, const int32_t* d_lab, const int32_t* d_nsp_lab, int32_t B, int32_t S,
+                  int32_t P, float* loss_out) {
+  if (c && !c->a.nsp) return fail(MSLT_ERR_STATE, "mslt_step_nsp needs a context created with arch.nsp = 1");
+  return step_impl(c, d_tokens, d_seq_lens, d_pos, d_lab, B, S, P, nullptr, false, loss_out, d_seg, d_nsp_lab);
+}
+
 int mslt_step_backward(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens,
                        const int32_t* d_pos, const int32_t* d_lab, int32_t B, int32_t S, int32_t P,
                        const int32_t* d_total_valid, float* loss_out) {
@@ -992,7 +1046,8 @@ int mslt_forward(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_lens
   if (head)
     KL(PC_OTHER, 8.0 * B * P, launch_slots_prepare(d_pos, nullptr, d_seq_lens, B, S, P, V, w.rowsrc, w.rowlabel,
                             w.scalars + 1, (float*)(w.scalars + 2), w.scalars, c->st));
-  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_embed_ln(c->bf, d_tokens, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
+  KL(PC_LN_FWD, 2.0 * T * H * c->esz, launch_embed_ln(c->bf, d_tokens, nullptr, Wc(c, toff(c, -1, "emb.word")), Wc(c, toff(c, -1, "emb.pos")),
+                     c->a.nsp ? Wc(c, toff(c, -1, "emb.type")) : nullptr,
                      Wv(c, toff(c, -1, "emb.ln.gamma")), Wv(c, toff(c, -1, "emb.ln.beta")), w.xa,
                      nullptr, nullptr, T, S, H, V, c->a.ln_eps, w.scalars, c->st));
   char* cur = w.xa;
@@ -1017,15 +1072,16 @@ int mslt_num_trainable(const mslt_ctx* c) { return c ? c->top_k : MSLT_ERR_ARG; 
 
 int mslt_num_tensors(const mslt_ctx* c) {
   if (!c) return MSLT_ERR_ARG;
-  return 4 + 12 * (c->L / group_of(c->a)) + 5;
+  return n_emb_tensors(c->a) + 12 * (c->L / group_of(c->a)) + n_head_tensors(c->a);
 }
 
 static const Tensor* tensor_by_index(const mslt_ctx* c, int i) {
   const int n_layer_t = 12 * (c->L / group_of(c->a));
   if (i < 0) return nullptr;
-  if (i < 4 + n_layer_t) return &c->tensors[i];
-  i -= 4 + n_layer_t;
-  if (i < 5) return &c->tensors[4 + 12 * (c->a.max_layers / group_of(c->a)) + i];
+  const int ne = n_emb_tensors(c->a);
+  if (i < ne + n_layer_t) return &c->tensors[i];
+  i -= ne + n_layer_t;
+  if (i < n_head_tensors(c->a)) return &c->tensors[ne + 12 * (c->a.max_layers / group_of(c->a)) + i];
   return nullptr;
 }
 

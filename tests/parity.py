@@ -23,7 +23,9 @@ from paper_2011_13635_b200 import inputs as I
 #   is at most half of such an element, so its first-step update is off by at most
 #   lr * eps * tol_grad * G / (|g_ref| / 2 + eps)^2 (never more than lr / 4), plus update_max for
 #   the rounding of the arithmetic itself.
-TOL = {"fp32": dict(loss=2e-3, grad=1e-4, weight=1e-4, hidden=1e-4, update_l1=2e-3, update_max=1e-4),
+#   (fp32 update_l1: gradients as small as eps = 1e-6, e.g. those of the pooler under the second
+#   objective, make g / (|g| + eps) amplify a 1e-4 gradient error to a few 1e-3 in the mean.)
+TOL = {"fp32": dict(loss=2e-3, grad=1e-4, weight=1e-4, hidden=1e-4, update_l1=5e-3, update_max=1e-4),
        "bf16": dict(loss=2e-3, grad=3e-2, weight=3e-2, hidden=3e-2, update_l1=0.15, update_max=1e-3)}
 
 
@@ -75,7 +77,8 @@ def build_pair(cfg: I.StageConfig, lr: float, max_layers=None, init_layers=None,
 def compare_step(m, oracle, cfg, batch, tol, report=None):
     """One step on both sides; asserts loss, gradients, weights and the frozen slice."""
     import torch
-    tok, lens, pos, lab = batch
+    tok, lens, pos, lab = batch[:4]
+    seg, nlab = (batch[4], batch[5]) if len(batch) == 6 else (None, None)   # both objectives
     names = oracle.trainable_names()
     all_names = list(oracle.p.keys())
     frozen = [n for n in all_names if n not in names]
@@ -86,8 +89,13 @@ def compare_step(m, oracle, cfg, batch, tol, report=None):
     ow_before = {n: oracle.p[n].copy() for n in names}
 
     d_tok, d_lens, d_pos, d_lab = to_cuda(torch, tok, lens if cfg.varlen else None, pos, lab)
-    loss_g = m.mslt_step(d_tok, d_lens, d_pos, d_lab)
-    loss_o = oracle.step(tok, lens, pos, lab)
+    if len(batch) == 6:
+        d_seg, d_nlab = to_cuda(torch, seg, nlab)
+        loss_g = m.mslt_step_nsp(d_tok, d_lens, d_seg, d_pos, d_lab, d_nlab)
+        loss_o = oracle.step(tok, lens, pos, lab, seg, nlab)
+    else:
+        loss_g = m.mslt_step(d_tok, d_lens, d_pos, d_lab)
+        loss_o = oracle.step(tok, lens, pos, lab)
     rel_loss = abs(loss_g - loss_o) / abs(loss_o)
     assert rel_loss < tol["loss"], (loss_g, loss_o)
 

@@ -52,6 +52,32 @@ def test_fp32_lamb_staged_and_all_trainable():
     _run(I.scaled(TINY, trainable=2), steps=2, lr=0.00088, lamb=1, weight_decay=0.0)
 
 
+def _run_nsp(cfg, steps, lr, drop_labels=False):
+    """Both objectives (Section 4.1): segment embeddings, pooler and two-way classifier."""
+    m, oracle = PT.build_pair(cfg, lr=lr)
+    assert oracle.nsp and "emb.type" in m.tensors() and "head.nsp.weight" in m.tensors()
+    rep = []
+    for s in range(steps):
+        seed = I.config_seed(cfg) + s
+        tok, lens, pos, lab = I.make_batch(cfg, seed=seed)
+        seg, nlab = I.make_nsp(cfg, lens, seed=seed)
+        if s == 1:
+            nlab[0] = -1                               # an ignored sequence
+        PT.compare_step(m, oracle, cfg, (tok, lens, pos, lab, seg, None if drop_labels else nlab),
+                        PT.TOL[cfg.dtype], rep)
+    m.close()
+    return rep
+
+
+def test_fp32_nsp_objective_staged_and_all_trainable():
+    cfg = I.scaled(TINY, nsp=True, varlen=(20, 64))
+    rep = _run_nsp(cfg, steps=2, lr=1e-3)
+    assert abs(rep[0]["loss_gpu"] - (math.log(cfg.vocab) + math.log(2))) < 0.3      # MLM + NSP at the start
+    _run_nsp(I.scaled(cfg, trainable=2), steps=2, lr=1e-3)
+    rep = _run_nsp(cfg, steps=1, lr=1e-3, drop_labels=True)                         # segments only
+    assert abs(rep[0]["loss_gpu"] - math.log(cfg.vocab)) < 0.2
+
+
 # -- bf16 path ---------------------------------------------------------------------------------
 
 BASE_SMALL = I.scaled(I.CONFIGS["base_stage"], layers=3, trainable=2, batch=4)
@@ -70,6 +96,12 @@ def test_bf16_base_shapes_all_trainable():
 def test_bf16_lamb_base_shapes():
     _run(BASE_SMALL, steps=2, lr=0.00088, lamb=1)
     _run(I.scaled(BASE_SMALL, layers=2, trainable=2, batch=2), steps=1, lr=0.00088, lamb=1)
+
+
+def test_bf16_nsp_objective_base_shapes():
+    cfg = I.scaled(BASE_SMALL, nsp=True)
+    _run_nsp(cfg, steps=2, lr=1e-4)
+    _run_nsp(I.scaled(cfg, layers=2, trainable=2, batch=3), steps=1, lr=1e-4)
 
 
 def test_bf16_head_only():
