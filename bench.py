@@ -233,9 +233,11 @@ def aggregate(ms_local: float, batch_per_rank: int, steps: int, world: int, dist
     return ms, batch_per_rank * world * steps / (ms * 1e-3)
 
 
-# DRAM bytes per launch of the contraction kernel from ncu captures of single launches (summaries
-# and commands under profiles/); None where the kernel has changed since the counters were taken.
-GEMM_DRAM_BYTES_PER_LAUNCH = None
+# DRAM bytes (read + write) per launch of the contraction kernel from ncu captures of single launches
+# of the four forward products of a BERT-Base layer (profiles/gemm_tc_kernel_frozen_layer_shapes_16384.md):
+# QKV 53.0 MB, out-proj 53.6 MB, FFN1 80.9 MB, FFN2 144.3 MB; the bench line carries their mean, which
+# holds for the BERT-Base configurations only.  None once the kernel changes.
+GEMM_DRAM_BYTES_PER_LAUNCH = {"base": 82.9e6}
 
 
 def gemm_peaks(peaks, clocks):
@@ -349,7 +351,7 @@ def measure(cfg, args, torch, dist, world, rank, local, steps, warmup, headline)
             rec["roofline"] = dict(
                 bound="tensor", kernel="gemm_tc_kernel (linear-layer products of the step)",
                 achieved=lin_tflops, peak=peak, unit="TFLOP/s", frac=lin_tflops / peak,
-                traffic=GEMM_DRAM_BYTES_PER_LAUNCH,
+                traffic=GEMM_DRAM_BYTES_PER_LAUNCH.get("base") if cfg.hidden == 768 and cfg.batch * cfg.seq == 16384 else None,
                 peak_source=f"{peaks['source']}: cuBLAS bf16 8192^3, {regime} figure (median SM clock "
                             f"{clocks.get('sm_mhz')} of {clocks.get('sm_max_mhz')} MHz in the timed region)",
                 frac_of_burst=lin_tflops / burst, frac_of_sustained=lin_tflops / sustained,
@@ -439,7 +441,7 @@ def run_ours(args, cfg):
                                       "--iters", "20", "--only", "attention,ln,colsum,ce"], emit=None)
             line["hbm_kernels_alone"] = {
                 r["kernel"]: dict(us=r["us"], gbs=r["gbs"], frac_of_measured_copy=r["gbs"] / peaks["hbm_gbs"],
-                                  dram_bytes_ncu=HBM_DRAM_BYTES_NCU.get(r["kernel"]))
+                                  dram_bytes_ncu=HBM_DRAM_BYTES_NCU.get(r["kernel"]) if cfg.name.startswith("base") else None)
                 for r in recs}
             line["hbm_kernels_alone"]["clocks"] = clk2.summary()
             torch.cuda.empty_cache()
@@ -452,8 +454,11 @@ def run_ours(args, cfg):
 
 
 # DRAM bytes per launch of the memory-bound kernels at the op_bench sizes, from one-kernel ncu captures
-# (profiles/); keys are op_bench's kernel names.  Empty until the captures are taken for this build.
-HBM_DRAM_BYTES_NCU = {}
+# (profiles/memory_bound_kernels_base_16384.md); keys are op_bench's kernel names; read + write, outputs
+# that were still in L2 at kernel end are not in the write counter.
+HBM_DRAM_BYTES_NCU = {"layernorm": 25.2e6, "layernorm_bwd": 50.7e6, "colsum_hidden": 25.2e6, "colsum_ffn": 101.3e6,
+                      "cross_entropy(sync)": 436.6e6, "attention_fused": 79.0e6,
+                      "attention_fused_with_probs": 98.9e6, "attention_fused_backward": 191.3e6}
 
 
 # ------------------------------------------------------------------------------------------------
