@@ -842,24 +842,235 @@ colsum_kernel(const T* __restrict__ x, int64_t ld, int rows, int N, int rows_per
 
 // ---------------------------------------------------------------------------------------
 // Embedding gradient: dword[token[t], :] += dz[t, :], dpos[t % S, :] += dz[t, :].
+// Without atomics on hot rows, and with the same bits on every run: the rows are
+// grouped by token id with a counting sort whose order is fixed (block of 256 rows, then position
+// inside the block), one thread block per token id then adds its rows in that order, and the
+// position table gets a plain sum over the batch.
+//   counts [nb][V]  (nb = ceil(T / 256)): rows of block b with token v, turned into the exclusive
+//                   prefix over blocks;  total[V], start[V];  order[T]: rows sorted by (token, row).
 // ---------------------------------------------------------------------------------------
-template <typename T>
-__global__ void embed_scatter_kernel(const T* __restrict__ dz, const int* __restrict__ tokens,
-                                     float* __restrict__ dword, float* __restrict__ dpos, int S,
-                                     int H, int V) {
-  constexpr int VN = VecT<T>::N;
-  const int t = blockIdx.x;
+constexpr int ES_BLOCK = 256;   // rows per sort block
+constexpr int ES_TOKENS = 8;    // token ids per block of the reduction kernel
+constexpr int ES_CHUNK = 64;    // rows one block adds for a frequent token
+constexpr int ES_MAX_SLOTS = 2048;  // chunk slots: at most T / ES_CHUNK + (tokens above ES_CHUNK) <= 2 T / ES_CHUNK
+
+// counts is laid out [V][nb] so that a token's per-block counts are contiguous
+__global__ void __launch_bounds__(ES_BLOCK)
+embed_sort_count_kernel(const int* __restrict__ tokens, int T, int V, int nb, int* __restrict__ counts,
+                        int* __restrict__ rank) {
+  __shared__ int tk[ES_BLOCK];
+  const int t = blockIdx.x * ES_BLOCK + threadIdx.x;
+  int tok = t < T ? tokens[t] : -1;
+  if (t < T && (tok < 0 || tok >= V)) tok = 0;
+  tk[threadIdx.x] = tok;
+  __syncthreads();
+  if (t >= T) return;
+  int r = 0;
+  for (int j = 0; j < (int)threadIdx.x; j++) r += tk[j] == tok ? 1 : 0;  // rows of this block before me with my token
+  rank[t] = r;
+  atomicAdd(counts + (int64_t)tok * nb + blockIdx.x, 1);  // integer: the result does not depend on the order
+}
+
+// Per token: exclusive prefix of its counts over the row blocks and its total; per block of 256
+// tokens: exclusive scan of the totals (local start) and the block's sum.
+__global__ void __launch_bounds__(256)
+embed_sort_prefix_kernel(int* __restrict__ counts, int nb, int V, int* __restrict__ total,
+                         int* __restrict__ start_local, int* __restrict__ blocksum, int* __restrict__ hot) {
+  __shared__ int part[256];
+  const int v = blockIdx.x * 256 + threadIdx.x;
+  int run = 0;
+  if (v < V) {
+    int* row = counts + (int64_t)v * nb;
+    for (int b = 0; b < nb; b++) {
+      const int c = row[b];
+      row[b] = run;
+      run += c;
+    }
+    total[v] = run;
+    // A token with more than ES_CHUNK rows is summed in chunks of ES_CHUNK rows by several blocks.
+    // hot[0] = chunks handed out, hot[1] = such tokens; then per chunk slot (token, chunk index) and
+    // per hot token (token, first slot).  Which slot a token gets is arbitrary and changes nothing:
+    // the rows of a chunk and the chunks of a token are always added in the same order.
+    if (run > ES_CHUNK) {
+      const int nch = (run + ES_CHUNK - 1) / ES_CHUNK;
+      const int base = atomicAdd(hot, nch);
+      const int h = atomicAdd(hot + 1, 1);
+      hot[2 + 2 * ES_MAX_SLOTS + 2 * h] = v;
+      hot[2 + 2 * ES_MAX_SLOTS + 2 * h + 1] = base;
+      for (int k = 0; k < nch; k++) {
+        hot[2 + 2 * (base + k)] = v;
+        hot[2 + 2 * (base + k) + 1] = k;
+      }
+    }
+  }
+  part[threadIdx.x] = run;
+  __syncthreads();
+  for (int o = 1; o < 256; o <<= 1) {
+    const int add = threadIdx.x >= o ? part[threadIdx.x - o] : 0;
+    __syncthreads();
+    part[threadIdx.x] += add;
+    __syncthreads();
+  }
+  if (v < V) start_local[v] = part[threadIdx.x] - run;
+  if (threadIdx.x == 255) blocksum[blockIdx.x] = part[255];
+}
+
+// exclusive scan of the block sums (at most 1024 blocks of 256 tokens) in place
+__global__ void __launch_bounds__(1024)
+embed_sort_scan_kernel(int* __restrict__ blocksum, int n) {
+  __shared__ int part[1024];
+  const int mine = threadIdx.x < n ? blocksum[threadIdx.x] : 0;
+  part[threadIdx.x] = mine;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {
+    const int add = threadIdx.x >= o ? part[threadIdx.x - o] : 0;
+    __syncthreads();
+    part[threadIdx.x] += add;
+    __syncthreads();
+  }
+  if (threadIdx.x < n) blocksum[threadIdx.x] = part[threadIdx.x] - mine;
+}
+
+__global__ void embed_sort_place_kernel(const int* __restrict__ tokens, int T, int V, int nb,
+                                        const int* __restrict__ counts, const int* __restrict__ rank,
+                                        const int* __restrict__ start_local, const int* __restrict__ blockoff,
+                                        int* __restrict__ order) {
+  const int t = blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= T) return;
   int tok = tokens[t];
   if (tok < 0 || tok >= V) tok = 0;
-  float* wr = dword + (int64_t)tok * H;
-  float* pr = dpos + (int64_t)(t % S) * H;
-  for (int c = threadIdx.x * VN; c < H; c += blockDim.x * VN) {
-    float a[VN];
-    VecT<T>::load(dz + (int64_t)t * H + c, a);
+  order[blockoff[tok >> 8] + start_local[tok] + counts[(int64_t)tok * nb + t / ES_BLOCK] + rank[t]] = t;
+}
+
+// Adds the rows order[first .. first + n) of dz in that order: H / VN column threads times G row
+// groups; group g takes the rows g, g + G, ... with eight loads in flight and the groups' partial sums
+// meet in shared memory in a fixed order.  The result is added to dst[0 .. H) (add) or stored there.
+template <typename T, int NT>
+__device__ __forceinline__ void es_sum_rows(const T* __restrict__ dz, const int* __restrict__ seg, int n, int H,
+                                            float* es_part, float* __restrict__ dst, bool add) {
+  constexpr int VN = VecT<T>::N;
+  const int colthreads = H / VN;
+  const int G = NT / colthreads;
+  const int ct = threadIdx.x % colthreads, g = threadIdx.x / colthreads;
+  float acc[VN];
 #pragma unroll
-    for (int e = 0; e < VN; e++) {
-      atomicAdd(wr + c + e, a[e]);
-      atomicAdd(pr + c + e, a[e]);
+  for (int e = 0; e < VN; e++) acc[e] = 0.f;
+  if (g < G) {
+    int i = g;
+    for (; i + 7 * G < n; i += 8 * G) {
+      float a[8][VN];
+#pragma unroll
+      for (int u = 0; u < 8; u++) VecT<T>::load(dz + (int64_t)seg[i + u * G] * H + ct * VN, a[u]);
+#pragma unroll
+      for (int u = 0; u < 8; u++)
+#pragma unroll
+        for (int e = 0; e < VN; e++) acc[e] += a[u][e];
+    }
+    for (; i < n; i += G) {
+      float a[VN];
+      VecT<T>::load(dz + (int64_t)seg[i] * H + ct * VN, a);
+#pragma unroll
+      for (int e = 0; e < VN; e++) acc[e] += a[e];
+    }
+#pragma unroll
+    for (int e = 0; e < VN; e++) es_part[g * H + ct * VN + e] = acc[e];
+  }
+  __syncthreads();
+  const int used = min(G, n);  // groups beyond the segment's length hold zeros: skip them
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float s = 0.f;
+    for (int k = 0; k < used; k++) s += es_part[k * H + c];
+    dst[c] = add ? dst[c] + s : s;
+  }
+  __syncthreads();
+}
+
+// dword[v, :] += sum of the dz rows of token v, for the tokens with at most ES_CHUNK rows.  Token ids
+// are dealt out with a stride of the grid size: frequent ids are neighbours (ids follow frequency rank
+// in natural text and in the synthetic batches) and must not share a block.
+template <typename T>
+__global__ void __launch_bounds__(256)
+embed_word_grad_kernel(const T* __restrict__ dz, const int* __restrict__ order, const int* __restrict__ start_local,
+                       const int* __restrict__ blockoff, const int* __restrict__ total,
+                       float* __restrict__ dword, int H, int V) {
+  extern __shared__ float es_part[];  // [G][H]
+  for (int v = blockIdx.x; v < V; v += gridDim.x) {
+    const int n = total[v];
+    if (n == 0 || n > ES_CHUNK) continue;  // the same for every thread of the block
+    es_sum_rows<T, 256>(dz, order + blockoff[v >> 8] + start_local[v], n, H, es_part, dword + (int64_t)v * H, true);
+  }
+}
+
+// frequent tokens, first half: block = chunk slot, partial[slot, :] = sum of the chunk's rows
+template <typename T>
+__global__ void __launch_bounds__(1024)
+embed_word_hot_chunk_kernel(const T* __restrict__ dz, const int* __restrict__ order,
+                            const int* __restrict__ start_local, const int* __restrict__ blockoff,
+                            const int* __restrict__ total, const int* __restrict__ hot,
+                            float* __restrict__ partial, int H) {
+  extern __shared__ float es_part[];
+  const int slot = blockIdx.x;
+  if (slot >= min(hot[0], ES_MAX_SLOTS)) return;
+  const int v = hot[2 + 2 * slot], k = hot[2 + 2 * slot + 1];
+  const int n = min(ES_CHUNK, total[v] - k * ES_CHUNK);
+  es_sum_rows<T, 1024>(dz, order + blockoff[v >> 8] + start_local[v] + k * ES_CHUNK, n, H, es_part,
+                 partial + (int64_t)slot * H, false);
+}
+
+// second half: block = frequent token, dword[v, :] += its chunks' partial sums in chunk order
+__global__ void embed_word_hot_sum_kernel(const int* __restrict__ total, const int* __restrict__ hot,
+                                          const float* __restrict__ partial, float* __restrict__ dword, int H) {
+  const int h = blockIdx.x;
+  if (h >= min(hot[1], ES_MAX_SLOTS / 2)) return;
+  const int v = hot[2 + 2 * ES_MAX_SLOTS + 2 * h], base = hot[2 + 2 * ES_MAX_SLOTS + 2 * h + 1];
+  const int nch = (total[v] + ES_CHUNK - 1) / ES_CHUNK;
+  for (int c = threadIdx.x; c < H; c += blockDim.x) {
+    float s = 0.f;
+    for (int k = 0; k < nch; k++) s += partial[(int64_t)(base + k) * H + c];
+    dword[(int64_t)v * H + c] += s;
+  }
+}
+
+// dpos[s, :] += sum over the batch of dz[b * S + s, :].  Block (s, column slab of 32 vectors): 32
+// column threads times 8 row groups over the batch, combined in shared memory in a fixed order.
+template <typename T>
+__global__ void __launch_bounds__(256)
+embed_pos_grad_kernel(const T* __restrict__ dz, float* __restrict__ dpos, int B, int S, int H) {
+  constexpr int VN = VecT<T>::N;
+  __shared__ float part[8][32 * VN];
+  const int s = blockIdx.x;
+  const int lane = threadIdx.x & 31, g = threadIdx.x >> 5;
+  const int c = (blockIdx.y * 32 + lane) * VN;
+  float acc[VN];
+#pragma unroll
+  for (int e = 0; e < VN; e++) acc[e] = 0.f;
+  if (c < H) {
+    int b = g;
+    for (; b + 24 < B; b += 32) {
+      float a[4][VN];
+#pragma unroll
+      for (int u = 0; u < 4; u++) VecT<T>::load(dz + ((int64_t)(b + 8 * u) * S + s) * H + c, a[u]);
+#pragma unroll
+      for (int u = 0; u < 4; u++)
+#pragma unroll
+        for (int e = 0; e < VN; e++) acc[e] += a[u][e];
+    }
+    for (; b < B; b += 8) {
+      float a[VN];
+      VecT<T>::load(dz + ((int64_t)b * S + s) * H + c, a);
+#pragma unroll
+      for (int e = 0; e < VN; e++) acc[e] += a[e];
+    }
+  }
+#pragma unroll
+  for (int e = 0; e < VN; e++) part[g][lane * VN + e] = acc[e];
+  __syncthreads();
+  for (int i = threadIdx.x; i < 32 * VN; i += 256) {
+    const int col = blockIdx.y * 32 * VN + i;
+    if (col < H) {
+      float t = 0.f;
+      for (int k = 0; k < 8; k++) t += part[k][i];
+      dpos[(int64_t)s * H + col] += t;
     }
   }
 }
@@ -1245,11 +1456,30 @@ void launch_colsum(bool bf, const void* x, int64_t ld, int rows, int N, float* o
   DISPATCH_T(bf, (colsum_kernel<T><<<dim3(gx, gy), 256, 0, st>>>((const T*)x, ld, rows, N, rpb, out)));
 }
 
-void launch_embed_scatter(bool bf, const void* dz, const int* tokens, float* dword, float* dpos,
-                          int rows, int S, int H, int V, cudaStream_t st) {
-  if (rows <= 0) return;
-  DISPATCH_T(bf, (embed_scatter_kernel<T><<<rows, 128, 0, st>>>((const T*)dz, tokens, dword, dpos, S,
-                                                               H, V)));
+void launch_embed_grad_sorted(bool bf, const void* dz, const int* tokens, float* dword, float* dpos, int B, int S,
+                              int H, int V, int* counts, int* total, int* start, int* rank, int* order,
+                              int* blocksum, int* hot, float* partial, cudaStream_t st) {
+  const int T = B * S;
+  if (T <= 0) return;
+  const int nb = div_up(T, ES_BLOCK), vb = div_up(V, 256);
+  cudaMemsetAsync(counts, 0, (size_t)nb * V * sizeof(int), st);
+  cudaMemsetAsync(hot, 0, 2 * sizeof(int), st);
+  embed_sort_count_kernel<<<nb, ES_BLOCK, 0, st>>>(tokens, T, V, nb, counts, rank);
+  embed_sort_prefix_kernel<<<vb, 256, 0, st>>>(counts, nb, V, total, start, blocksum, hot);
+  embed_sort_scan_kernel<<<1, 1024, 0, st>>>(blocksum, vb);
+  embed_sort_place_kernel<<<div_up(T, 256), 256, 0, st>>>(tokens, T, V, nb, counts, rank, start, blocksum, order);
+  const int vn = bf ? 8 : 4;
+  const size_t smem = (size_t)(1024 / (H / vn)) * H * sizeof(float), smem_small = (size_t)(256 / (H / vn)) * H * sizeof(float);
+  // at most T / ES_CHUNK tokens have more than ES_CHUNK rows, and they have at most 2 T / ES_CHUNK chunks
+  const int max_hot = std::min(ES_MAX_SLOTS / 2, T / ES_CHUNK), max_slots = std::min(ES_MAX_SLOTS, 2 * (T / ES_CHUNK));
+  DISPATCH_T(bf, (embed_word_grad_kernel<T><<<div_up(V, ES_TOKENS), 256, smem_small, st>>>(
+                     (const T*)dz, order, start, blocksum, total, dword, H, V)));
+  if (max_slots > 0) {
+    DISPATCH_T(bf, (embed_word_hot_chunk_kernel<T><<<max_slots, 1024, smem, st>>>((const T*)dz, order, start, blocksum,
+                                                                              total, hot, partial, H)));
+    embed_word_hot_sum_kernel<<<max_hot, 256, 0, st>>>(total, hot, partial, dword, H);
+  }
+  DISPATCH_T(bf, (embed_pos_grad_kernel<T><<<dim3(S, div_up(H, 32 * vn)), 256, 0, st>>>((const T*)dz, dpos, B, S, H)));
 }
 
 void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,

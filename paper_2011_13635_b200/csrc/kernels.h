@@ -47,8 +47,14 @@ void launch_loss_reduce(const float* nll, int R, const float* inv_n, float* loss
 // out[n] += sum over rows; N a multiple of the 16-byte vector width, out has room for N floats
 void launch_colsum(bool bf, const void* x, int64_t ld, int rows, int N, float* out,
                    cudaStream_t st);
-void launch_embed_scatter(bool bf, const void* dz, const int* tokens, float* dword, float* dpos,
-                          int rows, int S, int H, int V, cudaStream_t st);
+// The embedding gradients without hot-row atomics and with run-to-run identical bits: counting sort
+// of the rows by token id, one block per token id, batch sum per position.  Needs H / (16 bytes of
+// activation) <= 1024 column threads and V <= 262144.  Scratch: counts [ceil(T/256) * V], total [V],
+// start [V], rank [T], order [T], blocksum [1024], hot [2 + 3 * 2048] (ints), partial [2048 * H] (floats);
+// needs T <= 65536 and H / (16-byte vector) <= 256.  Nine launches.
+void launch_embed_grad_sorted(bool bf, const void* dz, const int* tokens, float* dword, float* dpos, int B, int S,
+                              int H, int V, int* counts, int* total, int* start, int* rank, int* order,
+                              int* blocksum, int* hot, float* partial, cudaStream_t st);
 // t_dev: step count in device memory (incremented here); bc_dev: two floats that receive the bias
 // corrections of this step
 void launch_adam(const AdamChunk* chunks, int n_chunks, float* w, const float* g, float* m, float* v,

@@ -81,6 +81,8 @@ struct Workspace {
   char* z0;
   float* st0;
   char *hm, *ut, *gt, *tm, *dlogits, *dtm, *dgt, *dhm;
+  int *es_counts, *es_total, *es_start, *es_rank, *es_order, *es_blocksum, *es_hot;
+  float* es_partial;  // embedding backward: rows sorted by token id
   int* nsp_rowsrc;                          // NSP head: first-token row of every sequence
   char *cls, *up, *pooled, *dup, *dcls;     // [B,H] each
   float *hst, *logits, *nll, *dtm32;
@@ -144,13 +146,15 @@ int check_arch(const mslt_arch* a) {
     return fail(MSLT_ERR_ARG, "dtype 1 (bf16 tensor-core path) needs head dim 64");
   if (a->dtype != 0 && a->dtype != 1) return fail(MSLT_ERR_ARG, "dtype must be 0 or 1");
   if (a->ffn <= 0 || a->ffn % 64) return fail(MSLT_ERR_ARG, "ffn must be a multiple of 64");
-  if (a->vocab < 2) return fail(MSLT_ERR_ARG, "vocab too small");
+  if (a->vocab < 2 || a->vocab > 262144) return fail(MSLT_ERR_ARG, "vocab must lie in [2, 262144]");
   if (a->init_layers < 1 || a->max_layers < a->init_layers)
     return fail(MSLT_ERR_ARG, "need 1 <= init_layers <= max_layers");
   if (a->max_batch < 1 || a->max_pred < 1) return fail(MSLT_ERR_ARG, "bad batch/pred capacity");
   if (a->max_seq < 8 || a->max_seq % 8 || a->max_seq > 512)
     return fail(MSLT_ERR_ARG, "max_seq must be a multiple of 8 in [8, 512]");
   if (a->max_pos < a->max_seq) return fail(MSLT_ERR_ARG, "max_pos < max_seq");
+  if ((int64_t)a->max_batch * a->max_seq > 65536)
+    return fail(MSLT_ERR_ARG, "max_batch * max_seq must not exceed 65536 tokens");
   if (!(a->ln_eps >= 0.f)) return fail(MSLT_ERR_ARG, "ln_eps must be >= 0");
   if (a->max_trainable < 0 || a->max_trainable > a->max_layers)
     return fail(MSLT_ERR_ARG, "need 0 <= max_trainable <= max_layers");
@@ -250,6 +254,14 @@ void plan_workspace(const mslt_arch& a, const std::vector<Tensor>& tensors, char
   w.layer.resize(trainable_slots(a));
   for (int l = 0; l < trainable_slots(a); l++) take_layer(w.layer[l]);
   w.z0 = take(T * H * E);
+  w.es_counts = (int*)take(((T + 255) / 256) * (int64_t)a.vocab * 4);
+  w.es_total = (int*)take((int64_t)a.vocab * 4);
+  w.es_start = (int*)take((int64_t)a.vocab * 4);
+  w.es_rank = (int*)take(T * 4);
+  w.es_order = (int*)take(T * 4);
+  w.es_blocksum = (int*)take(1024 * 4);
+  w.es_hot = (int*)take((2 + 3 * 2048) * 4);
+  w.es_partial = (float*)take(2048 * H * 4);
   w.st0 = (float*)take(T * 2 * 4);
   w.hm = take(R * H * E); w.ut = take(R * H * E); w.gt = take(R * H * E); w.tm = take(R * H * E);
   w.hst = (float*)take(R * 2 * 4);
@@ -924,8 +936,12 @@ static int step_impl(mslt_ctx* c, const int32_t* d_tokens, const int32_t* d_seq_
   if (full) {
     KL(PC_LN_BWD, 3.0 * T * H * c->esz, launch_ln_bwd(c->bf, dx, w.z0, w.st0, Wv(c, toff(c, -1, "emb.ln.gamma")), w.dz2,
                      G(c, toff(c, -1, "emb.ln.gamma")), G(c, toff(c, -1, "emb.ln.beta")), nullptr, T, H, c->st));
-    KL(PC_OTHER, 1.0 * T * H * c->esz, launch_embed_scatter(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
-                            G(c, toff(c, -1, "emb.pos")), T, S, H, V, c->st));
+    // rows grouped by token id (counting sort), one block per id, batch sum per position: no hot-row
+    // atomics, same bits on every run
+    KL(PC_OTHER, 2.0 * T * H * c->esz, launch_embed_grad_sorted(c->bf, w.dz2, d_tokens, G(c, toff(c, -1, "emb.word")),
+                            G(c, toff(c, -1, "emb.pos")), B, S, H, V, w.es_counts, w.es_total, w.es_start,
+                            w.es_rank, w.es_order, w.es_blocksum, w.es_hot, w.es_partial, c->st));
+    c->launches += 8;
     if (c->a.nsp)
       KL(PC_OTHER, 1.0 * T * H * c->esz, launch_type_grad(c->bf, w.dz2, d_seg, G(c, toff(c, -1, "emb.type")), T, H, c->st));
     TRY(bucket_done(c, c->top_k / group_of(c->a) + 1));

@@ -245,3 +245,23 @@ def test_captured_step_replays_like_eager_steps():
     assert abs(l0 - l1) < 1e-3 * abs(l0)
     assert PT.max_rel(w1, w0) < 1e-3                            # atomics reorder sums, nothing more
     assert PT.max_rel(v1, v0) < 1e-2
+
+
+def test_embedding_gradients_have_the_same_bits_on_every_run():
+    """The embedding backward groups rows by token id in a fixed order and sums positions over the
+    batch without atomics: two runs of the same all-trainable step give identical bits (fp32 path;
+    on the bf16 path the tied decoder's split-k weight gradient, which lands in the same table, is
+    summed with vector reductions, so only the position table is compared there)."""
+    import torch
+    for cfg in (I.scaled(CFG32, trainable=4), I.scaled(CFG16, trainable=4)):
+        got = []
+        for _ in range(2):
+            m, _ = PT.build_pair(cfg, lr=1e-3)
+            d = PT.to_cuda(torch, *I.make_batch(cfg))
+            m.mslt_step(d[0], None, d[2], d[3])
+            got.append((m.mslt_get_grad("emb.pos"), m.mslt_get_grad("emb.word")))
+            m.close()
+        assert np.array_equal(got[0][0], got[1][0])
+        assert np.abs(got[0][0]).max() > 0
+        if cfg.dtype == "fp32":
+            assert np.array_equal(got[0][1], got[1][1])
