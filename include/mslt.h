@@ -329,8 +329,10 @@ int mslt_debug_starve_next_attention(int32_t on);
 /*
  * Measurement hook: how the dtype-1 contraction kernel tiles its output from now on, process
  * wide.  0 (the default): the library chooses; 1: one CTA per 128 x BN tile; 2: a pair of CTAs per
- * 256 x 256 tile wherever the shape allows it.  Results are identical up to summation order; only
- * the speed differs.  Used by the micro-benchmarks to compare the two forms on one shape.
+ * 256 x 256 tile wherever the shape allows it.  Adding 4 to any of these makes the bf16 epilogues
+ * store their rows from registers instead of through shared memory and the copy engine.  Results
+ * are identical up to summation order; only the speed differs.  Used by the micro-benchmarks to
+ * compare the forms on one shape.
  */
 int mslt_debug_set_gemm_variant(int32_t variant);
 

@@ -50,6 +50,8 @@ struct TcParams {
   long long ldd, d_bo, d_bi;
   int d_fp32, accumulate, vec_ok;
   int direct;           // rows of D (and aux) may be stored straight from registers, 32 bytes at a time
+  int tma_store;        // bf16 D leaves through shared memory and tile stores of 32 rows x 64 columns
+  int d_perm[3];        // slots of D's (row, inner-batch, outer-batch) coordinates in its tensor map
   float alpha;
   const float* bias;
   int act;
@@ -139,6 +141,25 @@ __device__ __forceinline__ void row32_store_bf16(bf16* dst, const float2 (&w)[16
                  "r"(h[8 * c + 6]), "r"(h[8 * c + 7])
                  : "memory");
 }
+// The same 32 columns into a 32-row x 128-byte staging tile in the 128-byte swizzle layout of the
+// output's tensor map: row `lane`, 16-byte units 4 * half .. 4 * half + 3, unit u stored at
+// position u ^ (row & 7).  Eight neighbouring lanes hit eight different bank groups.
+__device__ __forceinline__ void row32_stage_bf16(uint32_t tile, int lane, int half, const float2 (&w)[16]) {
+  uint32_t h[16];
+#pragma unroll
+  for (int e = 0; e < 16; e++) {
+    const __nv_bfloat162 t = __float22bfloat162_rn(w[e]);
+    h[e] = *reinterpret_cast<const uint32_t*>(&t);
+  }
+  const uint32_t row = tile + (uint32_t)lane * 128u;
+#pragma unroll
+  for (int c = 0; c < 4; c++) {
+    const uint32_t u = (uint32_t)((4 * half + c) ^ (lane & 7));
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(row + u * 16u), "r"(h[4 * c]), "r"(h[4 * c + 1]),
+                 "r"(h[4 * c + 2]), "r"(h[4 * c + 3])
+                 : "memory");
+  }
+}
 __device__ __forceinline__ void row32_store_f32(float* dst, const float2 (&w)[16], int accumulate) {
   if (accumulate) {
 #pragma unroll
@@ -162,10 +183,12 @@ __device__ __forceinline__ void row32_store_f32(float* dst, const float2 (&w)[16
 // `direct`: this lane's row exists and the whole chunk lies inside the output, so the lane stores
 // its 32 columns itself; otherwise the chunk goes through the staging buffer, which handles ragged
 // edges element by element (every lane of the warp takes the same branch).
+// `tile` != 0: the bf16 result goes into that staging tile (shared-memory address) as half `half`
+// of its 64 columns instead, for a tile store by the caller.
 template <int kMode>
 __device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)[32], const uint4 (&x)[4],
                                           const float* bias_c, uint8_t* stg, int lane, long long zoff,
-                                          int m_warp, int n0, bool direct) {
+                                          int m_warp, int n0, bool direct, uint32_t tile = 0, int half = 0) {
   float2 v[16];
   const float2 al = splat2(p.alpha);
   const float4* b4 = reinterpret_cast<const float4*>(bias_c);
@@ -210,7 +233,8 @@ __device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)
     else stage_store_f32(stg, lane, v, reinterpret_cast<float*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok,
                          p.accumulate);
   } else {
-    if (direct) { if (row_ok) row32_store_bf16(reinterpret_cast<bf16*>(p.D) + off, v); }
+    if (tile) row32_stage_bf16(tile, lane, half, v);
+    else if (direct) { if (row_ok) row32_store_bf16(reinterpret_cast<bf16*>(p.D) + off, v); }
     else stage_store_bf16(stg, lane, v, reinterpret_cast<bf16*>(p.D) + zoff, p.ldd, m_warp, n0, p.M, p.N, p.vec_ok);
   }
 }
@@ -220,7 +244,7 @@ __device__ __forceinline__ void epi_chunk(const TcParams& p, const uint32_t (&a)
 template <int kMode, bool kPair>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-               const TcParams p) {
+               const __grid_constant__ CUtensorMap tmD, const TcParams p) {
   constexpr bool kSoftmax = kMode == EPI_SOFTMAX;
   constexpr bool kHasX = kMode == EPI_RESIDUAL || kMode == EPI_DGELU;
   extern __shared__ uint8_t smem_raw[];
@@ -461,6 +485,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     const int hsel = (warp - FIRST_EPI_WARP) >> 2;    // which of the two warps of the quarter
     uint8_t* stg = staging + (size_t)(warp - FIRST_EPI_WARP) * STAGING_BYTES;
     float* bias_s = reinterpret_cast<float*>(stg + 2048);  // bias of this warp's columns, chunk by chunk
+    float* bias_r = reinterpret_cast<float*>((uint8_t*)bars + 256) + (warp - FIRST_EPI_WARP) * 32;
     uint32_t tile = 0;
     bool ok = true;
     if constexpr (kMode != EPI_GENERIC && !kSoftmax) {
@@ -496,16 +521,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         z_ -= c ? p.batch : 0;
         sp_ += d_sp + c;
       };
+      // This warp's i-th chunk, in units of 32 columns.  The two warps of a quarter interleave
+      // their chunks; with tile stores they interleave pairs of chunks, so that a warp owns whole
+      // 64-column (128-byte) groups.
+      const bool tma_out = p.tma_store != 0;
+      auto ccol = [&](int i) { return tma_out ? 2 * (hsel + 2 * (i >> 1)) + (i & 1) : hsel + 2 * i; };
+      const uint32_t stg_tile = smem_u32(stg);
       // bias values of this warp's columns of tile `nt_`, one value per lane and chunk
       auto fetch_bias = [&](int nt_, float (&b)[4]) {
 #pragma unroll
         for (int i = 0; i < 4; i++) {
-          const int n = nt_ * p.bn + (hsel + 2 * i) * 32 + lane;
+          const int n = nt_ * p.bn + ccol(i) * 32 + lane;
           b[i] = (i < nch && p.bias && n < p.N) ? p.bias[n] : 0.f;
         }
       };
       float bnext[4];
-      if (w_first < p.total_work) {
+      if (w_first < p.total_work && !tma_out) {
         fetch_bias(nt, bnext);
 #pragma unroll
         for (int i = 0; i < 4; i++) bias_s[i * 32 + lane] = bnext[i];
@@ -522,7 +553,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int n_base = nt * p.bn;
         const float* bias_t = bias_s + (tile & 1) * 128;
         const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + acc * 256;
-        auto chunk_n0 = [&](int i) { return n_base + (hsel + 2 * i) * 32; };
+        auto chunk_n0 = [&](int i) { return n_base + ccol(i) * 32; };
         auto chunk_ok = [&](int i) { return i < nch && chunk_n0(i) < p.N; };
         auto prefetch_x = [&](int i, uint4 (&x)[4]) {
           if (kHasXf && row_ok) {
@@ -534,7 +565,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         // the next work item and its bias (the loads travel while this tile is worked on)
         int nt2 = nt, mt2 = mt, z2 = z, sp2 = sp;
         advance(nt2, mt2, z2, sp2);
-        const bool more = w + w_step < p.total_work;
+        const bool more = w + w_step < p.total_work && !tma_out;  // (of interest to the bias hand-over only)
         if (more) fetch_bias(nt2, bnext);
         uint4 x[4];
         const bool c0ok = chunk_ok(0);
@@ -557,7 +588,35 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             if (has_next) prefetch_x(i + 1, x);
           }
           const int n0 = chunk_n0(i);
-          epi_chunk<kMode>(p, a, xc, bias_t + i * 32, stg, lane, zoff, m_warp, n0, p.direct && n0 + 32 <= p.N);  // warp-uniform
+          if (tma_out) {
+            // an even chunk opens a 64-column group: the tile store of the previous group must
+            // have read the staging tile; an odd chunk, or the last one, closes it
+            if (!(i & 1)) {
+              if (lane == 0) tma_store_wait_read();
+              __syncwarp();
+            }
+            // The staging buffer holds the output tile, so the chunk's bias comes straight from
+            // global memory (32 floats that every lane reads alike: one L1 line), or, for a
+            // ragged chunk or no bias at all, from 32 floats of scratch.
+            const float* bias_c = p.bias + n0;
+            if (!p.bias || n0 + 32 > p.N) {
+              __syncwarp();
+              bias_r[lane] = (p.bias && n0 + lane < p.N) ? p.bias[n0 + lane] : 0.f;
+              __syncwarp();
+              bias_c = bias_r;
+            }
+            epi_chunk<kMode>(p, a, xc, bias_c, stg, lane, zoff, m_warp, n0, p.direct != 0, stg_tile, i & 1);
+            if ((i & 1) || !has_next) {
+              fence_proxy_async_smem();
+              __syncwarp();
+              if (lane == 0 && m_warp < p.M) {
+                auto slot = [&](int sl) { return p.d_perm[0] == sl ? m_warp : (p.d_perm[1] == sl ? zi : zo); };
+                tma_store_4d(&tmD, stg_tile, n0 - (i & 1) * 32, slot(1), slot(2), slot(3));
+              }
+            }
+          } else {
+            epi_chunk<kMode>(p, a, xc, bias_t + i * 32, stg, lane, zoff, m_warp, n0, p.direct && n0 + 32 <= p.N);  // warp-uniform
+          }
         };
         if (c0ok && kHasXf) {
           // the flavours with a row-shaped extra operand have no registers to spare for a second
@@ -565,7 +624,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           uint32_t ra[32];
           for (int i = 0;; i++) {
             const bool v1 = chunk_ok(i + 1);
-            tc_ld32_issue(trow + (hsel + 2 * i) * 32, ra);
+            tc_ld32_issue(trow + ccol(i) * 32, ra);
             tc_ld32_wait(ra);
             if (!v1) release_acc();
             work(ra, i, v1);
@@ -573,16 +632,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
           }
         } else if (c0ok) {
           uint32_t ra[32], rb[32];
-          tc_ld32_issue(trow + hsel * 32, ra);
+          tc_ld32_issue(trow + ccol(0) * 32, ra);
           for (int i = 0;; i += 2) {
             const bool v1 = chunk_ok(i + 1);
             tc_ld32_wait(ra);
-            if (v1) tc_ld32_issue(trow + (hsel + 2 * (i + 1)) * 32, rb); else release_acc();
+            if (v1) tc_ld32_issue(trow + ccol(i + 1) * 32, rb); else release_acc();
             work(ra, i, v1);
             if (!v1) break;
             const bool v2 = chunk_ok(i + 2);
             tc_ld32_wait(rb);
-            if (v2) tc_ld32_issue(trow + (hsel + 2 * (i + 2)) * 32, ra); else release_acc();
+            if (v2) tc_ld32_issue(trow + ccol(i + 2) * 32, ra); else release_acc();
             work(rb, i + 1, v2);
             if (!v2) break;
           }
@@ -826,6 +885,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
       }
       }
     }
+    // tile stores read this CTA's shared memory: they end before the CTA does
+    if (p.tma_store && lane == 0) tma_store_wait_all();
   }
 
   tc_fence_before();
@@ -851,7 +912,8 @@ void gemm_tc_starve_next(int on) { g_starve_next.store(on ? 1 : 0); }
 // Measurement hook (mslt_debug_set_gemm_variant): 0 = automatic choice, 1 = one CTA per tile,
 // 2 = a CTA pair per 256 x 256 tile wherever the shape allows it.
 static std::atomic<int> g_tile_variant{0};
-void gemm_tc_set_variant(int v) { g_tile_variant.store(v); }
+static std::atomic<int> g_store_variant{0};  // 1 = no tile stores (bit 2 of the hook's argument)
+void gemm_tc_set_variant(int v) { g_tile_variant.store(v & 3); g_store_variant.store((v >> 2) & 1); }
 
 namespace {
 // Per-device facts and one-time set-up, indexed by device ordinal (a process may drive several GPUs).
@@ -947,7 +1009,9 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
     return MSLT_ERR_ARG;
   }
   const int stage_bytes = (pair ? 2 : 1) * (A_STAGE_BYTES + (pair ? p.bn / 2 : p.bn) * BK * 2);  // per CTA
-  const int book_bytes = 256 + (d.act == 3 ? 64 + 2 * NUM_EPI_WARPS * 32 * 4 : 0);
+  // barriers, then the softmax epilogue's exchange area or the 32 floats per epilogue warp that
+  // hold the bias of a ragged chunk when the staging buffers carry output tiles
+  const int book_bytes = 256 + (d.act == 3 ? 64 + 2 * NUM_EPI_WARPS * 32 * 4 : NUM_EPI_WARPS * 32 * 4);
   int stages = (smem_optin - NUM_EPI_WARPS * STAGING_BYTES - 1024 - book_bytes) / stage_bytes;
   if (stages > MAX_STAGES) stages = MAX_STAGES;
   if (stages < 2) { snprintf(err, 256, "gemm: not enough shared memory"); return MSLT_ERR_CUDA; }
@@ -999,7 +1063,28 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   else if (d.act == 1 && !d.residual) mode = d.aux ? EPI_GELU_AUX : EPI_GELU;
   else if (d.act == 2 && d.aux && !d.residual && x_ok) mode = EPI_DGELU;
 
-  typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const TcParams);
+  // Tile stores for the bf16 flavours: the output leaves through the copy engine as whole
+  // 128-byte lines.  Row stores from registers (2 x 32 bytes per lane and chunk) were measured to
+  // hold up the operand loads that share the SM's path to L2: 16384 x 2304 x 768 took 51.7 us with
+  // them, 41.3 us with the stores left out, and a load stream beside such stores fell from 68 to
+  // 12 bytes per clock per SM while beside copy-engine stores it kept 68.
+  MapVal md;
+  md.map = ma.map;
+  p.tma_store = 0;
+  if ((mode == EPI_STORE || mode == EPI_RESIDUAL || mode == EPI_GELU || mode == EPI_DGELU ||
+       (mode == EPI_GELU_AUX && p.direct && d.N % 32 == 0)) &&
+      p.bn >= 128 && p.vec_ok && d.N % 8 == 0 &&  // a tile store was seen to write whole 16-byte pieces
+      g_store_variant.load() != 1) {
+    char ignored[256];
+    if (get_map(d.D, d.M, d.N, d.ldd, 1, d.d_bo, d.d_bi, d.hdiv, nb, 32, &md, ignored) == 0) {
+      p.tma_store = 1;
+      for (int i = 0; i < 3; i++) p.d_perm[i] = md.perm[i];
+    } else {
+      md.map = ma.map;
+    }
+  }
+
+  typedef void (*KernelFn)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const TcParams);
   static const KernelFn kernels[EPI_COUNT][2] = {
       {gemm_tc_kernel<EPI_STORE, false>, gemm_tc_kernel<EPI_STORE, true>},
       {gemm_tc_kernel<EPI_RESIDUAL, false>, gemm_tc_kernel<EPI_RESIDUAL, true>},
@@ -1039,7 +1124,7 @@ int gemm_tc_launch(const mslt_gemm_desc& d, int* status, cudaStream_t st, char* 
   } else {
     cfg.gridDim = dim3(p.total_work < num_sms ? p.total_work : num_sms);
   }
-  cudaError_t e = cudaLaunchKernelEx(&cfg, fn, ma.map, mb.map, p);
+  cudaError_t e = cudaLaunchKernelEx(&cfg, fn, ma.map, mb.map, md.map, p);
   if (e != cudaSuccess) { snprintf(err, 256, "gemm: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
   return 0;
 }

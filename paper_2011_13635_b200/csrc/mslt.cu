@@ -1239,7 +1239,7 @@ int mslt_debug_starve_next_gemm(int32_t on) {
 }
 
 int mslt_debug_set_gemm_variant(int32_t variant) {
-  if (variant < 0 || variant > 2) return fail(MSLT_ERR_ARG, "variant must be 0, 1 or 2");
+  if (variant < 0 || (variant & 3) > 2 || variant > 6) return fail(MSLT_ERR_ARG, "variant must be 0, 1 or 2, plus 4 or not");
   gemm_tc_set_variant(variant);
   return 0;
 }

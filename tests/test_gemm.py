@@ -115,6 +115,25 @@ def test_epilogues(dtype):
     _run(dtype, 136, 200, 1000, "mn", "mn", d_fp32=True, accumulate=True)
 
 
+@pytest.mark.parametrize("variant", [0, 1, 2, 4, 6], ids=["auto", "single", "pair", "auto-rowstores", "pair-rowstores"])
+def test_bf16_epilogues_over_several_wide_tiles(variant):
+    """Every bf16 epilogue flavour on outputs of several 256-wide tiles with ragged last tiles, in
+    each tiling form and with both ways of storing the output (through shared memory and the copy
+    engine, or row segments from registers)."""
+    from paper_2011_13635_b200 import binding as Bd
+    assert Bd.lib.mslt_debug_set_gemm_variant(variant) == 0
+    try:
+        _run(1, 700, 840, 200, "k", "k", bias=True)
+        _run(1, 700, 840, 200, "k", "k", bias=True, act=1, aux_out=True)
+        _run(1, 700, 832, 136, "k", "k", bias=True, act=1)
+        _run(1, 520, 800, 72, "k", "mn", act=2)
+        _run(1, 520, 800, 72, "k", "mn", bias=True, residual=True, alpha=0.125)
+        _run(1, 300, 1037, 192, "k", "k", bias=True)           # row pitch 1040: columns end inside a chunk
+        _run(1, 33, 168, 64, "mn", "k", bias=True, act=1)      # one 128-wide tile and a ragged second one
+    finally:
+        Bd.lib.mslt_debug_set_gemm_variant(0)
+
+
 def test_bf16_long_contraction_split_k():
     """Weight-gradient shape: small output, long contraction, partial sums added in fp32."""
     _run(1, 768, 256, 4096, "mn", "mn", d_fp32=True, accumulate=True)
