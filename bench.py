@@ -235,9 +235,9 @@ def aggregate(ms_local: float, batch_per_rank: int, steps: int, world: int, dist
 
 # DRAM bytes (read + write) per launch of the contraction kernel from ncu captures of single launches
 # of the four forward products of a BERT-Base layer (profiles/gemm_tc_kernel_frozen_layer_shapes_16384.md):
-# QKV 53.0 MB, out-proj 53.6 MB, FFN1 80.9 MB, FFN2 144.3 MB; the bench line carries their mean, which
+# QKV 47.7 MB, out-proj 53.1 MB, FFN1 73.6 MB, FFN2 144.2 MB; the bench line carries their mean, which
 # holds for the BERT-Base configurations only.  None once the kernel changes.
-GEMM_DRAM_BYTES_PER_LAUNCH = {"base": 82.9e6}
+GEMM_DRAM_BYTES_PER_LAUNCH = {"base": 79.7e6}
 
 
 def gemm_peaks(peaks, clocks):
