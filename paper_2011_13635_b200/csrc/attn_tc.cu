@@ -362,59 +362,49 @@ attn_fwd_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__
 
 // ---- forward for rows of 129..512 keys -----------------------------------------------------------
 // A work item is (sequence, head, tile of 128 queries); the keys come in blocks of 128.  The scores
-// of a row do not fit tensor memory next to the context, so the item runs two passes over the key
-// blocks: pass 1 forms the row maximum and the sum of exponentials (S = Q K_j^T only), pass 2
-// forms the scores again, writes P_j = exp(.)/sum as bf16 and accumulates C += P_j V_j.  The
-// second score product costs the tensor pipe little; what it buys is an exact softmax with no
-// rescaling of the context, and probabilities that can be stored as they are.
-// The two softmax groups take alternate score accumulators of the same item (a thread owns one
-// query row in its group's blocks) and exchange their partial (max, sum) between the passes.
-constexpr int AL_KV_STAGES = 4;
-constexpr int AL_KV_BYTES = 2 * AT_TILE_BYTES;   // K block and V block: 32 KB
+// of a row do not fit tensor memory next to the context, so an item runs two passes over the key
+// blocks.  When the probabilities are wanted: pass 1 forms the row maximum and the sum of
+// exponentials (S = Q K_j^T only), pass 2 forms the scores again, writes P_j = exp(.)/sum as bf16
+// and accumulates C += P_j V_j: an exact softmax with no rescaling of the context, and
+// probabilities that can be stored as they are.  When they are not wanted (a frozen layer), pass 1
+// forms the maximum only, pass 2 uses exp(s - max) as it is, sums it on the way, and the context
+// is divided by the sum at the end: half the exponentials.
+// Each of the two softmax groups owns every second item of the CTA, whole: its own Q tile, ring of
+// K / V tiles, score and context accumulators, P block, producer thread and MMA-issuing thread.  A
+// thread owns one query row of its group's item through all key blocks, so nothing is exchanged
+// between the groups, and the waits of one item (loads, the P hand-over, the last second product,
+// the context store) are covered by the other item's arithmetic.  Measured on the earlier form, in
+// which the two groups shared one item: 21 k cycles per item of which 8 k were exponentials.
+constexpr int AL_THREADS = NUM_THREADS + 64;     // warps 10 and 11: MMA issuer and producer of group 1
+constexpr int AL_RING = 3;                       // 16 KB tiles (a K block or a V block) per group
 constexpr int AL_P_BYTES = 2 * AT_TILE_BYTES;    // P_j as an MMA operand: 32 KB
+constexpr int AL_BARS_PER_GROUP = 4 + 2 * AL_RING + 6;
+constexpr long long AL_GROUP_SKEW_CYCLES = 2000;
 
-__global__ void __launch_bounds__(NUM_THREADS, 1)
+__global__ void __launch_bounds__(AL_THREADS, 1)
 attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                      const __grid_constant__ CUtensorMap tmV, const AttnParams p) {
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-  uint8_t* q_smem = smem;                                   // two Q tiles, by item parity
-  uint8_t* kv_smem = q_smem + 2 * AT_TILE_BYTES;            // ring of K/V blocks
-  uint8_t* p_smem = kv_smem + AL_KV_STAGES * AL_KV_BYTES;   // one P block
-  uint8_t* staging = p_smem + AL_P_BYTES;
-  float2* xstat = (float2*)(staging + NUM_EPI_WARPS * AT_STAGING);  // [2 items][2 groups][128 rows] (max, sum)
-  uint64_t* bars = (uint64_t*)(xstat + 2 * 2 * 128);
-  uint64_t* qfull_bar = bars;                       // [2]
-  uint64_t* qempty_bar = bars + 2;                  // [2]
-  uint64_t* kvfull_bar = bars + 4;                  // [AL_KV_STAGES]
-  uint64_t* kvempty_bar = bars + 4 + AL_KV_STAGES;  // [AL_KV_STAGES]
-  uint64_t* sfull_bar = bars + 4 + 2 * AL_KV_STAGES;       // [2] scores of the group's next block complete
-  uint64_t* sempty_bar = sfull_bar + 2;                    // [2] read by the group
-  uint64_t* pready_bar = sfull_bar + 4;                    // P block in shared memory
-  uint64_t* pfree_bar = sfull_bar + 5;                     // second product has read it
-  uint64_t* ofull_bar = sfull_bar + 6;                     // context of the item complete
-  uint64_t* oempty_bar = sfull_bar + 7;                    // read by both groups
-  uint64_t* x_bar = sfull_bar + 8;                         // partial row statistics of both groups written
-  uint32_t* tmem_slot = (uint32_t*)(sfull_bar + 9);
+  uint8_t* q_smem = smem;                                        // [group] Q tile
+  uint8_t* ring_smem = q_smem + 2 * AT_TILE_BYTES;               // [group][AL_RING] K or V tile
+  uint8_t* p_smem = ring_smem + 2 * AL_RING * AT_TILE_BYTES;     // [group] P block
+  uint8_t* staging = p_smem + 2 * AL_P_BYTES;
+  uint64_t* bars = (uint64_t*)(staging + NUM_EPI_WARPS * AT_STAGING);
+  uint32_t* tmem_slot = (uint32_t*)(bars + 2 * AL_BARS_PER_GROUP);
   volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   if (threadIdx.x == 0) {
-    for (int a = 0; a < 2; a++) {
-      mbar_init(smem_u32(&qfull_bar[a]), 1);
-      mbar_init(smem_u32(&qempty_bar[a]), 1);
-      mbar_init(smem_u32(&sfull_bar[a]), 1);
-      mbar_init(smem_u32(&sempty_bar[a]), AT_GROUP_WARPS);
+    for (int g = 0; g < 2; g++) {
+      uint64_t* b = bars + g * AL_BARS_PER_GROUP;
+      for (int a = 0; a < 2 + 2 * AL_RING + 1; a++) mbar_init(smem_u32(&b[a]), 1);  // qfull, qempty, tfull[], tempty[], sfull
+      mbar_init(smem_u32(&b[2 + 2 * AL_RING + 1]), AT_GROUP_WARPS);  // sempty
+      mbar_init(smem_u32(&b[2 + 2 * AL_RING + 2]), AT_GROUP_WARPS);  // pready
+      mbar_init(smem_u32(&b[2 + 2 * AL_RING + 3]), 1);               // pfree
+      mbar_init(smem_u32(&b[2 + 2 * AL_RING + 4]), 1);               // ofull
+      mbar_init(smem_u32(&b[2 + 2 * AL_RING + 5]), AT_GROUP_WARPS);  // oempty
     }
-    for (int a = 0; a < AL_KV_STAGES; a++) {
-      mbar_init(smem_u32(&kvfull_bar[a]), 1);
-      mbar_init(smem_u32(&kvempty_bar[a]), 1);
-    }
-    mbar_init(smem_u32(pready_bar), AT_GROUP_WARPS);
-    mbar_init(smem_u32(pfree_bar), 1);
-    mbar_init(smem_u32(ofull_bar), 1);
-    mbar_init(smem_u32(oempty_bar), NUM_EPI_WARPS);
-    mbar_init(smem_u32(x_bar), NUM_EPI_WARPS);
     *abort_flag = 0;
     *reinterpret_cast<volatile long long*>(abort_flag + 1) = p.wait_limit;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -434,90 +424,119 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
   // Keys at or beyond the sequence's length have probability 0: an item covers only the
   // ceil(len / 128) key blocks that hold valid keys, and a query tile that lies wholly in the
   // padding is not computed at all (its context rows, which nothing may depend on, are zeroed).
-  // Every role derives the same counts from seq_lens; `ip` counts the items actually computed.
+  // Every role derives the same counts from seq_lens.
   auto item_len = [&](int zo) {
     int len = p.seq_lens ? p.seq_lens[zo] : p.S;
     return min(max(len, 1), p.S);
   };
   const int n_my = ((int)blockIdx.x < p.items) ? (p.items - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-  // Per item there are 2 * nkb score products, numbered t = 0, 1, ... over the CTA's whole run; the
-  // accumulator and the softmax group of product t are t & 1, its K/V stage t % AL_KV_STAGES.
+  // Which group this thread serves, and that group's barriers.  Running counts per group: ig items,
+  // tt ring tiles, sp score products, pv second products; each barrier's phase is the parity of
+  // the count it is used by.
+  const int g = warp == 0 ? 0 : (warp == 1 ? 0 : (warp >= 10 ? 1 : (warp - 2) >> 2));
+  uint64_t* gb = bars + g * AL_BARS_PER_GROUP;
+  const uint32_t qfull = smem_u32(&gb[0]), qempty = smem_u32(&gb[1]);
+  const uint32_t tfull0 = smem_u32(&gb[2]), tempty0 = smem_u32(&gb[2 + AL_RING]);
+  const uint32_t sfull = smem_u32(&gb[2 + 2 * AL_RING]), sempty = smem_u32(&gb[2 + 2 * AL_RING + 1]);
+  const uint32_t pready = smem_u32(&gb[2 + 2 * AL_RING + 2]), pfree = smem_u32(&gb[2 + 2 * AL_RING + 3]);
+  const uint32_t ofull = smem_u32(&gb[2 + 2 * AL_RING + 4]), oempty = smem_u32(&gb[2 + 2 * AL_RING + 5]);
+  uint8_t* my_q = q_smem + g * AT_TILE_BYTES;
+  uint8_t* my_ring = ring_smem + (size_t)g * AL_RING * AT_TILE_BYTES;
+  uint8_t* my_p = p_smem + (size_t)g * AL_P_BYTES;
+  const bool want_p = p.P != nullptr;
+  // Tiles of an item in the order the MMA thread uses them: pass 1: K_0 .. K_{n-1}; pass 2: K_0, then
+  // (K_j, V_{j-1}) for j = 1 .. n-1, then V_{n-1} (the scores of block j are issued before the second
+  // product of block j - 1, which has to wait for that block's probabilities).
 
-  if (warp == 0 && lane == 0 && !p.starve) {
-    // ------------------------------- TMA producer -------------------------------
+  if ((warp == 0 || warp == 11) && lane == 0 && !p.starve) {
+    // ------------------------------- TMA producer of group g -------------------------------
     bool ok = true;
-    uint32_t t = 0, ip = 0;
-    for (int i = 0; i < n_my && ok; i++) {
+    uint32_t tt = 0, ig = 0;
+    for (int i = g; i < n_my && ok; i += 2) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
       const int qt = w / nzh, zh = w - qt * nzh;  // query tile slowest: tiles that may be padding come last
       const int zo = zh / p.heads, zi = zh - zo * p.heads;
       const int len = item_len(zo);
       if (qt * 128 >= len) continue;
       const int nkb = (len + 127) >> 7;
-      const uint32_t qb = ip & 1, quse = ip >> 1;
-      ip++;
-      if (!mbar_wait(smem_u32(&qempty_bar[qb]), (quse & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      if (!mbar_wait(qempty, (ig & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+      ig++;
       int c[4];
       c[0] = 0; c[p.q_perm[0]] = qt * 128; c[p.q_perm[1]] = zi; c[p.q_perm[2]] = zo;
-      mbar_expect_tx(smem_u32(&qfull_bar[qb]), AT_TILE_BYTES);
-      tma_load_4d(smem_u32(q_smem + qb * AT_TILE_BYTES), &tmQ, smem_u32(&qfull_bar[qb]), c[0], c[1], c[2], c[3]);
-      for (int pass = 0; pass < 2 && ok; pass++)
-        for (int j = 0; j < nkb; j++, t++) {
-          const uint32_t s = t % AL_KV_STAGES, round = t / AL_KV_STAGES;
-          if (!mbar_wait(smem_u32(&kvempty_bar[s]), (round & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
-          const uint32_t fb = smem_u32(&kvfull_bar[s]);
-          const uint32_t dst = smem_u32(kv_smem + (size_t)s * AL_KV_BYTES);
-          mbar_expect_tx(fb, pass == 0 ? AT_TILE_BYTES : 2 * AT_TILE_BYTES);
-          c[0] = 0; c[p.k_perm[0]] = j * 128; c[p.k_perm[1]] = zi; c[p.k_perm[2]] = zo;
-          tma_load_4d(dst, &tmK, fb, c[0], c[1], c[2], c[3]);
-          if (pass == 1) {
-            c[0] = 0; c[p.v_perm[0]] = j * 128; c[p.v_perm[1]] = zi; c[p.v_perm[2]] = zo;
-            tma_load_4d(dst + AT_TILE_BYTES, &tmV, fb, c[0], c[1], c[2], c[3]);
-          }
+      mbar_expect_tx(qfull, AT_TILE_BYTES);
+      tma_load_4d(smem_u32(my_q), &tmQ, qfull, c[0], c[1], c[2], c[3]);
+      for (int idx = 0; idx < 3 * nkb; idx++, tt++) {
+        // which block, and K or V
+        int j = idx;
+        bool is_v = false;
+        if (idx >= nkb) {
+          const int k = idx - nkb;
+          if (k == 0) j = 0;
+          else if (k == 2 * nkb - 1) { j = nkb - 1; is_v = true; }
+          else if (k & 1) j = (k + 1) >> 1;
+          else { j = (k >> 1) - 1; is_v = true; }
         }
+        const uint32_t slot = tt % AL_RING, round = tt / AL_RING;
+        if (!mbar_wait(tempty0 + slot * 8, (round & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+        const uint32_t fb = tfull0 + slot * 8;
+        mbar_expect_tx(fb, AT_TILE_BYTES);
+        const int* perm = is_v ? p.v_perm : p.k_perm;
+        c[0] = 0; c[1] = 0; c[2] = 0; c[3] = 0;
+        c[perm[0]] = j * 128; c[perm[1]] = zi; c[perm[2]] = zo;
+        tma_load_4d(smem_u32(my_ring + (size_t)slot * AT_TILE_BYTES), is_v ? &tmV : &tmK, fb, c[0], c[1], c[2], c[3]);
+      }
     }
     if (!ok || *abort_flag) {  // give the copies in flight time to land before the CTA leaves
       const long long t0 = now_cycles();
       while (now_cycles() - t0 < 4000000ll) {}
     }
-  } else if (warp == 1 && lane == 0) {
-    // ------------------------------- MMA issuer -------------------------------
+  } else if ((warp == 1 || warp == 10) && lane == 0) {
+    // ------------------------------- MMA issuer of group g -------------------------------
     bool ok = true;
     const uint32_t hi = (uint32_t)(make_smem_desc(0, 16) >> 32);
     const uint32_t lbo_mn_lo = (uint32_t)make_smem_desc(0, 64 * BK * 2);
-    const uint32_t p_lo = (uint32_t)make_smem_desc(smem_u32(p_smem), 16);
-    uint32_t t = 0, u = 0, ip = 0;  // score products, second products and items so far
-    for (int i = 0; i < n_my && ok; i++) {
+    const uint32_t p_lo = (uint32_t)make_smem_desc(smem_u32(my_p), 16);
+    const uint32_t q_lo = (uint32_t)make_smem_desc(smem_u32(my_q), 16);
+    const uint32_t s_tmem = tmem_base + (uint32_t)g * 128, o_tmem = tmem_base + AT_O_COL + (uint32_t)g * 64;
+    uint32_t tt = 0, sp = 0, pv = 0, ig = 0;
+    if (g == 1) {
+      // The two groups do the same work at the same pace: started together they would want the
+      // exponential unit at the same moments and leave it idle at the same moments.  Half a block
+      // period of head start for group 0 keeps them out of step.
+      const long long t0 = now_cycles();
+      while (now_cycles() - t0 < AL_GROUP_SKEW_CYCLES) {}
+    }
+    for (int i = g; i < n_my && ok; i += 2) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
-      const int qt = w / nzh, zh = w - qt * nzh;  // query tile slowest: tiles that may be padding come last
+      const int qt = w / nzh, zh = w - qt * nzh;
       const int len = item_len(zh / p.heads);
       if (qt * 128 >= len) continue;
       const int nkb = (len + 127) >> 7;
-      const uint32_t qb = ip & 1, quse = ip >> 1, ipar = ip & 1;
-      ip++;
-      if (!mbar_wait(smem_u32(&qfull_bar[qb]), quse & 1, abort_flag, p.status)) { ok = false; break; }
-      const uint32_t q_lo = (uint32_t)make_smem_desc(smem_u32(q_smem + qb * AT_TILE_BYTES), 16);
-      auto issue_scores = [&](uint32_t tt) -> bool {
-        const uint32_t s = tt % AL_KV_STAGES, round = tt / AL_KV_STAGES, b = tt & 1, use = tt >> 1;
-        if (!mbar_wait(smem_u32(&kvfull_bar[s]), round & 1, abort_flag, p.status)) return false;
-        if (!mbar_wait(smem_u32(&sempty_bar[b]), (use & 1) ^ 1, abort_flag, p.status)) return false;
+      if (!mbar_wait(qfull, ig & 1, abort_flag, p.status)) { ok = false; break; }
+      auto issue_scores = [&]() -> bool {  // S = Q K^T with the K tile in ring position tt
+        const uint32_t slot = tt % AL_RING, round = tt / AL_RING;
+        if (!mbar_wait(tfull0 + slot * 8, round & 1, abort_flag, p.status)) return false;
+        if (!mbar_wait(sempty, (sp & 1) ^ 1, abort_flag, p.status)) return false;
         tc_fence_after();
-        const uint32_t k_lo = (uint32_t)make_smem_desc(smem_u32(kv_smem + (size_t)s * AL_KV_BYTES), 16);
+        const uint32_t k_lo = (uint32_t)make_smem_desc(smem_u32(my_ring + (size_t)slot * AT_TILE_BYTES), 16);
 #pragma unroll
         for (int k = 0; k < BK / UMMA_K; k++) {
           const uint64_t ad = ((uint64_t)hi << 32) | (q_lo + k * (UMMA_K * 2 / 16));
           const uint64_t bd = ((uint64_t)hi << 32) | (k_lo + k * (UMMA_K * 2 / 16));
-          tc_mma(tmem_base + b * 128, ad, bd, p.idesc_s, k > 0 ? 1u : 0u);
+          tc_mma(s_tmem, ad, bd, p.idesc_s, k > 0 ? 1u : 0u);
         }
-        tc_commit(smem_u32(&sfull_bar[b]));
+        tc_commit(sfull);
+        tc_commit(tempty0 + slot * 8);  // the K tile is free once the product has completed
+        tt++; sp++;
         return true;
       };
-      auto issue_pv = [&](uint32_t tt, int j) -> bool {  // C (+)= P_j V_j; V_j sits in the stage of product tt
-        if (!mbar_wait(smem_u32(pready_bar), u & 1, abort_flag, p.status)) return false;
-        if (j == 0 && !mbar_wait(smem_u32(oempty_bar), ipar ^ 1, abort_flag, p.status)) return false;
+      auto issue_pv = [&](int j) -> bool {  // C (+)= P_j V_j with the V tile in ring position tt
+        const uint32_t slot = tt % AL_RING, round = tt / AL_RING;
+        if (!mbar_wait(pready, pv & 1, abort_flag, p.status)) return false;
+        if (j == 0 && !mbar_wait(oempty, (ig & 1) ^ 1, abort_flag, p.status)) return false;
+        if (!mbar_wait(tfull0 + slot * 8, round & 1, abort_flag, p.status)) return false;
         tc_fence_after();
-        const uint32_t s = tt % AL_KV_STAGES;
-        const uint32_t sv = smem_u32(kv_smem + (size_t)s * AL_KV_BYTES + AT_TILE_BYTES);
+        const uint32_t sv = smem_u32(my_ring + (size_t)slot * AT_TILE_BYTES);
         const uint32_t v_lo = lbo_mn_lo | ((sv & 0x3FFFFu) >> 4);
 #pragma unroll
         for (int kb = 0; kb < 2; kb++)
@@ -525,74 +544,70 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           for (int k = 0; k < BK / UMMA_K; k++) {
             const uint64_t ad = ((uint64_t)hi << 32) | (p_lo + kb * (AT_TILE_BYTES / 16) + k * (UMMA_K * 2 / 16));
             const uint64_t bd = ((uint64_t)hi << 32) | (v_lo + kb * (AT_TILE_BYTES / 2 / 16) + k * (UMMA_K * 128 / 16));
-            tc_mma(tmem_base + AT_O_COL, ad, bd, p.idesc_o, (j > 0 || kb > 0 || k > 0) ? 1u : 0u);
+            tc_mma(o_tmem, ad, bd, p.idesc_o, (j > 0 || kb > 0 || k > 0) ? 1u : 0u);
           }
-        tc_commit(smem_u32(pfree_bar));
-        tc_commit(smem_u32(&kvempty_bar[s]));
-        u++;
+        tc_commit(pfree);
+        tc_commit(tempty0 + slot * 8);
+        tt++; pv++;
         return true;
       };
-      // pass 1: scores only; the K block is free as soon as its product has completed
-      for (int j = 0; j < nkb && ok; j++, t++) {
-        ok = issue_scores(t);
-        if (ok) tc_commit(smem_u32(&kvempty_bar[t % AL_KV_STAGES]));
+      for (int j = 0; j < nkb && ok; j++) ok = issue_scores();  // pass 1
+      if (ok) ok = issue_scores();                                 // pass 2
+      for (int j = 1; j < nkb && ok; j++) {
+        ok = issue_scores();
+        if (ok && j == nkb - 1) tc_commit(qempty);  // the last product that reads Q has been issued
+        if (ok) ok = issue_pv(j - 1);
       }
-      // pass 2: the second product of block j - 1 is issued after the scores of block j
-      for (int j = 0; j < nkb && ok; j++, t++) {
-        ok = issue_scores(t);
-        if (ok && j > 0) ok = issue_pv(t - 1, j - 1);
-      }
-      if (ok) ok = issue_pv(t - 1, nkb - 1);
-      if (ok) {
-        tc_commit(smem_u32(ofull_bar));
-        tc_commit(smem_u32(&qempty_bar[qb]));
-      }
+      if (ok && nkb == 1) tc_commit(qempty);
+      if (ok) ok = issue_pv(nkb - 1);
+      if (ok) tc_commit(ofull);
+      ig++;
     }
     if (!ok || *abort_flag) {
-      tc_commit(smem_u32(&sfull_bar[0]));
+      tc_commit(sfull);
       const long long t0 = now_cycles();
       while (now_cycles() - t0 < 2000000ll) {}
     }
-  } else if (warp >= 2) {
-    // ------------------------------- softmax groups -------------------------------
+  } else if (warp >= 2 && warp < 2 + NUM_EPI_WARPS) {
+    // ------------------------------- softmax group g -------------------------------
     const int q = warp & 3;
-    const int g = (warp - 2) >> 2;
     uint8_t* stg = staging + (size_t)(warp - 2) * AT_STAGING;
     const int r = q * 32 + lane;
     const float sl2 = p.scale * 1.4426950408889634f;
     const float2 k2 = splat2(sl2);
     bool ok = true;
-    uint32_t t = 0, u = 0, ip = 0;
+    uint32_t sp = 0, pv = 0, ig = 0;
     const uint32_t trow = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)g * 128;
-    for (int i = 0; i < n_my && ok; i++) {
+    const uint32_t orow = tmem_base + ((uint32_t)(q * 32) << 16) + AT_O_COL + (uint32_t)g * 64;
+    for (int i = g; i < n_my && ok; i += 2) {
       const int w = (int)blockIdx.x + i * (int)gridDim.x;
-      const int qt = w / nzh, zh = w - qt * nzh;  // query tile slowest: tiles that may be padding come last
+      const int qt = w / nzh, zh = w - qt * nzh;
       const int zo = zh / p.heads, zi = zh - zo * p.heads;
       const int len = item_len(zo);
       float2 v[4][16];
       bf16* cg = p.C + zo * p.c_bo + zi * p.c_bi + (long long)qt * 128 * p.c_ld;
-      bf16* pg = p.P ? p.P + zo * p.p_bo + zi * p.p_bi + (long long)qt * 128 * p.S : nullptr;
+      bf16* pg = want_p ? p.P + zo * p.p_bo + zi * p.p_bi + (long long)qt * 128 * p.S : nullptr;
       if (qt * 128 >= len) {
         // a query tile in the padding: zero context rows (finite, so that masked reads stay harmless)
 #pragma unroll
         for (int e = 0; e < 16; e++) v[0][e] = make_float2(0.f, 0.f);
-        stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, g * 32, p.S - qt * 128, 64, p.vec_ok_c);
+        stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, 0, p.S - qt * 128, 64, p.vec_ok_c);
+        stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, 32, p.S - qt * 128, 64, p.vec_ok_c);
         if (pg != nullptr)
-          for (int n0 = g * 32; n0 < p.S; n0 += 64)
+          for (int n0 = 0; n0 < p.S; n0 += 32)
             stage_store_bf16(stg, lane, v[0], pg, p.S, q * 32, n0, p.S - qt * 128, p.S, p.vec_ok_p);
         continue;
       }
       const int nkb = (len + 127) >> 7;
-      const uint32_t ipar = ip & 1;
-      ip++;
-      // reads this group's next score block into v, masks it; returns its row maximum
-      auto load_block = [&](uint32_t tt, int j, float& bm) -> bool {
-        if (!mbar_wait(smem_u32(&sfull_bar[g]), (tt >> 1) & 1, abort_flag, p.status)) return false;
+      // reads the group's next score block into v, masks it; returns its row maximum
+      auto load_block = [&](int j, float& bm) -> bool {
+        if (!mbar_wait(sfull, sp & 1, abort_flag, p.status)) return false;
+        sp++;
         tc_fence_after();
         tc_ld128(trow, v);
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&sempty_bar[g]));
+        if (lane == 0) mbar_arrive(sempty);
         float mc[4];
 #pragma unroll
         for (int c = 0; c < 4; c++) {
@@ -611,55 +626,56 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         bm = fmaxf(fmaxf(mc[0], mc[1]), fmaxf(mc[2], mc[3]));
         return true;
       };
-      // pass 1: running maximum (raw scores) and sum of 2^((s - max) * scale * log2 e)
+      // pass 1: running maximum of the raw scores; with probabilities wanted also the running sum
+      // of 2^((s - max) * scale * log2 e)
       float mr = -INFINITY, l = 0.f;
-      for (int j = 0; j < nkb && ok; j++, t++) {
-        if ((t & 1) != (uint32_t)g) continue;
+      for (int j = 0; j < nkb && ok; j++) {
         float bm;
-        if (!load_block(t, j, bm)) { ok = false; break; }
+        if (!load_block(j, bm)) { ok = false; break; }
         const float mn = fmaxf(mr, bm);
-        if (mn == -INFINITY) continue;  // nothing valid so far
-        const float2 nm2 = splat2(-mn * sl2);
-        float2 sc[4];
+        if (want_p && mn != -INFINITY) {
+          const float2 nm2 = splat2(-mn * sl2);
+          float2 sc[4];
 #pragma unroll
-        for (int c = 0; c < 4; c++) {
-          sc[c] = make_float2(0.f, 0.f);
+          for (int c = 0; c < 4; c++) {
+            sc[c] = make_float2(0.f, 0.f);
 #pragma unroll
-          for (int e = 0; e < 16; e++) {
-            const float2 a = __ffma2_rn(v[c][e], k2, nm2);
-            sc[c] = __fadd2_rn(sc[c], make_float2(fast_exp2(a.x), fast_exp2(a.y)));
+            for (int e = 0; e < 16; e++) {
+              const float2 a = __ffma2_rn(v[c][e], k2, nm2);
+              sc[c] = __fadd2_rn(sc[c], make_float2(fast_exp2(a.x), fast_exp2(a.y)));
+            }
           }
+          const float bs = ((sc[0].x + sc[0].y) + (sc[1].x + sc[1].y)) + ((sc[2].x + sc[2].y) + (sc[3].x + sc[3].y));
+          l = l * fast_exp2((mr - mn) * sl2) + bs;  // 2^(-inf) = 0 on the first valid block
         }
-        const float bs = ((sc[0].x + sc[0].y) + (sc[1].x + sc[1].y)) + ((sc[2].x + sc[2].y) + (sc[3].x + sc[3].y));
-        l = l * fast_exp2((mr - mn) * sl2) + bs;  // 2^(-inf) = 0 on the first valid block
         mr = mn;
       }
       if (!ok) break;
-      // exchange with the other group
-      float2* xs = xstat + (ipar * 2) * 128;
-      xs[g * 128 + r] = make_float2(mr, l);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(x_bar));
-      if (!mbar_wait(smem_u32(x_bar), ipar, abort_flag, p.status)) { ok = false; break; }
-      const float2 other = xs[(g ^ 1) * 128 + r];
-      const float M = fmaxf(mr, other.x);  // finite: at least one key of the row is valid
-      const float L = l * fast_exp2((mr - M) * sl2) + other.y * fast_exp2((other.x - M) * sl2);
-      const float2 inv = splat2(1.0f / L), nM2 = splat2(-M * sl2);
+      // mr is finite: at least one key of the row is valid
+      const float2 nM2 = splat2(-mr * sl2);
+      const float2 inv = splat2(want_p ? 1.0f / l : 1.0f);
+      float2 ls = make_float2(0.f, 0.f);  // without stored probabilities: the sum, formed in pass 2
       // pass 2
-      for (int j = 0; j < nkb && ok; j++, t++) {
-        if ((t & 1) != (uint32_t)g) { u++; continue; }
+      for (int j = 0; j < nkb && ok; j++) {
         float bm;
-        if (!load_block(t, j, bm)) { ok = false; break; }
+        if (!load_block(j, bm)) { ok = false; break; }
 #pragma unroll
         for (int c = 0; c < 4; c++)
 #pragma unroll
           for (int e = 0; e < 16; e++) {
             const float2 a = __ffma2_rn(v[c][e], k2, nM2);
-            v[c][e] = __fmul2_rn(make_float2(fast_exp2(a.x), fast_exp2(a.y)), inv);
+            const float2 ex = make_float2(fast_exp2(a.x), fast_exp2(a.y));
+            if (want_p) {
+              v[c][e] = __fmul2_rn(ex, inv);
+            } else {
+              v[c][e] = ex;
+              ls = __fadd2_rn(ls, ex);
+            }
           }
-        // the single P block is free once the previous second product has read it
-        if (!mbar_wait(smem_u32(pfree_bar), (u & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
-        uint8_t* prow = p_smem + r * 128;
+        // the group's P block is free once its previous second product has read it
+        if (!mbar_wait(pfree, (pv & 1) ^ 1, abort_flag, p.status)) { ok = false; break; }
+        pv++;
+        uint8_t* prow = my_p + r * 128;
 #pragma unroll
         for (int c = 0; c < 4; c++)
 #pragma unroll
@@ -672,8 +688,7 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
           }
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
         __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(pready_bar));
-        u++;
+        if (lane == 0) mbar_arrive(pready);
         if (pg != nullptr) {
           if (p.fast_p) {
             if (qt * 128 + r < p.S) {
@@ -690,25 +705,39 @@ attn_fwd_long_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_const
         }
       }
       if (!ok) break;
-      // context tile: this group stores 32 of its 64 columns
-      // key blocks past the length: their probabilities are 0 (this group zeroes its half of the columns)
+      // key blocks past the length: their probabilities are 0
       if (pg != nullptr && nkb * 128 < p.S) {
         float2 zr[16];
 #pragma unroll
         for (int e = 0; e < 16; e++) zr[e] = make_float2(0.f, 0.f);
-        for (int n0 = nkb * 128 + g * 32; n0 < p.S; n0 += 64)
+        for (int n0 = nkb * 128; n0 < p.S; n0 += 32)
           stage_store_bf16(stg, lane, zr, pg, p.S, q * 32, n0, p.S - qt * 128, p.S, p.vec_ok_p);
       }
-      if (!mbar_wait(smem_u32(ofull_bar), ipar, abort_flag, p.status)) { ok = false; break; }
+      // context tile: the row's 64 columns
+      if (!mbar_wait(ofull, ig & 1, abort_flag, p.status)) { ok = false; break; }
+      ig++;
       tc_fence_after();
-      tc_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + AT_O_COL + (uint32_t)g * 32, v[0]);
+      tc_ld32(orow, v[0]);
+      tc_ld32(orow + 32, v[1]);
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_u32(oempty_bar));
+      if (lane == 0) mbar_arrive(oempty);
+      if (!want_p) {
+        const float2 il = splat2(1.0f / (ls.x + ls.y));
+#pragma unroll
+        for (int e = 0; e < 16; e++) {
+          v[0][e] = __fmul2_rn(v[0][e], il);
+          v[1][e] = __fmul2_rn(v[1][e], il);
+        }
+      }
       if (p.fast_c) {
-        if (qt * 128 + r < p.S) store_row32_bf16(cg + (long long)r * p.c_ld + g * 32, v[0]);
+        if (qt * 128 + r < p.S) {
+          store_row32_bf16(cg + (long long)r * p.c_ld, v[0]);
+          store_row32_bf16(cg + (long long)r * p.c_ld + 32, v[1]);
+        }
       } else {
-        stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, g * 32, p.S - qt * 128, 64, p.vec_ok_c);
+        stage_store_bf16(stg, lane, v[0], cg, p.c_ld, q * 32, 0, p.S - qt * 128, 64, p.vec_ok_c);
+        stage_store_bf16(stg, lane, v[1], cg, p.c_ld, q * 32, 32, p.S - qt * 128, 64, p.vec_ok_c);
       }
     }
   }
@@ -1094,13 +1123,13 @@ int attn_fwd_launch(const void* qkv, void* probs, void* ctx, const int* seq_lens
   if (rc) return rc;
   for (int i = 0; i < 3; i++) { p.q_perm[i] = mq.perm[i]; p.k_perm[i] = mk.perm[i]; p.v_perm[i] = mv.perm[i]; }
   if (long_rows) {
-    const size_t smem_long = 2 * (size_t)AT_TILE_BYTES + (size_t)AL_KV_STAGES * AL_KV_BYTES + AL_P_BYTES +
-                             NUM_EPI_WARPS * AT_STAGING + 2 * 2 * 128 * sizeof(float2) + 1024 + 256;
+    const size_t smem_long = 2 * (size_t)AT_TILE_BYTES + 2 * (size_t)AL_RING * AT_TILE_BYTES + 2 * (size_t)AL_P_BYTES +
+                             NUM_EPI_WARPS * AT_STAGING + 1024 + 512;
     if ((int)smem_long > smem_optin) { snprintf(err, 256, "attention: not enough shared memory"); return MSLT_ERR_CUDA; }
     rc = attn_opt_in(attn_fwd_long_kernel, &adev->attr_long, smem_optin, err);
     if (rc) return rc;
     const int grid_long = p.items < num_sms ? p.items : num_sms;
-    attn_fwd_long_kernel<<<grid_long, NUM_THREADS, smem_long, st>>>(mq.map, mk.map, mv.map, p);
+    attn_fwd_long_kernel<<<grid_long, AL_THREADS, smem_long, st>>>(mq.map, mk.map, mv.map, p);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) { snprintf(err, 256, "attention: launch failed: %s", cudaGetErrorString(e)); return MSLT_ERR_CUDA; }
     g_attn_launches++;
